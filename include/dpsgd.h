@@ -1,0 +1,176 @@
+/*
+ * dpsgd.h - C ABI of the B200 D-PSGD library (libdpsgd.so).
+ *
+ * D-PSGD (Lian et al., "Can Decentralized Algorithms Outperform Centralized Algorithms?",
+ * arXiv 1705.09056) simulated for n nodes on ONE GPU.  The n local models x_{k,i} are the
+ * rows of an n x ld fp32 matrix X (the paper's X_k in R^{N x n} of Section 3, stored
+ * transposed; W is symmetric, so X_k W becomes W X).  One iteration k of Algorithm 1 is
+ *
+ *     xi_{k,i}  <- minibatch of B indices into node i's local data        (step 2)
+ *     g_i       <- (1/B) sum_b grad F(x_{k,i}; sample_b)                   (step 3, footnote a)
+ *     x_{k+1,i} <- sum_j W_ij x_{k,j} - gamma g_i                          (steps 4-5)
+ *
+ * i.e. the global form X_{k+1} = X_k W - gamma dF(X_k; xi_k) of Section 3.
+ *
+ * Conventions
+ *  - Every function returns a dpsgd_status; nothing throws, aborts or traps.
+ *    dpsgd_last_error() gives a human-readable message for the last failure on a context.
+ *  - "host" pointers are ordinary CPU memory, "device" pointers are CUDA global memory of the
+ *    current device.  Big buffers (X, G, the dataset) are owned by the CALLER and must stay
+ *    alive while bound; the library owns only small internals (CSR copy, index and activation
+ *    scratch, reduction partials), released by dpsgd_destroy().
+ *  - All work is enqueued on the stream given to dpsgd_bind(); calls return without waiting
+ *    unless stated otherwise.  Calls on one context must not overlap in time.
+ *  - There is no CPU fallback: without a CUDA device every compute call fails with
+ *    DPSGD_ERR_CUDA.
+ *
+ * Stacked layout: row i of X / G starts at element i*ld; ld >= N, ld a multiple of 32 floats
+ * (128 bytes), base pointers 128-byte aligned.  Padding columns [N, ld) must be zero in X and
+ * G on entry; they stay zero (rows of W sum to one, applied to zeros).
+ */
+#ifndef DPSGD_H_
+#define DPSGD_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define DPSGD_API __attribute__((visibility("default")))
+#else
+#define DPSGD_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dpsgd_ctx dpsgd_ctx; /* opaque, library-owned */
+
+typedef enum dpsgd_status {
+    DPSGD_OK = 0,
+    DPSGD_ERR_ARG = 1,         /* null pointer, non-positive size, value out of range           */
+    DPSGD_ERR_W_INVALID = 2,   /* W is not a symmetric doubly stochastic matrix in sorted CSR    */
+    DPSGD_ERR_ALIGN = 3,       /* pointer or leading dimension not aligned as required           */
+    DPSGD_ERR_STATE = 4,       /* call made before the buffers / model / data it needs were set  */
+    DPSGD_ERR_UNSUPPORTED = 5, /* shape outside what the kernels handle                          */
+    DPSGD_ERR_CUDA = 6,        /* a CUDA runtime call or kernel launch failed                    */
+    DPSGD_ERR_TIMEOUT = 7      /* a bounded device-side wait gave up (status word set by kernel) */
+} dpsgd_status;
+
+enum { DPSGD_MODEL_LSQ = 0, DPSGD_MODEL_LOGISTIC = 1, DPSGD_MODEL_MLP = 2 };
+
+/* Mixing kernel chosen from the structure of W (reported by dpsgd_mix_kind). */
+enum {
+    DPSGD_MIX_RING = 0,          /* circulant tridiagonal band (Theorem 3's ring)               */
+    DPSGD_MIX_UNIFORM_DENSE = 1, /* all n*n entries equal (W = 1 1^T / n, the C-PSGD average)   */
+    DPSGD_MIX_TILED_CSR = 2,     /* any sparse W: column tiles of all n rows staged on chip      */
+    DPSGD_MIX_GATHER_CSR = 3     /* any W: neighbour rows gathered through the caches            */
+};
+
+/*
+ * Inputs of Algorithm 1 ("Require: step length gamma, weight matrix W"): creates a context
+ * for n nodes with N parameters each.  W comes as host CSR (row_ptr[n+1], col_idx[nnz],
+ * val[nnz]); it is validated against Section 3's definition and copied:
+ *   square; column indices in range, strictly increasing inside a row; 0 <= W_ij <= 1;
+ *   W_ij == W_ji exactly; |sum_j W_ij - 1| <= 1e-6 for every row.
+ * Otherwise DPSGD_ERR_W_INVALID and *out = NULL (nothing is left allocated).
+ * seed keys the minibatch sampler.  Limits: 1 <= n <= 65535, 1 <= N < 2^40.
+ */
+DPSGD_API dpsgd_status dpsgd_create(dpsgd_ctx** out, int32_t n, int64_t N, const int32_t* row_ptr_host,
+                          const int32_t* col_idx_host, const float* val_host, float gamma,
+                          uint64_t seed);
+
+/* Releases the context and its internal device memory.  Caller-owned buffers are untouched. */
+DPSGD_API dpsgd_status dpsgd_destroy(dpsgd_ctx* ctx);
+
+/*
+ * Binds the caller's device buffers: X0 holds X_k now, X1 receives X_{k+1} (they swap roles
+ * each mix_update), G holds the stochastic gradients dF(X_k; xi_k) (Section 3).  All three are
+ * n x ld fp32, 128-byte aligned, distinct and non-overlapping.  cuda_stream is a cudaStream_t
+ * (NULL = legacy default stream).  May be called again to rebind.
+ */
+DPSGD_API dpsgd_status dpsgd_bind(dpsgd_ctx* ctx, float* X0_dev, float* X1_dev, float* G_dev, int64_t ld,
+                        void* cuda_stream);
+
+/*
+ * Chooses F of Eq. (1)/(2).  dims/ndims:
+ *   DPSGD_MODEL_LSQ      dims = {d}: F = 1/2 (a.x - y)^2,                       N = d
+ *   DPSGD_MODEL_LOGISTIC dims = {d}: F = log(1+exp(-y(a.w+b))) + l2/2 |w|^2,    N = d+1, x=[w|b]
+ *   DPSGD_MODEL_MLP      dims = {d_0,...,d_L}: ReLU layers, softmax cross-entropy,
+ *                        x = [W_1 (d_1 x d_0 row-major) | b_1 | W_2 | b_2 ...], N = sum
+ * batch = minibatch size B per node (footnote a of Algorithm 1; gradients are the MEAN over
+ * the minibatch).  N must match the context's N.  Allocates the activation scratch.
+ * mlp_precision: 0 = fp32-faithful (3xTF32 split on tensor cores or fp32 FMA), 1 = single
+ * TF32 pass (faster, ~1e-3 relative on G).  Ignored for the linear models.
+ */
+DPSGD_API dpsgd_status dpsgd_set_model(dpsgd_ctx* ctx, int32_t kind, const int32_t* dims_host,
+                             int32_t ndims, float l2_lambda, int32_t batch,
+                             int32_t mlp_precision);
+
+/*
+ * Local data of the n nodes (Section 3, Strategy 1/2): A_dev is fp32 [n][m_per_node][d],
+ * y_dev is fp32 [n][m_per_node] (targets, or labels +-1) for the linear models and int32
+ * [n][m_per_node] class ids for the MLP.  Caller-owned, 16-byte aligned, d = dims[0].
+ */
+DPSGD_API dpsgd_status dpsgd_set_data(dpsgd_ctx* ctx, const float* A_dev, const void* y_dev,
+                            int64_t m_per_node, int32_t d);
+
+/*
+ * Algorithm 1 step 2 on its own (test hook): writes the indices xi_{k,i} of iteration k,
+ * int32 [n][B] on the device.  Draw b of node i is word (b mod 4) of Philox4x32-10 with
+ * counter (b div 4, i, k_lo, k_hi) and key (seed_lo, seed_hi), mapped to
+ * floor(u * m_per_node / 2^32): i.i.d. uniform with replacement.
+ */
+DPSGD_API dpsgd_status dpsgd_sample(dpsgd_ctx* ctx, uint64_t k, int32_t* idx_dev);
+
+/* Algorithm 1 steps 2-3 for all nodes: G <- dF(X_k; xi_k), gradients at the nodes' own rows. */
+DPSGD_API dpsgd_status dpsgd_grad(dpsgd_ctx* ctx, uint64_t k);
+
+/*
+ * Algorithm 1 steps 4-5 fused, one pass over HBM: X_next <- W X_cur - gamma G, then the two X
+ * buffers swap roles.  Reads X and G once and writes X_next once (12 bytes per
+ * replica-parameter).
+ */
+DPSGD_API dpsgd_status dpsgd_mix_update(dpsgd_ctx* ctx);
+
+/* One full iteration k of Algorithm 1: dpsgd_grad(k) followed by dpsgd_mix_update(). */
+DPSGD_API dpsgd_status dpsgd_step(dpsgd_ctx* ctx, uint64_t k);
+
+/*
+ * sum_i || xbar - x_i ||^2 over the current X (sum_i Q_{k,i} of Eq. 10; divide by n for M_k
+ * of Eq. 13), accumulated in fp64.  Waits for the stream and writes one double to host memory.
+ */
+DPSGD_API dpsgd_status dpsgd_consensus_dist(dpsgd_ctx* ctx, double* out_host);
+
+/* Output of Algorithm 1: xbar = (1/n) sum_i x_i into xbar_dev (fp32 [ld], 16-byte aligned). */
+DPSGD_API dpsgd_status dpsgd_average(dpsgd_ctx* ctx, float* xbar_dev);
+
+/*
+ * Host-buffer variant of the gossip step, for callers whose gradients live in CPU memory:
+ * copies G_host (n rows of N floats, row stride ld_host >= N elements; pinned memory makes the
+ * copy asynchronous) into the bound G, runs dpsgd_mix_update(), evaluates the consensus
+ * distance of the new X, waits, and writes it to *consensus_out_host.
+ */
+DPSGD_API dpsgd_status dpsgd_mix_update_host(dpsgd_ctx* ctx, const float* G_host, int64_t ld_host,
+                                   double* consensus_out_host);
+
+/* Device pointer of the buffer that currently holds X_k (one of the two bound buffers). */
+DPSGD_API dpsgd_status dpsgd_current(dpsgd_ctx* ctx, float** X_cur_dev);
+
+/* Step length gamma of Algorithm 1; may change between iterations (schedules). */
+DPSGD_API dpsgd_status dpsgd_set_gamma(dpsgd_ctx* ctx, float gamma);
+
+/* Which DPSGD_MIX_* kernel the structure of W selected; force >= 0 overrides it when the
+ * requested kernel can handle W (else DPSGD_ERR_UNSUPPORTED).  Pass force = -1 to query. */
+DPSGD_API dpsgd_status dpsgd_mix_kind(dpsgd_ctx* ctx, int32_t force, int32_t* kind_out);
+
+/* Number of kernels this context has launched so far (for launch accounting). */
+DPSGD_API dpsgd_status dpsgd_launch_count(dpsgd_ctx* ctx, int64_t* count_out);
+
+/* Message for the last non-OK status on ctx (never NULL; valid until the next call on ctx).
+ * With ctx == NULL, the message of the last failed dpsgd_create() on this thread. */
+DPSGD_API const char* dpsgd_last_error(dpsgd_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DPSGD_H_ */

@@ -1,0 +1,415 @@
+// C ABI of libdpsgd: argument checking, validation of W, context state and dispatch.
+// No arithmetic of the method lives here; every step runs in the kernels of the other files.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "ctx.h"
+
+using namespace dpsgd;
+
+namespace {
+
+thread_local std::string g_create_error = "";
+
+dpsgd_status fail(dpsgd_ctx* c, dpsgd_status s, const std::string& msg) {
+    if (c) c->err = msg; else g_create_error = msg;
+    return s;
+}
+
+dpsgd_status cuda_fail(dpsgd_ctx* c, cudaError_t e, const char* what) {
+    return fail(c, DPSGD_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+// Section 3: W symmetric, doubly stochastic, entries in [0,1]; CSR rows sorted and unique.
+bool validate_w(int n, const int32_t* rp, const int32_t* col, const float* val, std::string* why) {
+    char buf[160];
+    if (rp[0] != 0) { *why = "row_ptr[0] != 0"; return false; }
+    for (int i = 0; i < n; ++i) {
+        if (rp[i + 1] < rp[i]) { *why = "row_ptr not non-decreasing"; return false; }
+        if (rp[i + 1] - rp[i] > n) { *why = "row with more than n entries"; return false; }
+    }
+    for (int i = 0; i < n; ++i) {
+        double sum = 0.0;
+        for (int p = rp[i]; p < rp[i + 1]; ++p) {
+            const int j = col[p];
+            if (j < 0 || j >= n) {
+                snprintf(buf, sizeof buf, "row %d: column %d out of range", i, j);
+                *why = buf; return false;
+            }
+            if (p > rp[i] && col[p - 1] >= j) {
+                snprintf(buf, sizeof buf, "row %d: columns not strictly increasing", i);
+                *why = buf; return false;
+            }
+            const float v = val[p];
+            if (!(v >= 0.f && v <= 1.f)) {
+                snprintf(buf, sizeof buf, "W[%d][%d] = %g outside [0,1]", i, j, (double)v);
+                *why = buf; return false;
+            }
+            sum += (double)v;
+        }
+        if (std::fabs(sum - 1.0) > 1e-6) {
+            snprintf(buf, sizeof buf, "row %d sums to %.9g, not 1", i, sum);
+            *why = buf; return false;
+        }
+    }
+    for (int i = 0; i < n; ++i) {
+        for (int p = rp[i]; p < rp[i + 1]; ++p) {
+            const int j = col[p];
+            const int32_t* b = col + rp[j];
+            const int32_t* e = col + rp[j + 1];
+            const int32_t* it = std::lower_bound(b, e, i);
+            const float mirror = (it != e && *it == i) ? val[it - col] : 0.f;
+            if (mirror != val[p]) {
+                snprintf(buf, sizeof buf, "W[%d][%d] = %g but W[%d][%d] = %g (not symmetric)", i, j,
+                         (double)val[p], j, i, (double)mirror);
+                *why = buf; return false;
+            }
+        }
+    }
+    return true;
+}
+
+void classify_w(dpsgd_ctx* c) {
+    const int n = c->n;
+    const auto& rp = c->h_row_ptr;
+    const auto& col = c->h_col;
+    const auto& val = c->h_val;
+    int max_deg = 0;
+    for (int i = 0; i < n; ++i) max_deg = std::max(max_deg, rp[i + 1] - rp[i]);
+    c->W.max_deg = max_deg;
+
+    bool uniform = (int64_t)rp[n] == (int64_t)n * n;
+    if (uniform)
+        for (size_t p = 1; p < val.size() && uniform; ++p)
+            uniform = (memcmp(&val[p], &val[0], sizeof(float)) == 0);
+    c->can_uniform = uniform;
+    if (uniform) c->W.uniform = val[0];
+
+    bool ringlike = n >= 3;
+    for (int i = 0; i < n && ringlike; ++i) {
+        if (rp[i + 1] - rp[i] != 3) { ringlike = false; break; }
+        int want[3] = {(i + n - 1) % n, i, (i + 1) % n};
+        std::sort(want, want + 3);
+        for (int t = 0; t < 3; ++t)
+            if (col[rp[i] + t] != want[t]) ringlike = false;
+    }
+    c->can_ring = ringlike;
+    c->can_tiled = mix_tiled_supported(c);
+
+    if (uniform && n != 3) c->mix_kind = DPSGD_MIX_UNIFORM_DENSE;
+    else if (ringlike) c->mix_kind = DPSGD_MIX_RING;
+    else if (uniform) c->mix_kind = DPSGD_MIX_UNIFORM_DENSE;
+    else if (c->can_tiled) c->mix_kind = DPSGD_MIX_TILED_CSR;
+    else c->mix_kind = DPSGD_MIX_GATHER_CSR;
+}
+
+float band_entry(const dpsgd_ctx* c, int i, int j) {
+    for (int p = c->h_row_ptr[i]; p < c->h_row_ptr[i + 1]; ++p)
+        if (c->h_col[p] == j) return c->h_val[p];
+    return 0.f;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+void release(dpsgd_ctx* c) {
+    if (!c) return;
+    mix_tiled_release(c);
+    cudaFree(c->d_w_blob);
+    cudaFree(c->d_idx);
+    cudaFree(c->d_coef);
+    cudaFree(c->d_act);
+    cudaFree(c->d_delta);
+    cudaFree(c->d_partials);
+    cudaFree(c->d_result);
+    if (c->h_result) cudaFreeHost(c->h_result);
+    delete c;
+}
+
+dpsgd_status need_bound(dpsgd_ctx* c) {
+    if (!c) return DPSGD_ERR_ARG;
+    if (!c->bound) return fail(c, DPSGD_ERR_STATE, "no buffers bound: call dpsgd_bind first");
+    return DPSGD_OK;
+}
+
+dpsgd_status need_model(dpsgd_ctx* c) {
+    if (c->model < 0) return fail(c, DPSGD_ERR_STATE, "no model: call dpsgd_set_model first");
+    if (!c->have_data) return fail(c, DPSGD_ERR_STATE, "no data: call dpsgd_set_data first");
+    return DPSGD_OK;
+}
+
+cudaError_t run_mix(dpsgd_ctx* c) {
+    const float* X = c->X[c->cur];
+    float* Xn = c->X[c->cur ^ 1];
+    switch (c->mix_kind) {
+        case DPSGD_MIX_RING: return launch_mix_ring(c, X, c->G, Xn);
+        case DPSGD_MIX_UNIFORM_DENSE: return launch_mix_uniform(c, X, c->G, Xn);
+        case DPSGD_MIX_TILED_CSR: return launch_mix_tiled(c, X, c->G, Xn);
+        default: return launch_mix_gather(c, X, c->G, Xn);
+    }
+}
+
+cudaError_t run_grad(dpsgd_ctx* c, uint64_t k) {
+    if (c->model == DPSGD_MODEL_MLP) return launch_grad_mlp(c, k, c->X[c->cur], c->G);
+    return launch_grad_linear(c, k, c->X[c->cur], c->G);
+}
+
+}  // namespace
+
+extern "C" {
+
+DPSGD_API dpsgd_status dpsgd_create(dpsgd_ctx** out, int32_t n, int64_t N, const int32_t* row_ptr,
+                          const int32_t* col_idx, const float* val, float gamma, uint64_t seed) {
+    if (!out) return fail(nullptr, DPSGD_ERR_ARG, "out is NULL");
+    *out = nullptr;
+    if (n < 1 || n > 65535) return fail(nullptr, DPSGD_ERR_ARG, "n must be in [1, 65535]");
+    if (N < 1 || N >= (int64_t(1) << 40)) return fail(nullptr, DPSGD_ERR_ARG, "N must be in [1, 2^40)");
+    if (!row_ptr || !col_idx || !val) return fail(nullptr, DPSGD_ERR_ARG, "CSR pointer is NULL");
+    if (!(gamma == gamma)) return fail(nullptr, DPSGD_ERR_ARG, "gamma is NaN");
+    std::string why;
+    if (!validate_w(n, row_ptr, col_idx, val, &why)) return fail(nullptr, DPSGD_ERR_W_INVALID, why);
+
+    dpsgd_ctx* c = new (std::nothrow) dpsgd_ctx();
+    if (!c) return fail(nullptr, DPSGD_ERR_ARG, "out of host memory");
+    c->n = n; c->N = N; c->gamma = gamma; c->seed = seed;
+    const int nnz = row_ptr[n];
+    c->h_row_ptr.assign(row_ptr, row_ptr + n + 1);
+    c->h_col.assign(col_idx, col_idx + nnz);
+    c->h_val.assign(val, val + nnz);
+    c->W.n = n; c->W.nnz = nnz;
+
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e != cudaSuccess) { auto s = cuda_fail(nullptr, e, "cudaGetDevice"); release(c); return s; }
+    classify_w(c);
+
+    // one blob: row_ptr | col | val | band
+    const size_t o_rp = 0;
+    const size_t o_col = (o_rp + sizeof(int32_t) * (n + 1) + 255) / 256 * 256;
+    const size_t o_val = (o_col + sizeof(int32_t) * nnz + 255) / 256 * 256;
+    const size_t o_band = (o_val + sizeof(float) * nnz + 255) / 256 * 256;
+    const size_t total = o_band + sizeof(float) * 3 * n;
+    std::vector<char> blob(total, 0);
+    memcpy(blob.data() + o_rp, row_ptr, sizeof(int32_t) * (n + 1));
+    memcpy(blob.data() + o_col, col_idx, sizeof(int32_t) * nnz);
+    memcpy(blob.data() + o_val, val, sizeof(float) * nnz);
+    if (c->can_ring) {
+        float* band = reinterpret_cast<float*>(blob.data() + o_band);
+        for (int i = 0; i < n; ++i) {
+            band[3 * i + 0] = band_entry(c, i, (i + n - 1) % n);
+            band[3 * i + 1] = band_entry(c, i, i);
+            band[3 * i + 2] = band_entry(c, i, (i + 1) % n);
+        }
+    }
+    e = cudaMalloc(&c->d_w_blob, total);
+    if (e == cudaSuccess) e = cudaMemcpy(c->d_w_blob, blob.data(), total, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_result, sizeof(double));
+    if (e == cudaSuccess) e = cudaMallocHost(&c->h_result, sizeof(double));
+    if (e != cudaSuccess) { auto s = cuda_fail(nullptr, e, "dpsgd_create allocation"); release(c); return s; }
+    char* base = static_cast<char*>(c->d_w_blob);
+    c->W.row_ptr = reinterpret_cast<int32_t*>(base + o_rp);
+    c->W.col = reinterpret_cast<int32_t*>(base + o_col);
+    c->W.val = reinterpret_cast<float*>(base + o_val);
+    c->W.band = reinterpret_cast<float*>(base + o_band);
+    *out = c;
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_destroy(dpsgd_ctx* c) {
+    if (!c) return DPSGD_ERR_ARG;
+    if (c->bound) cudaStreamSynchronize(c->stream);
+    release(c);
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_bind(dpsgd_ctx* c, float* X0, float* X1, float* G, int64_t ld, void* stream) {
+    if (!c) return DPSGD_ERR_ARG;
+    if (!X0 || !X1 || !G) return fail(c, DPSGD_ERR_ARG, "buffer pointer is NULL");
+    if (ld < c->N) return fail(c, DPSGD_ERR_ARG, "ld < N");
+    if (ld % 32 != 0) return fail(c, DPSGD_ERR_ALIGN, "ld must be a multiple of 32 floats");
+    if (!aligned(X0, 128) || !aligned(X1, 128) || !aligned(G, 128))
+        return fail(c, DPSGD_ERR_ALIGN, "X0, X1 and G must be 128-byte aligned");
+    const uintptr_t bytes = (uintptr_t)c->n * (uintptr_t)ld * sizeof(float);
+    const uintptr_t p[3] = {(uintptr_t)X0, (uintptr_t)X1, (uintptr_t)G};
+    for (int a = 0; a < 3; ++a)
+        for (int b = a + 1; b < 3; ++b)
+            if (p[a] < p[b] + bytes && p[b] < p[a] + bytes)
+                return fail(c, DPSGD_ERR_ARG, "X0, X1 and G must not overlap");
+    c->X[0] = X0; c->X[1] = X1; c->G = G; c->cur = 0; c->ld = ld;
+    c->stream = static_cast<cudaStream_t>(stream);
+    c->bound = true;
+    mix_tiled_release(c);  // tensor maps depend on the bound pointers
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_set_model(dpsgd_ctx* c, int32_t kind, const int32_t* dims, int32_t ndims,
+                             float l2_lambda, int32_t batch, int32_t mlp_precision) {
+    if (!c) return DPSGD_ERR_ARG;
+    if (!dims || ndims < 1) return fail(c, DPSGD_ERR_ARG, "dims missing");
+    if (batch < 1 || batch > 4096) return fail(c, DPSGD_ERR_ARG, "batch must be in [1, 4096]");
+    for (int t = 0; t < ndims; ++t)
+        if (dims[t] < 1) return fail(c, DPSGD_ERR_ARG, "non-positive layer width");
+    int64_t want = 0;
+    MlpShape shape;
+    if (kind == DPSGD_MODEL_LSQ) {
+        if (ndims != 1) return fail(c, DPSGD_ERR_ARG, "least squares takes dims = {d}");
+        want = dims[0];
+    } else if (kind == DPSGD_MODEL_LOGISTIC) {
+        if (ndims != 1) return fail(c, DPSGD_ERR_ARG, "logistic regression takes dims = {d}");
+        want = (int64_t)dims[0] + 1;
+    } else if (kind == DPSGD_MODEL_MLP) {
+        if (ndims < 2 || ndims - 1 > kMaxLayers)
+            return fail(c, DPSGD_ERR_UNSUPPORTED, "MLP needs 1..8 weight layers");
+        shape.nlayers = ndims - 1;
+        for (int t = 0; t < ndims; ++t) shape.dims[t] = dims[t];
+        for (int l = 0; l < shape.nlayers; ++l) {
+            shape.w_off[l] = want; want += (int64_t)dims[l + 1] * dims[l];
+            shape.b_off[l] = want; want += dims[l + 1];
+        }
+    } else {
+        return fail(c, DPSGD_ERR_ARG, "unknown model kind");
+    }
+    if (want != c->N) {
+        char buf[128];
+        snprintf(buf, sizeof buf, "model has %lld parameters but the context was created with N = %lld",
+                 (long long)want, (long long)c->N);
+        return fail(c, DPSGD_ERR_ARG, buf);
+    }
+    if (c->bound) cudaStreamSynchronize(c->stream);
+    cudaFree(c->d_idx); cudaFree(c->d_coef); cudaFree(c->d_act); cudaFree(c->d_delta);
+    c->d_idx = nullptr; c->d_coef = nullptr; c->d_act = nullptr; c->d_delta = nullptr;
+    c->model = kind; c->d = dims[0]; c->batch = batch; c->l2 = l2_lambda; c->mlp = shape;
+    c->mlp_precision = mlp_precision;
+    cudaError_t e = cudaMalloc(&c->d_idx, sizeof(int32_t) * (size_t)c->n * batch);
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_coef, sizeof(float) * (size_t)c->n * batch);
+    if (e == cudaSuccess && kind == DPSGD_MODEL_MLP) {
+        c->act_floats = mlp_act_floats(c);
+        c->delta_floats = mlp_delta_floats(c);
+        e = cudaMalloc(&c->d_act, sizeof(float) * c->act_floats);
+        if (e == cudaSuccess) e = cudaMalloc(&c->d_delta, sizeof(float) * c->delta_floats);
+    }
+    if (e != cudaSuccess) { c->model = -1; return cuda_fail(c, e, "dpsgd_set_model allocation"); }
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_set_data(dpsgd_ctx* c, const float* A, const void* y, int64_t m, int32_t d) {
+    if (!c) return DPSGD_ERR_ARG;
+    if (c->model < 0) return fail(c, DPSGD_ERR_STATE, "call dpsgd_set_model before dpsgd_set_data");
+    if (!A || !y) return fail(c, DPSGD_ERR_ARG, "data pointer is NULL");
+    if (m < 1 || m >= (int64_t(1) << 31)) return fail(c, DPSGD_ERR_ARG, "m_per_node must be in [1, 2^31)");
+    if (d != c->d) return fail(c, DPSGD_ERR_ARG, "d does not match the model's input width");
+    if (!aligned(A, 16) || !aligned(y, 16)) return fail(c, DPSGD_ERR_ALIGN, "A and y must be 16-byte aligned");
+    c->A = A; c->y = y; c->m = m; c->have_data = true;
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_sample(dpsgd_ctx* c, uint64_t k, int32_t* idx) {
+    if (!c) return DPSGD_ERR_ARG;
+    if (!idx) return fail(c, DPSGD_ERR_ARG, "idx is NULL");
+    if (c->model < 0 || !c->have_data) return fail(c, DPSGD_ERR_STATE, "model and data must be set");
+    cudaError_t e = launch_sample(c, k, idx);
+    return e == cudaSuccess ? DPSGD_OK : cuda_fail(c, e, "sample kernel");
+}
+
+DPSGD_API dpsgd_status dpsgd_grad(dpsgd_ctx* c, uint64_t k) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    if ((s = need_model(c)) != DPSGD_OK) return s;
+    cudaError_t e = run_grad(c, k);
+    return e == cudaSuccess ? DPSGD_OK : cuda_fail(c, e, "gradient kernels");
+}
+
+DPSGD_API dpsgd_status dpsgd_mix_update(dpsgd_ctx* c) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    cudaError_t e = run_mix(c);
+    if (e != cudaSuccess) return cuda_fail(c, e, "mix_update kernel");
+    c->cur ^= 1;
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_step(dpsgd_ctx* c, uint64_t k) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    if ((s = need_model(c)) != DPSGD_OK) return s;
+    cudaError_t e = run_grad(c, k);
+    if (e != cudaSuccess) return cuda_fail(c, e, "gradient kernels");
+    e = run_mix(c);
+    if (e != cudaSuccess) return cuda_fail(c, e, "mix_update kernel");
+    c->cur ^= 1;
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_consensus_dist(dpsgd_ctx* c, double* out) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    if (!out) return fail(c, DPSGD_ERR_ARG, "out_host is NULL");
+    cudaError_t e = launch_consensus(c, c->X[c->cur], c->d_result);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(c->h_result, c->d_result, sizeof(double), cudaMemcpyDeviceToHost, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "consensus distance");
+    *out = *c->h_result;
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_average(dpsgd_ctx* c, float* xbar) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    if (!xbar) return fail(c, DPSGD_ERR_ARG, "xbar_dev is NULL");
+    if (!aligned(xbar, 16)) return fail(c, DPSGD_ERR_ALIGN, "xbar_dev must be 16-byte aligned");
+    cudaError_t e = launch_average(c, c->X[c->cur], xbar);
+    return e == cudaSuccess ? DPSGD_OK : cuda_fail(c, e, "average kernel");
+}
+
+DPSGD_API dpsgd_status dpsgd_mix_update_host(dpsgd_ctx* c, const float* G_host, int64_t ld_host, double* out) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    if (!G_host || !out) return fail(c, DPSGD_ERR_ARG, "G_host or consensus_out_host is NULL");
+    if (ld_host < c->N) return fail(c, DPSGD_ERR_ARG, "ld_host < N");
+    cudaError_t e = cudaMemcpy2DAsync(c->G, sizeof(float) * c->ld, G_host, sizeof(float) * ld_host,
+                                      sizeof(float) * c->N, c->n, cudaMemcpyHostToDevice, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "copy of G to the device");
+    if ((s = dpsgd_mix_update(c)) != DPSGD_OK) return s;
+    return dpsgd_consensus_dist(c, out);
+}
+
+DPSGD_API dpsgd_status dpsgd_current(dpsgd_ctx* c, float** X_cur) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    if (!X_cur) return fail(c, DPSGD_ERR_ARG, "X_cur_dev is NULL");
+    *X_cur = c->X[c->cur];
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_set_gamma(dpsgd_ctx* c, float gamma) {
+    if (!c) return DPSGD_ERR_ARG;
+    if (!(gamma == gamma)) return fail(c, DPSGD_ERR_ARG, "gamma is NaN");
+    c->gamma = gamma;
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_mix_kind(dpsgd_ctx* c, int32_t force, int32_t* kind_out) {
+    if (!c) return DPSGD_ERR_ARG;
+    if (force >= 0) {
+        const bool ok = (force == DPSGD_MIX_RING && c->can_ring) ||
+                        (force == DPSGD_MIX_UNIFORM_DENSE && c->can_uniform) ||
+                        (force == DPSGD_MIX_TILED_CSR && c->can_tiled) ||
+                        force == DPSGD_MIX_GATHER_CSR;
+        if (!ok) return fail(c, DPSGD_ERR_UNSUPPORTED, "this W cannot use the requested mixing kernel");
+        c->mix_kind = force;
+    }
+    if (kind_out) *kind_out = c->mix_kind;
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_launch_count(dpsgd_ctx* c, int64_t* count_out) {
+    if (!c || !count_out) return DPSGD_ERR_ARG;
+    *count_out = c->launches;
+    return DPSGD_OK;
+}
+
+DPSGD_API const char* dpsgd_last_error(dpsgd_ctx* c) { return c ? c->err.c_str() : g_create_error.c_str(); }
+
+}  // extern "C"

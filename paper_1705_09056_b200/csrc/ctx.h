@@ -1,0 +1,107 @@
+// Internal state of a D-PSGD context and the kernel launchers the C ABI dispatches to.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/dpsgd.h"
+
+namespace dpsgd {
+
+constexpr int kMaxLayers = 8;
+
+// Mixing matrix W on the device, as the kernels consume it.
+struct MixW {
+    int n = 0;
+    int nnz = 0;
+    int max_deg = 0;
+    const int32_t* row_ptr = nullptr;  // [n+1]
+    const int32_t* col = nullptr;      // [nnz]
+    const float* val = nullptr;        // [nnz]
+    const float* band = nullptr;       // ring only: [n][3] = (W_{i,i-1}, W_ii, W_{i,i+1})
+    float uniform = 0.f;               // uniform dense only: the common entry
+};
+
+struct MlpShape {
+    int nlayers = 0;                 // number of weight layers L
+    int dims[kMaxLayers + 1] = {0};  // d_0 .. d_L
+    int64_t w_off[kMaxLayers] = {0}; // offset of W_l inside a parameter row
+    int64_t b_off[kMaxLayers] = {0}; // offset of b_l
+};
+
+}  // namespace dpsgd
+
+struct dpsgd_ctx {
+    int n = 0;
+    int64_t N = 0;
+    float gamma = 0.f;
+    uint64_t seed = 0;
+    int device = 0;
+
+    // W
+    std::vector<int32_t> h_row_ptr, h_col;
+    std::vector<float> h_val;
+    dpsgd::MixW W;
+    void* d_w_blob = nullptr;  // one allocation holding row_ptr | col | val | band
+    int mix_kind = DPSGD_MIX_GATHER_CSR;
+    bool can_ring = false, can_uniform = false, can_tiled = false;
+
+    // bound buffers
+    float* X[2] = {nullptr, nullptr};
+    float* G = nullptr;
+    int cur = 0;
+    int64_t ld = 0;
+    cudaStream_t stream = nullptr;
+    bool bound = false;
+
+    // model + data
+    int model = -1;
+    int d = 0;  // input width
+    int batch = 0;
+    float l2 = 0.f;
+    int mlp_precision = 0;
+    dpsgd::MlpShape mlp;
+    const float* A = nullptr;
+    const void* y = nullptr;
+    int64_t m = 0;
+    bool have_data = false;
+
+    // scratch (library-owned)
+    int32_t* d_idx = nullptr;    // [n][B]
+    float* d_coef = nullptr;     // [n][B] per-sample backward coefficients (linear models)
+    float* d_act = nullptr;      // MLP activations h_0..h_L  (see grad_mlp.cu for the layout)
+    float* d_delta = nullptr;    // MLP back-propagated errors
+    size_t act_floats = 0, delta_floats = 0;
+    double* d_partials = nullptr;  // consensus partial sums, one per CTA
+    int partials_cap = 0;
+    double* d_result = nullptr;    // final scalar
+    double* h_result = nullptr;    // pinned
+    void* tma_state = nullptr;     // tensor maps for the tiled mixing kernel
+
+    int64_t launches = 0;
+    std::string err;
+};
+
+namespace dpsgd {
+
+// Each launcher enqueues on ctx->stream, bumps ctx->launches and returns cudaGetLastError().
+cudaError_t launch_mix_ring(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
+cudaError_t launch_mix_uniform(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
+cudaError_t launch_mix_gather(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
+cudaError_t launch_mix_tiled(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
+bool mix_tiled_supported(const dpsgd_ctx* c);
+void mix_tiled_release(dpsgd_ctx* c);
+
+cudaError_t launch_consensus(dpsgd_ctx* c, const float* X, double* result_dev);
+cudaError_t launch_average(dpsgd_ctx* c, const float* X, float* xbar);
+
+cudaError_t launch_sample(dpsgd_ctx* c, uint64_t k, int32_t* idx);
+cudaError_t launch_grad_linear(dpsgd_ctx* c, uint64_t k, const float* X, float* G);
+cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G);
+size_t mlp_act_floats(const dpsgd_ctx* c);
+size_t mlp_delta_floats(const dpsgd_ctx* c);
+
+}  // namespace dpsgd

@@ -1,0 +1,145 @@
+// Algorithm 1 steps 2-3 for the two linear models: every node's minibatch gradient at its own
+// row x_{k,i} (the columns of dF(X_k; xi_k), Section 3), as the mean over B samples.
+//
+//   least squares : F = 1/2 (a.x - y)^2             g = (1/B) sum_b (a_b.x - y_b) a_b
+//   logistic      : F = log(1 + exp(-y (a.w + c)))  g_w = (1/B) sum_b -y_b s_b a_b + l2 w,
+//                   x = [w | c]                     g_c = (1/B) sum_b -y_b s_b,  s_b = sigma(-y_b z_b)
+//
+// Two kernels: a batched GEMV "forward" (one warp per (node, sample): draw the index, dot the
+// gathered data row with the node's parameters by warp shuffles, turn it into the per-sample
+// coefficient) and a rank-B "backward" (G_i = sum_b coef_b a_b).  All reductions run in a
+// fixed order, so results are bit-reproducible.
+#include "ctx.h"
+#include "philox.cuh"
+
+namespace dpsgd {
+namespace {
+
+constexpr int kFwdWarps = 8;
+
+__device__ __forceinline__ float warp_allsum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+template <int VEC>
+__global__ void __launch_bounds__(kFwdWarps * 32)
+glm_forward_kernel(const float* __restrict__ X, int64_t ld, const float* __restrict__ A,
+                   const float* __restrict__ y, int64_t m, int d, int B, int n, uint64_t seed,
+                   uint64_t k, int model, int32_t* __restrict__ idx, float* __restrict__ coef) {
+    const int w = blockIdx.x * kFwdWarps + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (w >= n * B) return;
+    const int node = w / B, b = w - node * B;
+    const int32_t j = sample_index(seed, k, (uint32_t)node, (uint32_t)b, (uint32_t)m);
+    const float* row = A + ((int64_t)node * m + j) * d;
+    const float* x = X + (int64_t)node * ld;
+    float acc = 0.f;
+    if (VEC == 4) {
+        const float4* r4 = reinterpret_cast<const float4*>(row);
+        const float4* x4 = reinterpret_cast<const float4*>(x);
+        for (int c = lane; c < d / 4; c += 32) {
+            const float4 a = __ldg(r4 + c), v = __ldg(x4 + c);
+            acc = fmaf(a.x, v.x, acc); acc = fmaf(a.y, v.y, acc);
+            acc = fmaf(a.z, v.z, acc); acc = fmaf(a.w, v.w, acc);
+        }
+    } else {
+        for (int c = lane; c < d; c += 32) acc = fmaf(__ldg(row + c), __ldg(x + c), acc);
+    }
+    const float dot = warp_allsum(acc);
+    if (lane == 0) {
+        const float yv = __ldg(y + (int64_t)node * m + j);
+        float cf;
+        if (model == DPSGD_MODEL_LSQ) {
+            cf = (dot - yv) / (float)B;
+        } else {
+            const float z = dot + __ldg(x + d);
+            const float s = 1.f / (1.f + expf(yv * z));
+            cf = -yv * s / (float)B;
+        }
+        idx[w] = j;
+        coef[w] = cf;
+    }
+}
+
+// blockDim = (64, 4): 64 column groups x 4 interleaved slices of the minibatch.
+template <int VEC>
+__global__ void __launch_bounds__(256)
+glm_backward_kernel(const float* __restrict__ X, float* __restrict__ G, int64_t ld,
+                    const float* __restrict__ A, int64_t m, int d, int B, int model, float l2,
+                    const int32_t* __restrict__ idx, const float* __restrict__ coef) {
+    __shared__ float red[4][64][VEC];
+    const int node = blockIdx.y;
+    const int tx = threadIdx.x, ty = threadIdx.y;
+    const int col = (blockIdx.x * 64 + tx) * VEC;       // first of VEC columns
+    const bool live = col < d;
+    float acc[VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
+    const int32_t* ix = idx + (int64_t)node * B;
+    const float* cf = coef + (int64_t)node * B;
+    if (live) {
+        const float* base = A + (int64_t)node * m * d + col;
+        for (int b = ty; b < B; b += 4) {
+            const float w = __ldg(cf + b);
+            const float* row = base + (int64_t)__ldg(ix + b) * d;
+            if (VEC == 4) {
+                const float4 a = __ldg(reinterpret_cast<const float4*>(row));
+                acc[0] = fmaf(w, a.x, acc[0]); acc[1 % VEC] = fmaf(w, a.y, acc[1 % VEC]);
+                acc[2 % VEC] = fmaf(w, a.z, acc[2 % VEC]); acc[3 % VEC] = fmaf(w, a.w, acc[3 % VEC]);
+            } else {
+                acc[0] = fmaf(w, __ldg(row), acc[0]);
+            }
+        }
+    }
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) red[ty][tx][v] = acc[v];
+    __syncthreads();
+    if (ty == 0 && live) {
+        float* g = G + (int64_t)node * ld + col;
+        const float* x = X + (int64_t)node * ld + col;
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) {
+            float s = ((red[0][tx][v] + red[1][tx][v]) + red[2][tx][v]) + red[3][tx][v];
+            if (model == DPSGD_MODEL_LOGISTIC) s = fmaf(l2, __ldg(x + v), s);
+            g[v] = s;
+        }
+    }
+    // bias gradient (logistic) and zero padding: columns [d, ld)
+    if (blockIdx.x == 0 && ty == 1) {
+        for (int64_t c = d + tx; c < ld; c += 64) {
+            float s = 0.f;
+            if (model == DPSGD_MODEL_LOGISTIC && c == d)
+                for (int b = 0; b < B; ++b) s += __ldg(cf + b);
+            G[(int64_t)node * ld + c] = s;
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_grad_linear(dpsgd_ctx* c, uint64_t k, const float* X, float* G) {
+    const int n = c->n, B = c->batch, d = c->d;
+    const float* y = static_cast<const float*>(c->y);
+    const int fwd_grid = (n * B + kFwdWarps - 1) / kFwdWarps;
+    const bool vec = (d % 4 == 0);
+    if (vec)
+        glm_forward_kernel<4><<<fwd_grid, kFwdWarps * 32, 0, c->stream>>>(
+            X, c->ld, c->A, y, c->m, d, B, n, c->seed, k, c->model, c->d_idx, c->d_coef);
+    else
+        glm_forward_kernel<1><<<fwd_grid, kFwdWarps * 32, 0, c->stream>>>(
+            X, c->ld, c->A, y, c->m, d, B, n, c->seed, k, c->model, c->d_idx, c->d_coef);
+    const int vw = vec ? 4 : 1;
+    dim3 grid((d + 64 * vw - 1) / (64 * vw), n), block(64, 4);
+    if (vec)
+        glm_backward_kernel<4><<<grid, block, 0, c->stream>>>(X, G, c->ld, c->A, c->m, d, B, c->model,
+                                                              c->l2, c->d_idx, c->d_coef);
+    else
+        glm_backward_kernel<1><<<grid, block, 0, c->stream>>>(X, G, c->ld, c->A, c->m, d, B, c->model,
+                                                              c->l2, c->d_idx, c->d_coef);
+    c->launches += 2;
+    return cudaGetLastError();
+}
+
+}  // namespace dpsgd
