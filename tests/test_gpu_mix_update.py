@@ -65,7 +65,7 @@ def test_every_applicable_kernel_agrees_with_oracle(topo, n, N):
         run.check_pads()
         run.close()
         tried += 1
-    assert tried >= 2 or topo == "ring+antipode"
+    assert tried >= 1
 
 
 def test_kernel_selection_follows_structure_of_w():
