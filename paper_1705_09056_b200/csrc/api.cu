@@ -204,8 +204,9 @@ DPSGD_API dpsgd_status dpsgd_create(dpsgd_ctx** out, int32_t n, int64_t N, const
     }
     e = cudaMalloc(&c->d_w_blob, total);
     if (e == cudaSuccess) e = cudaMemcpy(c->d_w_blob, blob.data(), total, cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaMalloc(&c->d_result, sizeof(double));
-    if (e == cudaSuccess) e = cudaMallocHost(&c->h_result, sizeof(double));
+    if (e == cudaSuccess) e = cudaMalloc(&c->d_result, sizeof(ResultBlock));
+    if (e == cudaSuccess) e = cudaMemset(c->d_result, 0, sizeof(ResultBlock));
+    if (e == cudaSuccess) e = cudaMallocHost(&c->h_result, sizeof(ResultBlock));
     if (e != cudaSuccess) { auto s = cuda_fail(nullptr, e, "dpsgd_create allocation"); release(c); return s; }
     char* base = static_cast<char*>(c->d_w_blob);
     c->W.row_ptr = reinterpret_cast<int32_t*>(base + o_rp);
@@ -345,12 +346,16 @@ DPSGD_API dpsgd_status dpsgd_consensus_dist(dpsgd_ctx* c, double* out) {
     dpsgd_status s = need_bound(c);
     if (s != DPSGD_OK) return s;
     if (!out) return fail(c, DPSGD_ERR_ARG, "out_host is NULL");
-    cudaError_t e = launch_consensus(c, c->X[c->cur], c->d_result);
+    cudaError_t e = launch_consensus(c, c->X[c->cur], &c->d_result->value);
     if (e == cudaSuccess)
-        e = cudaMemcpyAsync(c->h_result, c->d_result, sizeof(double), cudaMemcpyDeviceToHost, c->stream);
+        e = cudaMemcpyAsync(c->h_result, c->d_result, sizeof(ResultBlock), cudaMemcpyDeviceToHost, c->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
     if (e != cudaSuccess) return cuda_fail(c, e, "consensus distance");
-    *out = *c->h_result;
+    *out = c->h_result->value;
+    if (c->h_result->status != 0) {
+        cudaMemsetAsync(&c->d_result->status, 0, sizeof(int), c->stream);
+        return fail(c, DPSGD_ERR_TIMEOUT, "a kernel gave up waiting for a tile copy; X is not valid");
+    }
     return DPSGD_OK;
 }
 

@@ -25,6 +25,13 @@ struct MixW {
     float uniform = 0.f;               // uniform dense only: the common entry
 };
 
+// Written by the device, read back by the synchronising calls.
+struct ResultBlock {
+    double value;   // consensus distance
+    int status;     // 0, or a dpsgd_status set by a kernel whose bounded wait ran out
+    int pad;
+};
+
 struct MlpShape {
     int nlayers = 0;                 // number of weight layers L
     int dims[kMaxLayers + 1] = {0};  // d_0 .. d_L
@@ -77,8 +84,8 @@ struct dpsgd_ctx {
     size_t act_floats = 0, delta_floats = 0;
     double* d_partials = nullptr;  // consensus partial sums, one per CTA
     int partials_cap = 0;
-    double* d_result = nullptr;    // final scalar
-    double* h_result = nullptr;    // pinned
+    dpsgd::ResultBlock* d_result = nullptr;  // final scalar + device status word
+    dpsgd::ResultBlock* h_result = nullptr;  // pinned
     void* tma_state = nullptr;     // tensor maps for the tiled mixing kernel
 
     int64_t launches = 0;
