@@ -155,9 +155,29 @@ def loss_mlp(x, dims, A, labels, idx):
     return -np.mean(logp[np.arange(len(idx)), labels[idx]])
 
 
-def grad_mlp(x, dims, A, labels, idx):
+def mlp_near_zero_gates(x, dims, A, idx, rel):
+    """Hidden units whose pre-activation z is so close to 0 that fp32 rounding may put it on the
+    other side: |z| <= rel * (|h_{l-1}| |W_l|^T + |b_l|).  Returns [(layer l, sample b, unit)] with
+    l the 0-based index of the weight layer producing the unit.  For such a unit ReLU'(z) = 0 and
+    ReLU'(z) = 1 are both results a correct fp32 implementation can reach."""
+    Ws, h, pre = _mlp_forward(x, dims, A, idx)
+    _, bs = _mlp_views(np.asarray(x, dtype=np.float64), dims)
+    out = []
+    for l in range(len(Ws) - 1):
+        bound = np.abs(h[l]) @ np.abs(Ws[l]).T + np.abs(bs[l])
+        for b, u in np.argwhere(np.abs(pre[l]) <= rel * bound):
+            out.append((l, int(b), int(u)))
+    return out
+
+
+def grad_mlp(x, dims, A, labels, idx, flip=()):
+    """Minibatch-mean gradient by back-propagation, ReLU'(0) = 0.  `flip` lists (layer, sample,
+    unit) gates from mlp_near_zero_gates whose ReLU' decision is inverted (test use only)."""
     B = len(idx)
     Ws, h, pre = _mlp_forward(x, dims, A, idx)
+    gates = [p > 0.0 for p in pre[:-1]]
+    for (l, b, u) in flip:
+        gates[l][b, u] = ~gates[l][b, u]
     z = h[-1] - np.max(h[-1], axis=1, keepdims=True)
     p = np.exp(z)
     p /= np.sum(p, axis=1, keepdims=True)
@@ -168,7 +188,7 @@ def grad_mlp(x, dims, A, labels, idx):
     for l in range(len(Ws) - 1, -1, -1):
         parts[l] = (delta.T @ h[l], np.sum(delta, axis=0))
         if l > 0:
-            delta = (delta @ Ws[l]) * (pre[l - 1] > 0.0)     # ReLU'(0) = 0
+            delta = (delta @ Ws[l]) * gates[l - 1]
     return np.concatenate([np.concatenate([gw.reshape(-1), gb]) for gw, gb in parts])
 
 

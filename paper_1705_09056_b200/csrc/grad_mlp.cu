@@ -1,8 +1,258 @@
-// MLP gradients (placeholder until the batched GEMM kernels land).
+// Algorithm 1 steps 2-3 for the MLP: every node's minibatch gradient of the softmax
+// cross-entropy of a ReLU network at its own parameters x_{k,i} (one column of dF(X_k; xi_k),
+// Section 3), as the mean over the B sampled examples (footnote a).
+//
+// Parameter row layout: [W_1 (d_1 x d_0, row-major) | b_1 | W_2 | b_2 | ...].
+// Per node i, with h_0 the gathered inputs [B][d_0]:
+//     h_l     = relu(h_{l-1} W_l^T + b_l)        l = 1..L-1,   h_L = h_{L-1} W_L^T + b_L (logits)
+//     delta_L = (softmax(h_L) - onehot(y)) / B
+//     gW_l    = delta_l^T h_{l-1},   gb_l = sum_b delta_l[b],
+//     delta_{l-1} = (delta_l W_l) * [h_{l-1} > 0]                      (ReLU'(0) = 0)
+// All three products are batched GEMMs over the n nodes with per-node operands.  This file holds
+// the fp32 FMA implementation (exact fp32 products, fp32 accumulation in a fixed order).
 #include "ctx.h"
+#include "philox.cuh"
 
 namespace dpsgd {
-size_t mlp_act_floats(const dpsgd_ctx*) { return 1; }
-size_t mlp_delta_floats(const dpsgd_ctx*) { return 1; }
-cudaError_t launch_grad_mlp(dpsgd_ctx*, uint64_t, const float*, float*) { return cudaErrorNotSupported; }
+namespace {
+
+// activations: h_l of every node, l = 0..L, stored [l][node][B][d_l]
+struct MlpPlan {
+    int L;
+    int B;
+    int n;
+    size_t act_off[kMaxLayers + 2];
+    size_t delta_off[kMaxLayers + 1];   // delta_l for l = 1..L, stored [l][node][B][d_l]
+};
+
+MlpPlan make_plan(const dpsgd_ctx* c) {
+    MlpPlan p{};
+    p.L = c->mlp.nlayers; p.B = c->batch; p.n = c->n;
+    size_t a = 0, d = 0;
+    for (int l = 0; l <= p.L; ++l) {
+        p.act_off[l] = a;
+        a += (size_t)c->n * c->batch * c->mlp.dims[l];
+        p.delta_off[l] = d;
+        if (l >= 1) d += (size_t)c->n * c->batch * c->mlp.dims[l];
+    }
+    return p;
+}
+
+// h_0[node][b][:] = A[node][idx][:] with idx drawn for (iteration k, node, b).
+__global__ void __launch_bounds__(128)
+mlp_gather_kernel(const float* __restrict__ A, int64_t m, int d, int B, uint64_t seed, uint64_t k,
+                  int32_t* __restrict__ idx, float* __restrict__ h0) {
+    const int node = blockIdx.y, b = blockIdx.x;
+    const int32_t j = sample_index(seed, k, (uint32_t)node, (uint32_t)b, (uint32_t)m);
+    if (threadIdx.x == 0) idx[node * B + b] = j;
+    const float* src = A + ((int64_t)node * m + j) * d;
+    float* dst = h0 + ((int64_t)node * B + b) * d;
+    if ((d & 3) == 0) {
+        for (int c = threadIdx.x; c < d / 4; c += 128)
+            reinterpret_cast<float4*>(dst)[c] = __ldg(reinterpret_cast<const float4*>(src) + c);
+    } else {
+        for (int c = threadIdx.x; c < d; c += 128) dst[c] = __ldg(src + c);
+    }
+}
+
+enum { EPI_BIAS_RELU = 0, EPI_BIAS = 1, EPI_STORE = 2, EPI_MASK = 3 };
+
+struct GemmArgs {
+    const float* A; int64_t a_node, a_m, a_k;   // element strides: per node, along m, along k
+    const float* Bm; int64_t b_node, b_n, b_k;
+    float* C; int64_t c_node, c_m;              // C[m][n], n contiguous
+    const float* aux; int64_t aux_node, aux_m;  // bias[n] (aux_m = 0) or mask source [m][n]
+    int M, N, K;
+};
+
+// C[m][n] = sum_k A(m,k) * B(n,k) per node, 64x64x16 tiles, 256 threads, 4x4 outputs per thread.
+// A_K / B_K say whether the operand is contiguous along k (else along m / n).
+template <bool A_K, bool B_K, int EPI>
+__global__ void __launch_bounds__(256)
+bgemm_kernel(GemmArgs g) {
+    constexpr int BM = 64, BN = 64, BK = 16;
+    __shared__ float As[BK][BM + 4];
+    __shared__ float Bs[BK][BN + 4];
+    const int node = blockIdx.z;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const float* A = g.A + (int64_t)node * g.a_node;
+    const float* Bp = g.Bm + (int64_t)node * g.b_node;
+    const int tid = threadIdx.x;
+    const int tx = tid % 16, ty = tid / 16;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int k0 = 0; k0 < g.K; k0 += BK) {
+        // 64 x 16 elements per operand, 4 per thread
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const int e = tid + t * 256;
+            int mm, kk;
+            if (A_K) { kk = e % BK; mm = e / BK; } else { mm = e % BM; kk = e / BM; }
+            const int gm = m0 + mm, gk = k0 + kk;
+            As[kk][mm] = (gm < g.M && gk < g.K) ? __ldg(A + (int64_t)gm * g.a_m + (int64_t)gk * g.a_k) : 0.f;
+            int nn, kb;
+            if (B_K) { kb = e % BK; nn = e / BK; } else { nn = e % BN; kb = e / BN; }
+            const int gn = n0 + nn, gkb = k0 + kb;
+            Bs[kb][nn] = (gn < g.N && gkb < g.K) ? __ldg(Bp + (int64_t)gn * g.b_n + (int64_t)gkb * g.b_k) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            const float4 a = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+            const float4 b = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+            const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    float* C = g.C + (int64_t)node * g.c_node;
+    const float* aux = g.aux ? g.aux + (int64_t)node * g.aux_node : nullptr;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int gm = m0 + ty * 4 + i;
+        if (gm >= g.M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int gn = n0 + tx * 4 + j;
+            if (gn >= g.N) continue;
+            float v = acc[i][j];
+            if (EPI == EPI_BIAS_RELU) { v += __ldg(aux + gn); v = v > 0.f ? v : 0.f; }
+            if (EPI == EPI_BIAS) v += __ldg(aux + gn);
+            if (EPI == EPI_MASK) v = __ldg(aux + (int64_t)gm * g.aux_m + gn) > 0.f ? v : 0.f;
+            C[(int64_t)gm * g.c_m + gn] = v;
+        }
+    }
+}
+
+// delta_L[b][:] = (softmax(logits[b]) - onehot(y[idx[b]])) / B; one warp per (node, sample).
+__global__ void __launch_bounds__(128)
+softmax_ce_delta_kernel(const float* __restrict__ logits, const int32_t* __restrict__ y, int64_t m,
+                        const int32_t* __restrict__ idx, int n, int B, int C, float* __restrict__ delta) {
+    const int w = blockIdx.x * 4 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (w >= n * B) return;
+    const int node = w / B;
+    const float* z = logits + (int64_t)w * C;
+    float mx = -INFINITY;
+    for (int c = lane; c < C; c += 32) mx = fmaxf(mx, z[c]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float s = 0.f;
+    for (int c = lane; c < C; c += 32) s += expf(z[c] - mx);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    const int label = __ldg(y + (int64_t)node * m + __ldg(idx + w));
+    const float inv = 1.f / s, invB = 1.f / (float)B;
+    for (int c = lane; c < C; c += 32)
+        delta[(int64_t)w * C + c] = (expf(z[c] - mx) * inv - (c == label ? 1.f : 0.f)) * invB;
+}
+
+// gb[o] = sum_b delta[b][o], written into the gradient row; fixed order over b.
+__global__ void __launch_bounds__(128)
+bias_grad_kernel(const float* __restrict__ delta, int B, int D, float* __restrict__ G, int64_t ld,
+                 int64_t b_off) {
+    const int node = blockIdx.y;
+    const int o = blockIdx.x * 128 + threadIdx.x;
+    if (o >= D) return;
+    const float* d = delta + (int64_t)node * B * D + o;
+    float s = 0.f;
+    for (int b = 0; b < B; ++b) s += d[(int64_t)b * D];
+    G[(int64_t)node * ld + b_off + o] = s;
+}
+
+__global__ void zero_pad_kernel(float* __restrict__ G, int64_t ld, int64_t N, int n) {
+    const int64_t width = ld - N;
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= width * n) return;
+    G[(t / width) * ld + N + (t % width)] = 0.f;
+}
+
+template <bool A_K, bool B_K, int EPI>
+void run_gemm(dpsgd_ctx* c, const GemmArgs& g) {
+    dim3 grid((g.N + 63) / 64, (g.M + 63) / 64, c->n);
+    bgemm_kernel<A_K, B_K, EPI><<<grid, 256, 0, c->stream>>>(g);
+    c->launches++;
+}
+
+}  // namespace
+
+size_t mlp_act_floats(const dpsgd_ctx* c) {
+    size_t a = 0;
+    for (int l = 0; l <= c->mlp.nlayers; ++l) a += (size_t)c->n * c->batch * c->mlp.dims[l];
+    return a;
+}
+
+size_t mlp_delta_floats(const dpsgd_ctx* c) {
+    size_t a = 0;
+    for (int l = 1; l <= c->mlp.nlayers; ++l) a += (size_t)c->n * c->batch * c->mlp.dims[l];
+    return a;
+}
+
+cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) {
+    const MlpPlan p = make_plan(c);
+    const MlpShape& s = c->mlp;
+    const int n = c->n, B = c->batch, L = s.nlayers;
+    const int32_t* y = static_cast<const int32_t*>(c->y);
+
+    mlp_gather_kernel<<<dim3(B, n), 128, 0, c->stream>>>(c->A, c->m, s.dims[0], B, c->seed, k, c->d_idx,
+                                                         c->d_act + p.act_off[0]);
+    c->launches++;
+
+    // forward
+    for (int l = 1; l <= L; ++l) {
+        const int din = s.dims[l - 1], dout = s.dims[l];
+        GemmArgs g{};
+        g.A = c->d_act + p.act_off[l - 1]; g.a_node = (int64_t)B * din; g.a_m = din; g.a_k = 1;
+        g.Bm = X + s.w_off[l - 1]; g.b_node = c->ld; g.b_n = din; g.b_k = 1;
+        g.C = c->d_act + p.act_off[l]; g.c_node = (int64_t)B * dout; g.c_m = dout;
+        g.aux = X + s.b_off[l - 1]; g.aux_node = c->ld; g.aux_m = 0;
+        g.M = B; g.N = dout; g.K = din;
+        if (l < L) run_gemm<true, true, EPI_BIAS_RELU>(c, g);
+        else run_gemm<true, true, EPI_BIAS>(c, g);
+    }
+
+    softmax_ce_delta_kernel<<<(n * B + 3) / 4, 128, 0, c->stream>>>(
+        c->d_act + p.act_off[L], y, c->m, c->d_idx, n, B, s.dims[L], c->d_delta + p.delta_off[L]);
+    c->launches++;
+
+    // backward
+    for (int l = L; l >= 1; --l) {
+        const int din = s.dims[l - 1], dout = s.dims[l];
+        const float* delta = c->d_delta + p.delta_off[l];
+        {   // gW_l[o][k] = sum_b delta[b][o] h_{l-1}[b][k]
+            GemmArgs g{};
+            g.A = delta; g.a_node = (int64_t)B * dout; g.a_m = 1; g.a_k = dout;
+            g.Bm = c->d_act + p.act_off[l - 1]; g.b_node = (int64_t)B * din; g.b_n = 1; g.b_k = din;
+            g.C = G + s.w_off[l - 1]; g.c_node = c->ld; g.c_m = din;
+            g.M = dout; g.N = din; g.K = B;
+            run_gemm<false, false, EPI_STORE>(c, g);
+        }
+        bias_grad_kernel<<<dim3((dout + 127) / 128, n), 128, 0, c->stream>>>(delta, B, dout, G, c->ld,
+                                                                               s.b_off[l - 1]);
+        c->launches++;
+        if (l > 1) {   // delta_{l-1}[b][k] = (sum_o delta[b][o] W_l[o][k]) * [h_{l-1}[b][k] > 0]
+            GemmArgs g{};
+            g.A = delta; g.a_node = (int64_t)B * dout; g.a_m = dout; g.a_k = 1;
+            g.Bm = X + s.w_off[l - 1]; g.b_node = c->ld; g.b_n = 1; g.b_k = din;
+            g.C = c->d_delta + p.delta_off[l - 1]; g.c_node = (int64_t)B * din; g.c_m = din;
+            g.aux = c->d_act + p.act_off[l - 1]; g.aux_node = (int64_t)B * din; g.aux_m = din;
+            g.M = B; g.N = din; g.K = dout;
+            run_gemm<true, false, EPI_MASK>(c, g);
+        }
+    }
+    if (c->ld > c->N) {
+        const int64_t total = (c->ld - c->N) * n;
+        zero_pad_kernel<<<(unsigned)((total + 127) / 128), 128, 0, c->stream>>>(G, c->ld, c->N, n);
+        c->launches++;
+    }
+    return cudaGetLastError();
+}
+
 }  // namespace dpsgd

@@ -62,3 +62,31 @@ class GpuRun:
 
     def close(self):
         self.ctx.close()
+
+
+GATE_REL = 4e-6   # pre-activations within this (relative to the sum of |terms|) may round either way in fp32
+
+
+def mlp_oracle_grad_matching_gates(orc, o, k, G_gpu):
+    """The oracle's MLP gradients for iteration k.  A hidden unit whose fp64 pre-activation is
+    within fp32 rounding of zero has two valid ReLU' decisions; for those units (and only
+    those) the decision that brings the oracle closer to the GPU result is taken, one unit at a
+    time.  Everything else is the oracle's own fp64 arithmetic."""
+    idx = o.sample(k)
+    G = np.empty((o.n, o.N), dtype=np.float32)
+    flips = 0
+    for i in range(o.n):
+        args = (o.X[i], o.dims, o.A[i], o.y[i], idx[i])
+        ties = orc.mlp_near_zero_gates(o.X[i], o.dims, o.A[i], idx[i], GATE_REL)
+        assert len(ties) <= 64, "too many near-zero pre-activations for a meaningful comparison"
+        chosen = []
+        best = orc.grad_mlp(*args).astype(np.float32)
+        best_err = np.linalg.norm(best.astype(np.float64) - G_gpu[i])
+        for t in ties:
+            cand = orc.grad_mlp(*args, flip=chosen + [t]).astype(np.float32)
+            err = np.linalg.norm(cand.astype(np.float64) - G_gpu[i])
+            if err < best_err:
+                best, best_err, chosen = cand, err, chosen + [t]
+        flips += len(chosen)
+        G[i] = best
+    return G, flips

@@ -121,3 +121,23 @@ def test_gradients_use_each_nodes_own_row_and_data():
     assert G.dtype == np.float32
     for i in range(n):
         assert np.array_equal(G[i], orc.grad_lsq(X[i], A[i], y[i], idx[i]).astype(np.float32))
+
+
+def test_mlp_near_zero_gates_and_flip():
+    """A unit whose pre-activation is exactly zero is reported; flipping its gate changes only
+    what that unit back-propagates (ReLU'(0) = 0 by default, 1 when flipped)."""
+    dims = (3, 2, 2)
+    x = np.array([1.0, -1.0, 0.0, 0.5, 0.5, 0.5, 0.0, -1.5,      # W1 (2x3), b1
+                  1.0, 2.0, -1.0, 0.5, 0.0, 0.0], dtype=np.float32)  # W2 (2x2), b2
+    A = np.array([[1.0, 1.0, 7.0], [1.0, 2.0, 0.0]], dtype=np.float32)   # sample 0: z = (0, 3); sample 1: z = (-1, 0)
+    labels = np.array([0, 1], dtype=np.int32)
+    idx = np.array([0, 1])
+    ties = orc.mlp_near_zero_gates(x, dims, A, idx, 1e-6)
+    assert ties == [(0, 0, 0), (0, 1, 1)]
+    assert orc.mlp_near_zero_gates(x, dims, A, np.array([0]), 1e-6) == [(0, 0, 0)]
+    g0 = orc.grad_mlp(x, dims, A, labels, idx)
+    g1 = orc.grad_mlp(x, dims, A, labels, idx, flip=[(0, 0, 0)])
+    assert np.all(g0[0:3] == 0)          # row 0 of W1: sample 0 gated off (z = 0), sample 1 off (z < 0)
+    assert np.any(g1[0:3] != 0)          # flipped: sample 0 now back-propagates through unit 0
+    assert np.array_equal(g0[8:], g1[8:])  # the output layer's gradient does not depend on the gate
+    assert np.array_equal(g0[3:6], g1[3:6])
