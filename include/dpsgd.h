@@ -153,6 +153,29 @@ DPSGD_API dpsgd_status dpsgd_average(dpsgd_ctx* ctx, float* xbar_dev);
 DPSGD_API dpsgd_status dpsgd_mix_update_host(dpsgd_ctx* ctx, const float* G_host, int64_t ld_host,
                                    double* consensus_out_host);
 
+/*
+ * (The paper has no counterpart: this is a packaging variant of dpsgd_consensus_dist.)
+ * Consensus distance for callers that must not trigger an allocation: a process whose device
+ * memory was handed to its own pool up front, a loop that cannot afford the device-wide
+ * synchronisation an allocation implies, or code that has a raw device pointer and no context
+ * (contexts allocate scratch).  It calls no cudaMalloc/cudaFree and no allocating library
+ * routine; the per-CTA partial sums live in a fixed 512 KB array inside the library image, which
+ * every GPU that loads the library keeps until the process exits.
+ *   X_dev   device, fp32 [n][ld], 128-byte aligned, ld a multiple of 32, columns [N, ld) zero
+ *   out_dev device, one double (8-byte aligned), written asynchronously on cuda_stream:
+ *           sum_i ||xbar - x_i||^2, the same value dpsgd_consensus_dist returns
+ * Limit: ld <= DPSGD_NOALLOC_MAX_LD (67,108,864 columns); larger inputs are refused with
+ * DPSGD_ERR_UNSUPPORTED and a message in dpsgd_last_error(NULL).  1 <= n <= 65535.
+ * The first call on each device looks up the array's device address (with that device current,
+ * which must be the device that owns X_dev); make that first call outside any stream capture.
+ * All calls in the process share the one array: it keeps the previous call's partial sums, each
+ * call overwrites the entries it reads before reading them, and two calls whose kernels overlap
+ * on the GPU (different streams) race on it - serialise them.
+ */
+#define DPSGD_NOALLOC_MAX_LD 67108864LL
+DPSGD_API dpsgd_status dpsgd_consensus_dist_noalloc(const float* X_dev, int32_t n, int64_t N, int64_t ld,
+                                                    void* cuda_stream, double* out_dev);
+
 /* Device pointer of the buffer that currently holds X_k (one of the two bound buffers). */
 DPSGD_API dpsgd_status dpsgd_current(dpsgd_ctx* ctx, float** X_cur_dev);
 

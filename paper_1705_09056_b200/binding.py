@@ -40,6 +40,7 @@ SIGNATURES = {
     "dpsgd_consensus_dist": [_vp, ctypes.POINTER(ctypes.c_double)],
     "dpsgd_average": [_vp, _vp],
     "dpsgd_mix_update_host": [_vp, _vp, _i64, ctypes.POINTER(ctypes.c_double)],
+    "dpsgd_consensus_dist_noalloc": [_vp, _i32, _i64, _i64, _vp, _vp],
     "dpsgd_current": [_vp, ctypes.POINTER(_vp)],
     "dpsgd_set_gamma": [_vp, _f32],
     "dpsgd_mix_kind": [_vp, _i32, ctypes.POINTER(_i32)],
@@ -83,6 +84,25 @@ def _ptr(t) -> int:
     if isinstance(t, np.ndarray):
         return t.ctypes.data
     return int(t)
+
+
+NOALLOC_MAX_LD = 67108864
+
+
+def consensus_dist_noalloc(X: torch.Tensor, N: int, out: torch.Tensor, stream=None) -> torch.Tensor:
+    """sum_i ||xbar - x_i||^2 of the rows of X (n x ld, columns [N, ld) zero) into the one-element
+    float64 CUDA tensor `out`, without any allocation inside the library: for callers that own
+    all device memory themselves or have no context.  Asynchronous on the stream; see
+    dpsgd_consensus_dist_noalloc in include/dpsgd.h for the size limit and the shared scratch."""
+    lib = load_library()
+    assert X.is_cuda and X.dtype == torch.float32 and X.is_contiguous() and X.dim() == 2
+    assert out.is_cuda and out.dtype == torch.float64 and out.numel() == 1
+    s = stream if stream is not None else torch.cuda.current_stream(X.device)
+    with torch.cuda.device(X.device):
+        st = lib.dpsgd_consensus_dist_noalloc(_ptr(X), X.shape[0], N, X.shape[1], s.cuda_stream, _ptr(out))
+    if st != OK:
+        raise DpsgdError(st, lib.dpsgd_last_error(None).decode())
+    return out
 
 
 class Dpsgd:

@@ -158,6 +158,11 @@ cudaError_t run_grad(dpsgd_ctx* c, uint64_t k) {
 
 }  // namespace
 
+namespace dpsgd {
+// Lets entry points that take no context leave a message for dpsgd_last_error(NULL).
+void set_thread_error(const std::string& msg) { g_create_error = msg; }
+}  // namespace dpsgd
+
 extern "C" {
 
 DPSGD_API dpsgd_status dpsgd_create(dpsgd_ctx** out, int32_t n, int64_t N, const int32_t* row_ptr,

@@ -6,6 +6,8 @@
 // fp64, so no cancellation against |x| occurs.  Columns are combined by warp shuffles, one
 // fp64 partial per CTA, and a second single-CTA kernel adds the partials in a fixed order:
 // the result is bit-reproducible (no floating-point atomics).
+#include <mutex>
+
 #include "ctx.h"
 
 namespace dpsgd {
@@ -126,3 +128,84 @@ cudaError_t launch_average(dpsgd_ctx* c, const float* X, float* xbar) {
 }
 
 }  // namespace dpsgd
+
+// ---------------------------------------------------------------------------------------------
+// Consensus distance without any allocation.
+//
+// Some callers cannot let this library allocate: a process that handed its whole device-memory
+// budget to its own pool at start-up (a later cudaMalloc would fail or eat into someone else's
+// share), a latency-critical loop that must not hit the device-wide synchronisation an
+// allocation implies, or code that holds only a raw device pointer and has no dpsgd context (a
+// context allocates its scratch when it is created and grown).  For them the per-CTA partial
+// sums live in a fixed array inside the library image instead of a cudaMalloc'ed buffer.
+//
+// The array's name is only a host-side handle in host code; the kernels need its device
+// address, fetched once per device with cudaGetSymbolAddress while that device is current.
+// ---------------------------------------------------------------------------------------------
+namespace dpsgd {
+void set_thread_error(const std::string& msg);   // api.cu: message returned by dpsgd_last_error(NULL)
+namespace {
+
+constexpr int kNoAllocMaxCtas = 65536;                                   // 512 KB of partials per GPU
+constexpr int64_t kNoAllocMaxLd = (int64_t)kNoAllocMaxCtas * kThreads * 4;  // 67,108,864 columns
+constexpr int kNoAllocMaxDevices = 64;
+
+static __device__ __align__(256) double g_noalloc_partials[kNoAllocMaxCtas];
+
+std::mutex g_noalloc_mutex;
+double* g_noalloc_ptr[kNoAllocMaxDevices] = {nullptr};
+
+// Device address of the partials array on the current device (set up on the first call there).
+cudaError_t noalloc_scratch(double** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kNoAllocMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_noalloc_partials);
+        if (e != cudaSuccess) return e;
+        g_noalloc_ptr[dev] = static_cast<double*>(p);
+    }
+    *out = g_noalloc_ptr[dev];
+    return cudaSuccess;
+}
+
+dpsgd_status noalloc_fail(dpsgd_status s, const std::string& msg) {
+    set_thread_error(msg);
+    return s;
+}
+
+}  // namespace
+}  // namespace dpsgd
+
+extern "C" DPSGD_API dpsgd_status dpsgd_consensus_dist_noalloc(const float* X_dev, int32_t n, int64_t N,
+                                                               int64_t ld, void* cuda_stream,
+                                                               double* out_dev) {
+    using namespace dpsgd;
+    if (!X_dev || !out_dev) return noalloc_fail(DPSGD_ERR_ARG, "X_dev or out_dev is NULL");
+    if (n < 1 || n > 65535 || N < 1 || ld < N) return noalloc_fail(DPSGD_ERR_ARG, "need 1 <= n <= 65535 and 1 <= N <= ld");
+    if (ld % 32 != 0 || reinterpret_cast<uintptr_t>(X_dev) % 128 != 0 || reinterpret_cast<uintptr_t>(out_dev) % 8 != 0)
+        return noalloc_fail(DPSGD_ERR_ALIGN, "X_dev must be 128-byte aligned, ld a multiple of 32 floats, out_dev 8-byte aligned");
+    if (ld > kNoAllocMaxLd) {
+        char buf[160];
+        snprintf(buf, sizeof buf, "ld = %lld exceeds the %lld columns the built-in scratch array covers; "
+                 "use a context and dpsgd_consensus_dist instead", (long long)ld, (long long)kNoAllocMaxLd);
+        return noalloc_fail(DPSGD_ERR_UNSUPPORTED, buf);
+    }
+    double* partials = nullptr;
+    cudaError_t e = noalloc_scratch(&partials);
+    if (e != cudaSuccess) return noalloc_fail(DPSGD_ERR_CUDA, std::string("scratch set-up: ") + cudaGetErrorString(e));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t ld4 = ld / 4;
+    const int grid = (int)((ld4 + kThreads - 1) / kThreads);
+    // every partial in [0, grid) is overwritten by the first kernel before the second reads it, so
+    // whatever an earlier call left in the array is never seen
+    consensus_partial_kernel<8><<<grid, kThreads, 0, stream>>>(reinterpret_cast<const float4*>(X_dev), n, ld4,
+                                                               partials);
+    consensus_final_kernel<<<1, kThreads, 0, stream>>>(partials, grid, out_dev);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return noalloc_fail(DPSGD_ERR_CUDA, std::string("consensus kernels: ") + cudaGetErrorString(e));
+    return DPSGD_OK;
+}
