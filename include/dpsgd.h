@@ -99,8 +99,9 @@ DPSGD_API dpsgd_status dpsgd_bind(dpsgd_ctx* ctx, float* X0_dev, float* X1_dev, 
  *                        x = [W_1 (d_1 x d_0 row-major) | b_1 | W_2 | b_2 ...], N = sum
  * batch = minibatch size B per node (footnote a of Algorithm 1; gradients are the MEAN over
  * the minibatch).  N must match the context's N.  Allocates the activation scratch.
- * mlp_precision: 0 = fp32-faithful (3xTF32 split on tensor cores or fp32 FMA), 1 = single
- * TF32 pass (faster, ~1e-3 relative on G).  Ignored for the linear models.
+ * mlp_precision (MLP only): 0 = fp32-faithful on the tensor cores (each product as three TF32
+ * MMAs on split operands; minibatches above 128 use the fp32 FMA kernel), 1 = one TF32 MMA per
+ * product (faster, about 1e-3 relative on G), 2 = fp32 FMA kernel always.
  */
 DPSGD_API dpsgd_status dpsgd_set_model(dpsgd_ctx* ctx, int32_t kind, const int32_t* dims_host,
                              int32_t ndims, float l2_lambda, int32_t batch,

@@ -8,10 +8,13 @@
 //     delta_L = (softmax(h_L) - onehot(y)) / B
 //     gW_l    = delta_l^T h_{l-1},   gb_l = sum_b delta_l[b],
 //     delta_{l-1} = (delta_l W_l) * [h_{l-1} > 0]                      (ReLU'(0) = 0)
-// All three products are batched GEMMs over the n nodes with per-node operands.  This file holds
-// the fp32 FMA implementation (exact fp32 products, fp32 accumulation in a fixed order).
+// All three products are batched GEMMs over the n nodes with per-node operands.  They run on the
+// tensor cores (tc_gemm.cuh: tcgen05 TF32 MMAs, three per product for fp32-faithful results) when
+// the minibatch fits a 128-column tile, and otherwise - or when asked - on the fp32 FMA kernel
+// below (exact fp32 products, fp32 accumulation in a fixed order).
 #include "ctx.h"
 #include "philox.cuh"
+#include "tc_gemm.cuh"
 
 namespace dpsgd {
 namespace {
@@ -181,6 +184,38 @@ void run_gemm(dpsgd_ctx* c, const GemmArgs& g) {
     c->launches++;
 }
 
+template <int NT>
+cudaError_t launch_tc_nt(dpsgd_ctx* c, const tc::Args& a, int n_tiles) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc::tc_gemm_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)tc::smem_bytes<NT>());
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    dim3 grid((a.M + tc::kTileM - 1) / tc::kTileM, n_tiles, c->n);
+    tc::tc_gemm_kernel<NT><<<grid, tc::kThreads, tc::smem_bytes<NT>(), c->stream>>>(a);
+    c->launches++;
+    return cudaGetLastError();
+}
+
+bool vec_ok(const float* p, int64_t pitch, int64_t node_stride) {
+    return (reinterpret_cast<uintptr_t>(p) % 16 == 0) && (pitch % 4 == 0) && (node_stride % 4 == 0);
+}
+
+// C[n][m] = epi(sum_k A(m,k) B(n,k)); max_tile = widest column tile (multiple of 16, <= 128).
+cudaError_t run_tc(dpsgd_ctx* c, tc::Args a, int max_tile) {
+    a.a_vec = vec_ok(a.A, a.a_pitch, a.a_node);
+    a.b_vec = vec_ok(a.B, a.b_pitch, a.b_node);
+    a.precise = c->mlp_precision == 0;
+    a.status = &c->d_result->status;
+    const int want = a.N < max_tile ? a.N : max_tile;
+    if (want <= 16) return launch_tc_nt<1>(c, a, (a.N + 15) / 16);
+    if (want <= 32) return launch_tc_nt<2>(c, a, (a.N + 31) / 32);
+    if (want <= 64) return launch_tc_nt<4>(c, a, (a.N + 63) / 64);
+    return launch_tc_nt<8>(c, a, (a.N + 127) / 128);
+}
+
 }  // namespace
 
 size_t mlp_act_floats(const dpsgd_ctx* c) {
@@ -200,6 +235,7 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) 
     const MlpShape& s = c->mlp;
     const int n = c->n, B = c->batch, L = s.nlayers;
     const int32_t* y = static_cast<const int32_t*>(c->y);
+    const bool use_tc = c->mlp_precision != 2 && B <= 128;   // precision 2 = fp32 FMA kernel
 
     mlp_gather_kernel<<<dim3(B, n), 128, 0, c->stream>>>(c->A, c->m, s.dims[0], B, c->seed, k, c->d_idx,
                                                          c->d_act + p.act_off[0]);
@@ -214,7 +250,16 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) 
         g.C = c->d_act + p.act_off[l]; g.c_node = (int64_t)B * dout; g.c_m = dout;
         g.aux = X + s.b_off[l - 1]; g.aux_node = c->ld; g.aux_m = 0;
         g.M = B; g.N = dout; g.K = din;
-        if (l < L) run_gemm<true, true, EPI_BIAS_RELU>(c, g);
+        if (use_tc) {   // m = output unit, n = sample: h_l[b][o]
+            tc::Args a{};
+            a.A = g.Bm; a.a_node = g.b_node; a.a_pitch = din; a.a_kcontig = 1;
+            a.B = g.A; a.b_node = g.a_node; a.b_pitch = din; a.b_kcontig = 1;
+            a.C = g.C; a.c_node = g.c_node; a.c_pitch = dout;
+            a.aux = g.aux; a.aux_node = g.aux_node; a.aux_pitch = 0;
+            a.M = dout; a.N = B; a.K = din; a.epi = l < L ? tc::EPI_BIAS_RELU : tc::EPI_BIAS;
+            cudaError_t e = run_tc(c, a, 128);
+            if (e != cudaSuccess) return e;
+        } else if (l < L) run_gemm<true, true, EPI_BIAS_RELU>(c, g);
         else run_gemm<true, true, EPI_BIAS>(c, g);
     }
 
@@ -232,7 +277,15 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) 
             g.Bm = c->d_act + p.act_off[l - 1]; g.b_node = (int64_t)B * din; g.b_n = 1; g.b_k = din;
             g.C = G + s.w_off[l - 1]; g.c_node = c->ld; g.c_m = din;
             g.M = dout; g.N = din; g.K = B;
-            run_gemm<false, false, EPI_STORE>(c, g);
+            if (use_tc) {   // m = input unit k', n = output unit o: gW[o][k']
+                tc::Args a{};
+                a.A = g.Bm; a.a_node = g.b_node; a.a_pitch = din; a.a_kcontig = 0;
+                a.B = delta; a.b_node = (int64_t)B * dout; a.b_pitch = dout; a.b_kcontig = 0;
+                a.C = g.C; a.c_node = c->ld; a.c_pitch = din;
+                a.M = din; a.N = dout; a.K = B; a.epi = tc::EPI_STORE;
+                cudaError_t e = run_tc(c, a, 64);
+                if (e != cudaSuccess) return e;
+            } else run_gemm<false, false, EPI_STORE>(c, g);
         }
         bias_grad_kernel<<<dim3((dout + 127) / 128, n), 128, 0, c->stream>>>(delta, B, dout, G, c->ld,
                                                                                s.b_off[l - 1]);
@@ -244,7 +297,16 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) 
             g.C = c->d_delta + p.delta_off[l - 1]; g.c_node = (int64_t)B * din; g.c_m = din;
             g.aux = c->d_act + p.act_off[l - 1]; g.aux_node = (int64_t)B * din; g.aux_m = din;
             g.M = B; g.N = din; g.K = dout;
-            run_gemm<true, false, EPI_MASK>(c, g);
+            if (use_tc) {   // m = input unit k', n = sample: delta_{l-1}[b][k']
+                tc::Args a{};
+                a.A = g.Bm; a.a_node = c->ld; a.a_pitch = din; a.a_kcontig = 0;
+                a.B = delta; a.b_node = (int64_t)B * dout; a.b_pitch = dout; a.b_kcontig = 1;
+                a.C = g.C; a.c_node = g.c_node; a.c_pitch = din;
+                a.aux = g.aux; a.aux_node = g.aux_node; a.aux_pitch = din;
+                a.M = din; a.N = B; a.K = dout; a.epi = tc::EPI_MASK;
+                cudaError_t e = run_tc(c, a, 128);
+                if (e != cudaSuccess) return e;
+            } else run_gemm<true, false, EPI_MASK>(c, g);
         }
     }
     if (c->ld > c->N) {

@@ -1,0 +1,79 @@
+"""Runs whole D-PSGD iterations (sample + gradient + mix + update) of one model configuration
+and prints CUDA-event timings: replica-steps/s and the split between gradient and gossip step.
+
+  python -m paper_1705_09056_b200.run_config --config 2 --steps 50
+  (0 least squares, 1 logistic, 2 MLP 784-1024-10, 4 MLP 1024-2048-2048-10)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import binding, build, workloads as wl
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", type=int, default=2, choices=[0, 1, 2, 4])
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--n", type=int, default=0, help="override the node count")
+    ap.add_argument("--m", type=int, default=0, help="override the local dataset size")
+    ap.add_argument("--topology", default="")
+    ap.add_argument("--precision", type=int, default=0, help="MLP: 0 fp32-faithful, 1 single TF32 pass")
+    ap.add_argument("--consensus", action="store_true", help="evaluate the consensus distance every step")
+    args = ap.parse_args()
+
+    build.build()
+    dev = torch.device("cuda", 0)
+    over = {}
+    if args.n:
+        over["n"] = args.n
+    if args.m:
+        over["m"] = args.m
+    if args.topology:
+        over["topology"] = args.topology
+    w = wl.config(args.config, device=dev, **over)
+    X0 = wl.stack_rows(w.x0, w.n, w.ld)
+    X1, G = torch.zeros_like(X0), torch.zeros_like(X0)
+    ctx = binding.Dpsgd(w.n, w.N, *w.csr(), gamma=w.gamma, seed=1)
+    ctx.bind(X0, X1, G)
+    ctx.set_model(w.model, w.dims, w.l2_lambda, w.batch, args.precision)
+    ctx.set_data(w.A, w.y)
+
+    def timed(fn, reps):
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for k in range(reps):
+            fn(k)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    for k in range(args.warmup):
+        ctx.step(k)
+    l0 = ctx.launch_count()
+    if args.consensus:
+        def whole(k):
+            ctx.step(args.warmup + k)
+            ctx.consensus_dist()
+    else:
+        def whole(k):
+            ctx.step(args.warmup + k)
+    ms_step = timed(whole, args.steps)
+    launches = (ctx.launch_count() - l0) / args.steps
+    ms_grad = timed(lambda k: ctx.grad(k), max(3, args.steps // 5))
+    ms_mix = timed(lambda k: ctx.mix_update(), max(3, args.steps // 5))
+    print(json.dumps({
+        "workload": w.name, "n": w.n, "N": w.N, "dims": list(w.dims), "batch": w.batch, "topology": w.topology,
+        "mix_kernel": binding.MIX_NAMES[ctx.mix_kind()], "ms_per_step": ms_step,
+        "replica_steps_per_s": w.n / (ms_step * 1e-3), "ms_grad": ms_grad, "ms_mix_update": ms_mix,
+        "launches_per_step": launches, "consensus": ctx.consensus_dist()}))
+    ctx.close()
+
+
+if __name__ == "__main__":
+    main()

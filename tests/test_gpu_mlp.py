@@ -9,7 +9,7 @@ from gpu_util import GpuRun, row_rel_err, mlp_oracle_grad_matching_gates, TOL_ST
 
 pytestmark = pytest.mark.gpu
 
-TOL_G = 2e-5      # row-wise relative error of the fp32 gradient against the fp64 oracle
+TOL_G = 5e-5      # row-wise relative error of the gradient against the fp64 oracle (3 x TF32 products: ~2^-20 each)
 
 
 def _setup(w, seed, precision=0, X=None):
@@ -38,13 +38,14 @@ MLP_CASES = [
 ]
 
 
+@pytest.mark.parametrize("precision", [0, 2])     # tensor cores (3 x TF32) and the fp32 FMA kernel
 @pytest.mark.parametrize("n,dims,m,B", MLP_CASES)
-def test_mlp_gradient_and_step_match_oracle(n, dims, m, B):
+def test_mlp_gradient_and_step_match_oracle(n, dims, m, B, precision):
     w = wl.mlp_workload(n=n, dims=dims, m=m, batch=B, gamma=0.05, seed=11)
     rng = np.random.default_rng(1)
     # perturb the shared initial point per node so that rows differ; biases non-zero
     X = (np.tile(w.x0.numpy(), (n, 1)) + 0.02 * rng.standard_normal((n, w.N))).astype(np.float32)
-    run, o = _setup(w, seed=3, X=X)
+    run, o = _setup(w, seed=3, precision=precision, X=X)
     for k in (0, 7):
         o.set_x(X)
         run.ctx.current()[:, :w.N] = torch.from_numpy(X).cuda()
@@ -105,3 +106,24 @@ def test_mlp_dense_w_side_by_side_with_ring():
         assert abs(c - o_dense.consensus_dist()) <= 1e-3 * expect
         assert abs(ring.ctx.consensus_dist() - o_ring.consensus_dist()) <= 1e-3 * o_ring.consensus_dist()
     ring.close(); dense.close()
+
+
+def test_mlp_single_tf32_pass_is_close_but_looser():
+    """mlp_precision = 1: one TF32 MMA per product (10-bit mantissas): about 1e-3 on G."""
+    w = wl.mlp_workload(n=3, dims=(256, 512, 10), m=64, batch=32, gamma=0.05, seed=12)
+    run, o = _setup(w, seed=4, precision=1)
+    run.ctx.grad(0)
+    G_ref = o.grad(0)
+    err = row_rel_err(run.g(), G_ref)
+    assert 1e-6 < err <= 5e-3
+    run.close()
+
+
+def test_mlp_large_batch_uses_fma_kernel():
+    """Minibatches above 128 do not fit one accumulator tile and take the fp32 FMA path."""
+    w = wl.mlp_workload(n=2, dims=(64, 48, 6), m=300, batch=160, gamma=0.05, seed=13)
+    run, o = _setup(w, seed=5)
+    run.ctx.grad(0)
+    G_ref, _ = mlp_oracle_grad_matching_gates(orc, o, 0, run.g())
+    assert row_rel_err(run.g(), G_ref) <= TOL_G
+    run.close()
