@@ -184,36 +184,55 @@ void run_gemm(dpsgd_ctx* c, const GemmArgs& g) {
     c->launches++;
 }
 
-template <int NT>
-cudaError_t launch_tc_nt(dpsgd_ctx* c, const tc::Args& a, int n_tiles) {
+template <int NT, bool A_K, bool B_K, bool VEC>
+cudaError_t launch_tc_inst(dpsgd_ctx* c, const tc::Args& a, int n_tiles) {
     static bool attr_set = false;
+    auto kernel = tc::tc_gemm_kernel<NT, A_K, B_K, VEC>;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc::tc_gemm_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)tc::smem_bytes<NT>());
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     dim3 grid((a.M + tc::kTileM - 1) / tc::kTileM, n_tiles, c->n);
-    tc::tc_gemm_kernel<NT><<<grid, tc::kThreads, tc::smem_bytes<NT>(), c->stream>>>(a);
+    kernel<<<grid, tc::kThreads, tc::smem_bytes<NT>(), c->stream>>>(a);
     c->launches++;
     return cudaGetLastError();
 }
 
-bool vec_ok(const float* p, int64_t pitch, int64_t node_stride) {
-    return (reinterpret_cast<uintptr_t>(p) % 16 == 0) && (pitch % 4 == 0) && (node_stride % 4 == 0);
+template <int NT, bool VEC>
+cudaError_t launch_tc_nt(dpsgd_ctx* c, const tc::Args& a, int n_tiles) {
+    if (a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, true, true, VEC>(c, a, n_tiles);
+    if (!a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, false, true, VEC>(c, a, n_tiles);
+    if (!a.a_kcontig && !a.b_kcontig) return launch_tc_inst<NT, false, false, VEC>(c, a, n_tiles);
+    return cudaErrorInvalidValue;
+}
+
+// 128-bit loads need 16-byte aligned rows and whole chunks inside the matrix: the extent of the
+// operand's contiguous direction (which equals its pitch here) must be a multiple of 4.
+bool vec_ok(const float* p, int64_t pitch, int64_t node_stride, int contig_extent) {
+    return (reinterpret_cast<uintptr_t>(p) % 16 == 0) && (pitch % 4 == 0) && (node_stride % 4 == 0) &&
+           (contig_extent % 4 == 0);
 }
 
 // C[n][m] = epi(sum_k A(m,k) B(n,k)); max_tile = widest column tile (multiple of 16, <= 128).
 cudaError_t run_tc(dpsgd_ctx* c, tc::Args a, int max_tile) {
-    a.a_vec = vec_ok(a.A, a.a_pitch, a.a_node);
-    a.b_vec = vec_ok(a.B, a.b_pitch, a.b_node);
+    const bool vec = vec_ok(a.A, a.a_pitch, a.a_node, a.a_kcontig ? a.K : a.M) &&
+                     vec_ok(a.B, a.b_pitch, a.b_node, a.b_kcontig ? a.K : a.N);
+    a.a_vec = a.b_vec = vec;
     a.precise = c->mlp_precision == 0;
     a.status = &c->d_result->status;
     const int want = a.N < max_tile ? a.N : max_tile;
-    if (want <= 16) return launch_tc_nt<1>(c, a, (a.N + 15) / 16);
-    if (want <= 32) return launch_tc_nt<2>(c, a, (a.N + 31) / 32);
-    if (want <= 64) return launch_tc_nt<4>(c, a, (a.N + 63) / 64);
-    return launch_tc_nt<8>(c, a, (a.N + 127) / 128);
+    if (vec) {
+        if (want <= 16) return launch_tc_nt<1, true>(c, a, (a.N + 15) / 16);
+        if (want <= 32) return launch_tc_nt<2, true>(c, a, (a.N + 31) / 32);
+        if (want <= 64) return launch_tc_nt<4, true>(c, a, (a.N + 63) / 64);
+        return launch_tc_nt<8, true>(c, a, (a.N + 127) / 128);
+    }
+    if (want <= 16) return launch_tc_nt<1, false>(c, a, (a.N + 15) / 16);
+    if (want <= 32) return launch_tc_nt<2, false>(c, a, (a.N + 31) / 32);
+    if (want <= 64) return launch_tc_nt<4, false>(c, a, (a.N + 63) / 64);
+    return launch_tc_nt<8, false>(c, a, (a.N + 127) / 128);
 }
 
 }  // namespace

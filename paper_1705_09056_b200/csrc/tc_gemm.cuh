@@ -103,72 +103,121 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
     for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
 }
 
-// One 16-byte chunk of an operand tile: four consecutive elements along the operand's contiguous
-// direction, zero outside the matrix.  row / k are tile-global indices.
-template <bool KCONTIG>
-__device__ __forceinline__ float4 load_chunk(const float* __restrict__ src, int64_t pitch, int vec, int row, int k,
-                                             int rows, int K) {
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (KCONTIG) {
-        if (row >= rows || k >= K) return v;
-        const float* p = src + (int64_t)row * pitch + k;
-        if (vec && k + 3 < K) return __ldg(reinterpret_cast<const float4*>(p));
-        v.x = __ldg(p);
-        if (k + 1 < K) v.y = __ldg(p + 1);
-        if (k + 2 < K) v.z = __ldg(p + 2);
-        if (k + 3 < K) v.w = __ldg(p + 3);
-    } else {
-        if (row >= rows || k >= K) return v;
-        const float* p = src + (int64_t)k * pitch + row;
-        if (vec && row + 3 < rows) return __ldg(reinterpret_cast<const float4*>(p));
-        v.x = __ldg(p);
-        if (row + 1 < rows) v.y = __ldg(p + 1);
-        if (row + 2 < rows) v.z = __ldg(p + 2);
-        if (row + 3 < rows) v.w = __ldg(p + 3);
-    }
-    return v;
-}
-
-__device__ __forceinline__ void split_store(unsigned char* hi, unsigned char* lo, uint32_t off, float4 v, int precise) {
-    if (precise) {
-        float4 h, l;
-        h.x = __uint_as_float(__float_as_uint(v.x) & 0xFFFFE000u); l.x = v.x - h.x;
-        h.y = __uint_as_float(__float_as_uint(v.y) & 0xFFFFE000u); l.y = v.y - h.y;
-        h.z = __uint_as_float(__float_as_uint(v.z) & 0xFFFFE000u); l.z = v.z - h.z;
-        h.w = __uint_as_float(__float_as_uint(v.w) & 0xFFFFE000u); l.w = v.w - h.w;
-        *reinterpret_cast<float4*>(hi + off) = h;
-        *reinterpret_cast<float4*>(lo + off) = l;
-    } else {
-        *reinterpret_cast<float4*>(hi + off) = v;
-    }
-}
-
 __device__ __forceinline__ float pick(float4 v, int e) {
     return e == 0 ? v.x : (e == 1 ? v.y : (e == 2 ? v.z : v.w));
 }
 
-// Transposing store: element e of the lane's 128-bit load (four consecutive rows at one k) goes to
-// row (row4 + e), position (k%4) of k-chunk (k/4).  rot in 0..3 staggers the order per lane.
-__device__ __forceinline__ void split_store_rows(unsigned char* hi, unsigned char* lo, uint32_t off_row0, float4 v,
-                                                 int rot, int precise) {
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const int e = (j + rot) & 3;
-        const float x = pick(v, e);
-        const uint32_t off = off_row0 + (uint32_t)e * 16;
-        if (precise) {
-            const float h = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
-            *reinterpret_cast<float*>(hi + off) = h;
-            *reinterpret_cast<float*>(lo + off) = x - h;
+// One loader thread's share of an operand tile (ROWS x 32 k): ROWS/16 chunks of 16 bytes, i.e.
+// four consecutive elements along the operand's contiguous direction.
+//   KC  : the operand is contiguous along k in memory (element (r,k) at r*pitch + k)
+//   !KC : it is contiguous along its row index (element (r,k) at k*pitch + r) and is transposed
+//         on the way to shared memory
+//   VEC : 128-bit loads are legal (16-byte aligned rows, extent of the contiguous direction a
+//         multiple of 4); otherwise the four elements are loaded and bounds-checked one by one.
+// Lane mapping: 8 lanes along the slow direction x 4 lanes along the contiguous one, so a warp
+// reads 8 segments of 64 bytes; successive chunks of a thread are 16 rows apart.  Loads are
+// predicated, never branched around, so that all of a thread's loads are in flight together.
+template <int ROWS, bool KC, bool VEC>
+struct OperandLoader {
+    static constexpr int T = ROWS / 16;
+    const float* ptr0;
+    int64_t tstride, kstride;
+    int row0, kfix, rows, K;
+    uint32_t soff0;      // shared-memory byte offset of chunk 0 inside the hi (or lo) tile
+    int rot;
+
+    __device__ __forceinline__ void init(const float* src, int64_t pitch, int warp, int lane, int row_base,
+                                         int rows_, int K_) {
+        rows = rows_; K = K_;
+        if (KC) {
+            const int rl = (warp >> 1) * 8 + (lane & 7);
+            kfix = ((warp & 1) * 4 + (lane >> 3)) * 4;
+            row0 = row_base + rl;
+            ptr0 = src + (int64_t)row0 * pitch + kfix;
+            tstride = 16 * pitch; kstride = kBlockK;
+            soff0 = (uint32_t)(kfix >> 2) * (ROWS * 16) + (uint32_t)rl * 16;
+            rot = 0;
         } else {
-            *reinterpret_cast<float*>(hi + off) = x;
+            const int rl = (lane >> 3) * 4;
+            kfix = warp * 8 + (lane & 7);
+            row0 = row_base + rl;
+            ptr0 = src + (int64_t)kfix * pitch + row0;
+            tstride = 16; kstride = (int64_t)kBlockK * pitch;
+            soff0 = (uint32_t)(kfix >> 2) * (ROWS * 16) + (uint32_t)rl * 16 + (uint32_t)(kfix & 3) * 4;
+            rot = ((lane >> 2) & 1) + 2 * (lane >> 4);
         }
     }
-}
 
-// NT = column tile / 16 (B operand rows per CTA = 16 * NT <= 128).
+    __device__ __forceinline__ void fetch(int kb, float4 (&r)[T]) const {
+        const int k = kb * kBlockK + kfix;
+        const float* p = ptr0 + (int64_t)kb * kstride;
+#pragma unroll
+        for (int t = 0; t < T; ++t) {
+            const int row = row0 + 16 * t;
+            const float* q = p + (int64_t)t * tstride;
+            if (VEC) {
+                const bool in = (k < K) && (row < rows);
+                r[t] = in ? __ldg(reinterpret_cast<const float4*>(q)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            } else if (KC) {
+                const bool in = row < rows;
+                r[t].x = (in && k < K) ? __ldg(q) : 0.f;
+                r[t].y = (in && k + 1 < K) ? __ldg(q + 1) : 0.f;
+                r[t].z = (in && k + 2 < K) ? __ldg(q + 2) : 0.f;
+                r[t].w = (in && k + 3 < K) ? __ldg(q + 3) : 0.f;
+            } else {
+                const bool in = k < K;
+                r[t].x = (in && row < rows) ? __ldg(q) : 0.f;
+                r[t].y = (in && row + 1 < rows) ? __ldg(q + 1) : 0.f;
+                r[t].z = (in && row + 2 < rows) ? __ldg(q + 2) : 0.f;
+                r[t].w = (in && row + 3 < rows) ? __ldg(q + 3) : 0.f;
+            }
+        }
+    }
+
+    // Split each value into its TF32 head and the remainder and write both tiles (only the raw
+    // value when precise == 0).  K-major canonical layout: (r,k) at (k/4)*ROWS*16 + r*16 + (k%4)*4.
+    __device__ __forceinline__ void store(unsigned char* hi, unsigned char* lo, const float4 (&r)[T], int precise) const {
+#pragma unroll
+        for (int t = 0; t < T; ++t) {
+            const uint32_t off = soff0 + (uint32_t)t * 256;       // 16 rows further
+            const float4 v = r[t];
+            if (KC) {
+                if (precise) {
+                    float4 h, l;
+                    h.x = __uint_as_float(__float_as_uint(v.x) & 0xFFFFE000u); l.x = v.x - h.x;
+                    h.y = __uint_as_float(__float_as_uint(v.y) & 0xFFFFE000u); l.y = v.y - h.y;
+                    h.z = __uint_as_float(__float_as_uint(v.z) & 0xFFFFE000u); l.z = v.z - h.z;
+                    h.w = __uint_as_float(__float_as_uint(v.w) & 0xFFFFE000u); l.w = v.w - h.w;
+                    *reinterpret_cast<float4*>(hi + off) = h;
+                    *reinterpret_cast<float4*>(lo + off) = l;
+                } else {
+                    *reinterpret_cast<float4*>(hi + off) = v;
+                }
+            } else {
+                // the four elements go to four rows; the order is rotated per lane so that the 32
+                // scalar stores of a warp fall into 32 different banks
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int e = (j + rot) & 3;
+                    const float x = pick(v, e);
+                    const uint32_t o = off + (uint32_t)e * 16;
+                    if (precise) {
+                        const float h = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
+                        *reinterpret_cast<float*>(hi + o) = h;
+                        *reinterpret_cast<float*>(lo + o) = x - h;
+                    } else {
+                        *reinterpret_cast<float*>(hi + o) = x;
+                    }
+                }
+            }
+        }
+    }
+};
+
+// NT = column tile / 16 (B operand rows per CTA = 16 * NT <= 128); A_K / B_K: operand contiguous
+// along k in memory; VEC: both operands allow 128-bit loads.
 // Grid: (ceil(M/128), ceil(N/(16 NT)), nodes).
-template <int NT>
+template <int NT, bool A_K, bool B_K, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 tc_gemm_kernel(Args g) {
     constexpr int ROWS_A = kTileM, ROWS_B = 16 * NT;
@@ -182,19 +231,15 @@ tc_gemm_kernel(Args g) {
     uint64_t* empty = full + kStages;
     uint64_t* accum = empty + kStages;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
-    volatile int* aborted = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int node = blockIdx.z;
     const int m0 = blockIdx.x * kTileM, n0 = blockIdx.y * ROWS_B;
-    const float* A = g.A + (int64_t)node * g.a_node;
-    const float* Bp = g.B + (int64_t)node * g.b_node;
     const int KB = (g.K + kBlockK - 1) / kBlockK;
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(full + s, kLoaderThreads); mbar_init(empty + s, 1); }
         mbar_init(accum, 1);
-        *aborted = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 4) {
@@ -209,78 +254,38 @@ tc_gemm_kernel(Args g) {
 
     if (warp < 4) {
         // ------------------------------ loaders ------------------------------
-        float4 ra[TA], rb[TB];
-        auto fetch = [&](int kb) {
-            const int k0 = kb * kBlockK;
-#pragma unroll
-            for (int t = 0; t < TA; ++t) {
-                const int task = warp + 4 * t;
-                if (g.a_kcontig) {       // task -> (row group of 8, half of the 8 k-chunks)
-                    const int row = (task >> 1) * 8 + (lane & 7), kc = (task & 1) * 4 + (lane >> 3);
-                    ra[t] = load_chunk<true>(A, g.a_pitch, g.a_vec, m0 + row, k0 + kc * 4, g.M, g.K);
-                } else {                 // task -> (k group of 8, group of 4 chunks along m)
-                    const int k = (task & 3) * 8 + (lane & 7), m4 = (task >> 2) * 4 + (lane >> 3);
-                    ra[t] = load_chunk<false>(A, g.a_pitch, g.a_vec, m0 + m4 * 4, k0 + k, g.M, g.K);
-                }
-            }
-#pragma unroll
-            for (int t = 0; t < TB; ++t) {
-                const int task = warp + 4 * t;
-                if (g.b_kcontig) {
-                    const int row = (task >> 1) * 8 + (lane & 7), kc = (task & 1) * 4 + (lane >> 3);
-                    rb[t] = load_chunk<true>(Bp, g.b_pitch, g.b_vec, n0 + row, k0 + kc * 4, g.N, g.K);
-                } else {
-                    const int k = (task & 3) * 8 + (lane & 7), n4 = (task >> 2) * 4 + (lane >> 3);
-                    rb[t] = load_chunk<false>(Bp, g.b_pitch, g.b_vec, n0 + n4 * 4, k0 + k, g.N, g.K);
-                }
-            }
-        };
-        auto store = [&](int s) {
-            unsigned char* base = smem + s * STAGE;
-#pragma unroll
-            for (int t = 0; t < TA; ++t) {
-                const int task = warp + 4 * t;
-                if (g.a_kcontig) {
-                    const int row = (task >> 1) * 8 + (lane & 7), kc = (task & 1) * 4 + (lane >> 3);
-                    split_store(base, base + A_BYTES, (uint32_t)kc * (ROWS_A * 16) + (uint32_t)row * 16, ra[t], g.precise);
-                } else {
-                    const int k = (task & 3) * 8 + (lane & 7), m4 = (task >> 2) * 4 + (lane >> 3);
-                    const uint32_t off = (uint32_t)(k >> 2) * (ROWS_A * 16) + (uint32_t)(m4 * 4) * 16 + (uint32_t)(k & 3) * 4;
-                    split_store_rows(base, base + A_BYTES, off, ra[t], ((lane >> 2) & 1) + 2 * (lane >> 4), g.precise);
-                }
-            }
-#pragma unroll
-            for (int t = 0; t < TB; ++t) {
-                const int task = warp + 4 * t;
-                if (g.b_kcontig) {
-                    const int row = (task >> 1) * 8 + (lane & 7), kc = (task & 1) * 4 + (lane >> 3);
-                    split_store(base + 2 * A_BYTES, base + 2 * A_BYTES + B_BYTES,
-                                (uint32_t)kc * (ROWS_B * 16) + (uint32_t)row * 16, rb[t], g.precise);
-                } else {
-                    const int k = (task & 3) * 8 + (lane & 7), n4 = (task >> 2) * 4 + (lane >> 3);
-                    const uint32_t off = (uint32_t)(k >> 2) * (ROWS_B * 16) + (uint32_t)(n4 * 4) * 16 + (uint32_t)(k & 3) * 4;
-                    split_store_rows(base + 2 * A_BYTES, base + 2 * A_BYTES + B_BYTES, off, rb[t],
-                                     ((lane >> 2) & 1) + 2 * (lane >> 4), g.precise);
-                }
-            }
-        };
+        OperandLoader<ROWS_A, A_K, VEC> la;
+        OperandLoader<ROWS_B, B_K, VEC> lb;
+        la.init(g.A + (int64_t)node * g.a_node, g.a_pitch, warp, lane, m0, g.M, g.K);
+        lb.init(g.B + (int64_t)node * g.b_node, g.b_pitch, warp, lane, n0, g.N, g.K);
+        float4 ra0[TA], rb0[TB], ra1[TA], rb1[TB];       // two k-blocks in flight
         bool ok = true;
-        if (KB > 0) fetch(0);
-        for (int kb = 0; kb < KB && ok; ++kb) {
+        la.fetch(0, ra0); lb.fetch(0, rb0);
+        if (KB > 1) { la.fetch(1, ra1); lb.fetch(1, rb1); }
+        auto put = [&](int kb, const float4 (&ra)[TA], const float4 (&rb)[TB]) -> bool {
             const int s = kb % kStages;
             const uint32_t fill = (uint32_t)(kb / kStages);
-            if (!mbar_wait(empty + s, (fill & 1u) ^ 1u)) { ok = false; break; }
-            store(s);
+            if (!mbar_wait(empty + s, (fill & 1u) ^ 1u)) return false;
+            unsigned char* base = smem + s * STAGE;
+            la.store(base, base + A_BYTES, ra, g.precise);
+            lb.store(base + 2 * A_BYTES, base + 2 * A_BYTES + B_BYTES, rb, g.precise);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mbar_arrive(full + s);
-            if (kb + 1 < KB) fetch(kb + 1);
+            return true;
+        };
+        for (int kb = 0; kb < KB && ok; kb += 2) {
+            ok = put(kb, ra0, rb0);
+            if (ok && kb + 2 < KB) { la.fetch(kb + 2, ra0); lb.fetch(kb + 2, rb0); }
+            if (ok && kb + 1 < KB) {
+                ok = put(kb + 1, ra1, rb1);
+                if (ok && kb + 3 < KB) { la.fetch(kb + 3, ra1); lb.fetch(kb + 3, rb1); }
+            }
         }
         // ------------------------------ epilogue ------------------------------
         if (ok && !mbar_wait(accum, 0)) ok = false;
         ok = __all_sync(0xffffffffu, ok);      // tcgen05.ld below needs the whole warp
         if (!ok) {
             if (lane == 0) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
-            *aborted = 1;
         } else {
             tc_fence_after();
             const int m = m0 + warp * 32 + lane;
@@ -335,7 +340,7 @@ tc_gemm_kernel(Args g) {
             mma_commit(empty + s);      // frees the stage once these MMAs have read it
         }
         if (ok) mma_commit(accum);      // accumulator complete
-        else { atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT); *aborted = 1; }
+        else atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
     }
     tc_fence_before();
     __syncthreads();
