@@ -74,7 +74,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     for (uint32_t spin = 0; spin < kWaitSpins; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (spin > 64) __nanosleep(100);
+        if (spin > 4096) __nanosleep(128);    // try_wait already blocks briefly; sleep only on long waits
     }
     return false;
 }

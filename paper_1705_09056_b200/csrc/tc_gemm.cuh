@@ -28,8 +28,8 @@ constexpr int kLoaderThreads = 128;
 constexpr int kThreads = 160;          // 4 loader/epilogue warps + 1 MMA warp
 constexpr int kTileM = 128;
 constexpr int kBlockK = 32;            // fp32 elements per pipeline stage along k (4 MMAs of K = 8)
-constexpr int kStages = 2;
-constexpr uint32_t kWaitSpins = 1u << 22;
+constexpr int kStages = 1;            // one stage per CTA: four CTAs share an SM and overlap each other
+constexpr uint32_t kWaitSpins = 1u << 21;
 
 enum { EPI_BIAS_RELU = 0, EPI_BIAS = 1, EPI_STORE = 2, EPI_MASK = 3 };
 
@@ -62,9 +62,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    // try_wait itself blocks for a short hardware-defined slice, so plain polling is cheap; back
+    // off with nanosleep (coarse: it can cost a microsecond) only once the wait is clearly long
     for (uint32_t spin = 0; spin < kWaitSpins; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (spin > 32) __nanosleep(64);
+        if (spin > 4096) __nanosleep(128);
     }
     return false;
 }
@@ -218,7 +220,7 @@ struct OperandLoader {
 // along k in memory; VEC: both operands allow 128-bit loads.
 // Grid: (ceil(M/128), ceil(N/(16 NT)), nodes).
 template <int NT, bool A_K, bool B_K, bool VEC>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, NT <= 4 ? 4 : 2)
 tc_gemm_kernel(Args g) {
     constexpr int ROWS_A = kTileM, ROWS_B = 16 * NT;
     constexpr uint32_t A_BYTES = ROWS_A * kBlockK * 4, B_BYTES = ROWS_B * kBlockK * 4;
@@ -258,28 +260,22 @@ tc_gemm_kernel(Args g) {
         OperandLoader<ROWS_B, B_K, VEC> lb;
         la.init(g.A + (int64_t)node * g.a_node, g.a_pitch, warp, lane, m0, g.M, g.K);
         lb.init(g.B + (int64_t)node * g.b_node, g.b_pitch, warp, lane, n0, g.N, g.K);
-        float4 ra0[TA], rb0[TB], ra1[TA], rb1[TB];       // two k-blocks in flight
+        // One k-block per thread in flight: the proxy fence below also waits for the thread's
+        // outstanding global loads, so deeper register prefetch would not overlap anything.  Memory
+        // parallelism comes from the CTAs that share the SM.
+        float4 ra[TA], rb[TB];
         bool ok = true;
-        la.fetch(0, ra0); lb.fetch(0, rb0);
-        if (KB > 1) { la.fetch(1, ra1); lb.fetch(1, rb1); }
-        auto put = [&](int kb, const float4 (&ra)[TA], const float4 (&rb)[TB]) -> bool {
+        la.fetch(0, ra); lb.fetch(0, rb);
+        for (int kb = 0; kb < KB; ++kb) {
             const int s = kb % kStages;
             const uint32_t fill = (uint32_t)(kb / kStages);
-            if (!mbar_wait(empty + s, (fill & 1u) ^ 1u)) return false;
+            if (!mbar_wait(empty + s, (fill & 1u) ^ 1u)) { ok = false; break; }
             unsigned char* base = smem + s * STAGE;
             la.store(base, base + A_BYTES, ra, g.precise);
             lb.store(base + 2 * A_BYTES, base + 2 * A_BYTES + B_BYTES, rb, g.precise);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mbar_arrive(full + s);
-            return true;
-        };
-        for (int kb = 0; kb < KB && ok; kb += 2) {
-            ok = put(kb, ra0, rb0);
-            if (ok && kb + 2 < KB) { la.fetch(kb + 2, ra0); lb.fetch(kb + 2, rb0); }
-            if (ok && kb + 1 < KB) {
-                ok = put(kb + 1, ra1, rb1);
-                if (ok && kb + 3 < KB) { la.fetch(kb + 3, ra1); lb.fetch(kb + 3, rb1); }
-            }
+            if (kb + 1 < KB) { la.fetch(kb + 1, ra); lb.fetch(kb + 1, rb); }
         }
         // ------------------------------ epilogue ------------------------------
         if (ok && !mbar_wait(accum, 0)) ok = false;
