@@ -284,9 +284,10 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one mix_ring_kernel launch (ncu), or None while
-# no capture of the current kernel exists.
-TRAFFIC_BYTES_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one mix_ring_kernel launch.  Captured with ncu on
+# n = 64 x N = 2,000,000 (1.499 GB against 1.536 GB algorithmic) and scaled by 25,000,000 / 2,000,000:
+# traffic grows in proportion to N.  Set to None whenever mix_ring_kernel changes.
+TRAFFIC_BYTES_PER_LAUNCH = 18.74e9
 
 
 def main():

@@ -1,0 +1,134 @@
+"""GPU parity at the full sizes of the model configurations, on what the oracle can afford:
+all indices (bit-exact), whole steps where the oracle finishes in seconds, sampled nodes and
+column slices where it does not."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dpsgd_oracle as orc
+from paper_1705_09056_b200 import binding, workloads as wl
+from gpu_util import row_rel_err, mlp_oracle_grad_matching_gates, TOL_STEP
+
+pytestmark = pytest.mark.gpu
+
+
+def _need(gib):
+    free, _ = torch.cuda.mem_get_info()
+    if free < gib * 2 ** 30:
+        pytest.skip(f"needs {gib} GiB of device memory")
+
+
+def _context(w, seed):
+    X0 = wl.stack_rows(w.x0, w.n, w.ld)
+    X1, G = torch.zeros_like(X0), torch.zeros_like(X0)
+    ctx = binding.Dpsgd(w.n, w.N, *w.csr(), gamma=w.gamma, seed=seed)
+    ctx.bind(X0, X1, G)
+    ctx.set_model(w.model, w.dims, w.l2_lambda, w.batch, 0)
+    ctx.set_data(w.A, w.y)
+    return ctx, X0, X1, G
+
+
+def test_config2_full_size_logistic_steps():
+    """n = 16, 65536 x 4096 local samples per node (17.2 GB on the device).  The oracle sees the
+    sampled rows only: they are gathered by the oracle's own indices, which must equal the
+    library's bit for bit."""
+    _need(24)
+    w = wl.config(1, device="cuda")
+    seed = 4242
+    ctx, X0, X1, G = _context(w, seed)
+    csr = w.csr()
+    rng = np.random.default_rng(0)
+    X = (0.05 * rng.standard_normal((w.n, w.N))).astype(np.float32)
+    for k in (0, 1, 999):
+        idx = orc.sample_indices(seed, k, w.n, w.batch, w.m_per_node)
+        assert np.array_equal(ctx.sample(k).cpu().numpy(), idx)
+        it = torch.from_numpy(idx.astype(np.int64)).cuda()
+        A_s = torch.stack([w.A[i][it[i]] for i in range(w.n)]).cpu().numpy()      # [n][B][d]
+        y_s = torch.stack([w.y[i][it[i]] for i in range(w.n)]).cpu().numpy()
+        local = np.tile(np.arange(w.batch, dtype=np.int32), (w.n, 1))
+        G_ref = orc.gradients(X, orc.MODEL_LOGISTIC, w.dims, A_s, y_s, local, w.l2_lambda)
+        X_ref = orc.mix_update(X, G_ref, *csr, w.gamma)
+        ctx.current()[:, :w.N] = torch.from_numpy(X).cuda()
+        ctx.step(k)
+        assert row_rel_err(G[:, :w.N].cpu().numpy(), G_ref) <= 2e-5
+        assert row_rel_err(ctx.current()[:, :w.N].cpu().numpy(), X_ref) <= TOL_STEP
+        X = X_ref
+    ctx.close()
+
+
+def test_config3_full_size_mlp_steps():
+    """n = 32 ring, MLP 784-1024-10, 1875 samples per node, minibatch 32: whole steps."""
+    w = wl.config(2, device="cuda")
+    seed = 31
+    ctx, X0, X1, G = _context(w, seed)
+    A, y = w.A.cpu().numpy(), w.y.cpu().numpy()
+    o = orc.Oracle(w.n, w.N, *w.csr(), w.gamma, seed, w.model, w.dims, w.batch, 0.0, A, y)
+    o.set_x(np.tile(w.x0.cpu().numpy(), (w.n, 1)))
+    for k in range(3):
+        assert np.array_equal(ctx.sample(k).cpu().numpy(), o.sample(k))
+        ctx.current()[:, :w.N] = torch.from_numpy(o.X).cuda()      # per-step parity: same start
+        ctx.grad(k)
+        G_gpu = G[:, :w.N].cpu().numpy()
+        G_ref, _ = mlp_oracle_grad_matching_gates(orc, o, k, G_gpu)
+        assert row_rel_err(G_gpu, G_ref) <= 5e-5
+        ctx.mix_update()
+        X_ref = o.mix_update(G_ref)
+        assert row_rel_err(ctx.current()[:, :w.N].cpu().numpy(), X_ref) <= TOL_STEP
+    ctx.close()
+
+
+def test_config5_full_size_sampled_nodes_and_columns():
+    """n = 112, MLP 1024-2048-2048-10 (6.3 M parameters per node), ring next to the dense
+    averaging matrix.  The oracle computes the gradient of a few sampled nodes and the gossip
+    step on column slices of all rows; the consensus distance is checked against the closed form
+    it has under dense W."""
+    _need(16)
+    w = wl.config(4, device="cuda")
+    seed = 77
+    ctx, X0, X1, G = _context(w, seed)
+    rng = np.random.default_rng(3)
+    # rows differ: shared He init plus a small per-node perturbation
+    X0[:, :w.N] += 0.01 * torch.randn((w.n, w.N), device="cuda", generator=torch.Generator("cuda").manual_seed(5))
+    k = 11
+    idx = orc.sample_indices(seed, k, w.n, w.batch, w.m_per_node)
+    assert np.array_equal(ctx.sample(k).cpu().numpy(), idx)
+    ctx.grad(k)
+    nodes = [0, 55, 111] + [int(v) for v in rng.integers(1, 111, 2)]
+    for i in nodes:
+        x_i = X0[i, :w.N].cpu().numpy()
+        A_i, y_i = w.A[i].cpu().numpy(), w.y[i].cpu().numpy()
+        g_gpu = G[i, :w.N].cpu().numpy()
+        ties = orc.mlp_near_zero_gates(x_i, w.dims, A_i, idx[i], 4e-6)
+        best = None
+        chosen = []
+        for t in [None] + ties[:32]:
+            cand = orc.grad_mlp(x_i, w.dims, A_i, y_i, idx[i], flip=chosen + ([t] if t else [])).astype(np.float32)
+            err = np.linalg.norm(cand.astype(np.float64) - g_gpu)
+            if best is None or err < best[0]:
+                best = (err, cand)
+                if t:
+                    chosen.append(t)
+        ref = best[1]
+        assert np.linalg.norm(ref.astype(np.float64) - g_gpu) <= 5e-5 * np.linalg.norm(ref), i
+    # gossip step on column slices (separable per column), ring then dense
+    width = 20_000
+    starts = [0, w.N - width] + [int(s) for s in rng.integers(width, w.N - 2 * width, 2)]
+    Xh = {s: X0[:, s:s + width].cpu().numpy() for s in starts}
+    Gh = {s: G[:, s:s + width].cpu().numpy() for s in starts}
+    ctx.mix_update()
+    out = ctx.current()
+    for s in starts:
+        ref = orc.mix_update(Xh[s], Gh[s], *w.csr(), w.gamma)
+        assert row_rel_err(out[:, s:s + width].cpu().numpy(), ref) <= TOL_STEP
+    ctx.close()
+    # dense W: every row becomes xbar - gamma g_i, so the consensus distance is gamma^2 sum ||g_i - gbar||^2
+    wd = wl.Workload("mlp", w.n, w.N, "dense", w.gamma, 1)
+    dctx = binding.Dpsgd(w.n, w.N, *wd.csr(), gamma=w.gamma, seed=seed)
+    X1.zero_()
+    dctx.bind(X0, X1, G)
+    dctx.mix_update()
+    g64 = G[:, :w.N].double()
+    expect = float(np.float64(np.float32(w.gamma)) ** 2 * ((g64 - g64.mean(dim=0)) ** 2).sum())
+    got = dctx.consensus_dist()
+    assert abs(got - expect) <= 1e-3 * expect
+    dctx.close()
