@@ -184,27 +184,33 @@ void run_gemm(dpsgd_ctx* c, const GemmArgs& g) {
     c->launches++;
 }
 
-template <int NT, bool A_K, bool B_K, bool VEC>
+template <int NT, bool A_K, bool B_K, bool VEC, bool PRECISE>
 cudaError_t launch_tc_inst(dpsgd_ctx* c, const tc::Args& a, int n_tiles) {
     static bool attr_set = false;
-    auto kernel = tc::tc_gemm_kernel<NT, A_K, B_K, VEC>;
+    auto kernel = tc::tc_gemm_kernel<NT, A_K, B_K, VEC, PRECISE>;
+    constexpr size_t smem = tc::smem_bytes<NT, PRECISE>();
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)tc::smem_bytes<NT>());
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     dim3 grid((a.M + tc::kTileM - 1) / tc::kTileM, n_tiles, c->n);
-    kernel<<<grid, tc::kThreads, tc::smem_bytes<NT>(), c->stream>>>(a);
+    kernel<<<grid, tc::kThreads, smem, c->stream>>>(a);
     c->launches++;
     return cudaGetLastError();
 }
 
 template <int NT, bool VEC>
 cudaError_t launch_tc_nt(dpsgd_ctx* c, const tc::Args& a, int n_tiles) {
-    if (a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, true, true, VEC>(c, a, n_tiles);
-    if (!a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, false, true, VEC>(c, a, n_tiles);
-    if (!a.a_kcontig && !a.b_kcontig) return launch_tc_inst<NT, false, false, VEC>(c, a, n_tiles);
+    if (a.precise) {
+        if (a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, true, true, VEC, true>(c, a, n_tiles);
+        if (!a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, false, true, VEC, true>(c, a, n_tiles);
+        if (!a.a_kcontig && !a.b_kcontig) return launch_tc_inst<NT, false, false, VEC, true>(c, a, n_tiles);
+    } else {
+        if (a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, true, true, VEC, false>(c, a, n_tiles);
+        if (!a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, false, true, VEC, false>(c, a, n_tiles);
+        if (!a.a_kcontig && !a.b_kcontig) return launch_tc_inst<NT, false, false, VEC, false>(c, a, n_tiles);
+    }
     return cudaErrorInvalidValue;
 }
 

@@ -6,13 +6,17 @@
 // slice) on the TMEM columns.  tcgen05.mma kind::tf32 multiplies 10-bit-mantissa operands, so an
 // fp32-faithful product is built from three MMAs on split operands (a = a_hi + a_lo):
 //     a*b ~= a_hi*b_hi + a_lo*b_hi + a_hi*b_lo        (fp32 accumulation in TMEM)
-// The operands are fp32 in HBM.  Four loader warps read them with 128-bit loads (64-byte segments
-// per row), split them in registers and write hi / lo copies to shared memory directly in the
-// no-swizzle K-major canonical layout the MMA descriptors describe (core matrix = 8 rows x 16 B,
-// element (r,k) at (k/4)*LBO + r*16 + (k%4)*4).  An operand that is contiguous along m / n in
-// memory is transposed on the way: each lane scatters the four elements of its 128-bit load to
-// four rows, rotated per lane so that a warp's 32 stores hit 32 different banks.  (tcgen05 has
-// no no-swizzle MN-major mode for 32-bit operands.)  One thread of a fifth warp
+// The operands are fp32 in HBM.  Four loader warps read them with 128-bit loads, 64 k at a time,
+// shaped so that one warp instruction covers 256 contiguous bytes of a row (k-contiguous operand)
+// or 128 bytes of each of four k-rows (operand contiguous along m / n): measured on B200, 64-byte
+// pieces reach 2.5 TB/s, full 128-byte lines 3.5 and 256-byte runs 5.1.  The values are split in
+// registers and written as hi / lo copies to shared memory directly in the no-swizzle K-major
+// layout the MMA descriptors describe: element (r,k) at (k/4)*LBO + (r/8)*128 + (r%8)*16 + (k%4)*4.
+// The descriptor arithmetic is linear in LBO, so LBO carries 16 bytes of padding per chunk column
+// and the 128-bit stores of lanes that run along k fall into different banks.  An operand that is
+// contiguous along m / n is transposed on the way: each lane scatters the four elements of its load
+// to four rows, in an order rotated per lane so that a warp's 32 scalar stores hit 32 banks.
+// (tcgen05 has no no-swizzle MN-major mode for 32-bit operands.)  One thread of a fifth warp
 // issues the MMAs; tcgen05.commit releases a stage back to the loaders; the loader warps then
 // read the accumulator with tcgen05.ld and apply the epilogue with coalesced stores (m contiguous).
 // Every mbarrier wait is bounded; a wait that runs out raises the status word, and the CTA still
@@ -27,7 +31,8 @@ namespace tc {
 constexpr int kLoaderThreads = 128;
 constexpr int kThreads = 160;          // 4 loader/epilogue warps + 1 MMA warp
 constexpr int kTileM = 128;
-constexpr int kBlockK = 32;            // fp32 elements per pipeline stage along k (4 MMAs of K = 8)
+constexpr int kBlockK = 64;            // fp32 elements per pipeline stage along k (8 MMAs of K = 8)
+constexpr int kChunks = kBlockK / 4;   // 16-byte chunk columns per stage
 constexpr int kStages = 1;            // one stage per CTA: four CTAs share an SM and overlap each other
 constexpr uint32_t kWaitSpins = 1u << 21;
 
@@ -109,56 +114,57 @@ __device__ __forceinline__ float pick(float4 v, int e) {
     return e == 0 ? v.x : (e == 1 ? v.y : (e == 2 ? v.z : v.w));
 }
 
-// One loader thread's share of an operand tile (ROWS x 32 k): ROWS/16 chunks of 16 bytes, i.e.
-// four consecutive elements along the operand's contiguous direction.
-//   KC  : the operand is contiguous along k in memory (element (r,k) at r*pitch + k)
-//   !KC : it is contiguous along its row index (element (r,k) at k*pitch + r) and is transposed
-//         on the way to shared memory
+// Byte distance between consecutive 16-byte chunk columns of a ROWS-row operand tile.
+__host__ __device__ constexpr uint32_t tile_lbo(int rows) { return (uint32_t)rows * 16 + 16; }
+__host__ __device__ constexpr uint32_t tile_bytes(int rows) { return kChunks * tile_lbo(rows); }
+
+// One loader thread's share of an operand tile (ROWS x 64 k) as 16-byte chunks, i.e. four
+// consecutive elements along the operand's contiguous direction.
+//   KC  : the operand is contiguous along k in memory (element (r,k) at r*pitch + k).  Lanes 0-15
+//         cover the 16 chunks (256 bytes) of one row, lanes 16-31 the next row; a chunk is stored
+//         as it is (four k of one row).
+//   !KC : it is contiguous along its row index (element (r,k) at k*pitch + r) and is transposed on
+//         the way to shared memory.  ROWS/4 lanes cover all rows of one k (512 bytes for 128 rows);
+//         a thread loads the same four rows at four consecutive k, transposes the 4x4 block in
+//         registers (free) and stores four chunks, one per row, in an order rotated per lane so
+//         that the 128-bit stores of a quarter warp fall into different banks.
 //   VEC : 128-bit loads are legal (16-byte aligned rows, extent of the contiguous direction a
 //         multiple of 4); otherwise the four elements are loaded and bounds-checked one by one.
-// Lane mapping: 8 lanes along the slow direction x 4 lanes along the contiguous one, so a warp
-// reads 8 segments of 64 bytes; successive chunks of a thread are 16 rows apart.  Loads are
-// predicated, never branched around, so that all of a thread's loads are in flight together.
+// Loads are predicated, never branched around, so that all of a thread's loads are in flight together.
 template <int ROWS, bool KC, bool VEC>
 struct OperandLoader {
-    static constexpr int T = ROWS / 16;
-    const float* ptr0;
-    int64_t tstride, kstride;
-    int row0, kfix, rows, K;
-    uint32_t soff0;      // shared-memory byte offset of chunk 0 inside the hi (or lo) tile
-    int rot;
+    static constexpr int LPR = ROWS / 4;                       // !KC: lanes per k-row
+    static constexpr int G = 32 / LPR;                         // !KC: chunk columns per warp instruction
+    static constexpr int ROUNDS = (kChunks + 4 * G - 1) / (4 * G);
+    static constexpr int T = KC ? ROWS / 8 : 4 * ROUNDS;
+    static constexpr uint32_t LBO = tile_lbo(ROWS);
+    const float* src;
+    int64_t pitch;
+    int row_base, rows, K, warp, lane;
 
-    __device__ __forceinline__ void init(const float* src, int64_t pitch, int warp, int lane, int row_base,
+    __device__ __forceinline__ void init(const float* src_, int64_t pitch_, int warp_, int lane_, int row_base_,
                                          int rows_, int K_) {
-        rows = rows_; K = K_;
-        if (KC) {
-            const int rl = (warp >> 1) * 8 + (lane & 7);
-            kfix = ((warp & 1) * 4 + (lane >> 3)) * 4;
-            row0 = row_base + rl;
-            ptr0 = src + (int64_t)row0 * pitch + kfix;
-            tstride = 16 * pitch; kstride = kBlockK;
-            soff0 = (uint32_t)(kfix >> 2) * (ROWS * 16) + (uint32_t)rl * 16;
-            rot = 0;
-        } else {
-            const int rl = (lane >> 3) * 4;
-            kfix = warp * 8 + (lane & 7);
-            row0 = row_base + rl;
-            ptr0 = src + (int64_t)kfix * pitch + row0;
-            tstride = 16; kstride = (int64_t)kBlockK * pitch;
-            soff0 = (uint32_t)(kfix >> 2) * (ROWS * 16) + (uint32_t)rl * 16 + (uint32_t)(kfix & 3) * 4;
-            rot = ((lane >> 2) & 1) + 2 * (lane >> 4);
-        }
+        src = src_; pitch = pitch_; warp = warp_; lane = lane_; row_base = row_base_; rows = rows_; K = K_;
     }
+    // KC: tile-local row of chunk t (its 16-byte chunk column is lane & 15)
+    __device__ __forceinline__ int krow(int t) const { return (t * 4 + warp) * 2 + (lane >> 4); }
+    // !KC: chunk column of round u (rows are (lane % LPR) * 4 .. +3)
+    __device__ __forceinline__ int tcol(int u) const { return (u * 4 + warp) * G + lane / LPR; }
 
     __device__ __forceinline__ void fetch(int kb, float4 (&r)[T]) const {
-        const int k = kb * kBlockK + kfix;
-        const float* p = ptr0 + (int64_t)kb * kstride;
 #pragma unroll
         for (int t = 0; t < T; ++t) {
-            const int row = row0 + 16 * t;
-            const float* q = p + (int64_t)t * tstride;
+            int row, k;
+            bool tile_ok = true;
+            if (KC) { row = row_base + krow(t); k = kb * kBlockK + (lane & 15) * 4; }
+            else {
+                const int c = tcol(t >> 2);
+                tile_ok = c < kChunks;
+                row = row_base + (lane % LPR) * 4; k = kb * kBlockK + c * 4 + (t & 3);
+            }
+            const float* q = KC ? src + (int64_t)row * pitch + k : src + (int64_t)k * pitch + row;
             if (VEC) {
-                const bool in = (k < K) && (row < rows);
+                const bool in = tile_ok && (k < K) && (row < rows);
                 r[t] = in ? __ldg(reinterpret_cast<const float4*>(q)) : make_float4(0.f, 0.f, 0.f, 0.f);
             } else if (KC) {
                 const bool in = row < rows;
@@ -167,7 +173,7 @@ struct OperandLoader {
                 r[t].z = (in && k + 2 < K) ? __ldg(q + 2) : 0.f;
                 r[t].w = (in && k + 3 < K) ? __ldg(q + 3) : 0.f;
             } else {
-                const bool in = k < K;
+                const bool in = tile_ok && k < K;
                 r[t].x = (in && row < rows) ? __ldg(q) : 0.f;
                 r[t].y = (in && row + 1 < rows) ? __ldg(q + 1) : 0.f;
                 r[t].z = (in && row + 2 < rows) ? __ldg(q + 2) : 0.f;
@@ -176,39 +182,42 @@ struct OperandLoader {
         }
     }
 
+    template <bool PRECISE>
+    static __device__ __forceinline__ void put(unsigned char* hi, unsigned char* lo, uint32_t off, float4 v) {
+        if (PRECISE) {
+            float4 h, l;
+            h.x = __uint_as_float(__float_as_uint(v.x) & 0xFFFFE000u); l.x = v.x - h.x;
+            h.y = __uint_as_float(__float_as_uint(v.y) & 0xFFFFE000u); l.y = v.y - h.y;
+            h.z = __uint_as_float(__float_as_uint(v.z) & 0xFFFFE000u); l.z = v.z - h.z;
+            h.w = __uint_as_float(__float_as_uint(v.w) & 0xFFFFE000u); l.w = v.w - h.w;
+            *reinterpret_cast<float4*>(hi + off) = h;
+            *reinterpret_cast<float4*>(lo + off) = l;
+        } else {
+            *reinterpret_cast<float4*>(hi + off) = v;
+        }
+    }
+
     // Split each value into its TF32 head and the remainder and write both tiles (only the raw
-    // value when precise == 0).  K-major canonical layout: (r,k) at (k/4)*ROWS*16 + r*16 + (k%4)*4.
-    __device__ __forceinline__ void store(unsigned char* hi, unsigned char* lo, const float4 (&r)[T], int precise) const {
+    // value when !PRECISE).
+    template <bool PRECISE>
+    __device__ __forceinline__ void store(unsigned char* hi, unsigned char* lo, const float4 (&r)[T]) const {
+        if (KC) {
 #pragma unroll
-        for (int t = 0; t < T; ++t) {
-            const uint32_t off = soff0 + (uint32_t)t * 256;       // 16 rows further
-            const float4 v = r[t];
-            if (KC) {
-                if (precise) {
-                    float4 h, l;
-                    h.x = __uint_as_float(__float_as_uint(v.x) & 0xFFFFE000u); l.x = v.x - h.x;
-                    h.y = __uint_as_float(__float_as_uint(v.y) & 0xFFFFE000u); l.y = v.y - h.y;
-                    h.z = __uint_as_float(__float_as_uint(v.z) & 0xFFFFE000u); l.z = v.z - h.z;
-                    h.w = __uint_as_float(__float_as_uint(v.w) & 0xFFFFE000u); l.w = v.w - h.w;
-                    *reinterpret_cast<float4*>(hi + off) = h;
-                    *reinterpret_cast<float4*>(lo + off) = l;
-                } else {
-                    *reinterpret_cast<float4*>(hi + off) = v;
-                }
-            } else {
-                // the four elements go to four rows; the order is rotated per lane so that the 32
-                // scalar stores of a warp fall into 32 different banks
+            for (int t = 0; t < T; ++t)
+                put<PRECISE>(hi, lo, (uint32_t)(lane & 15) * LBO + (uint32_t)krow(t) * 16, r[t]);
+        } else {
+            const int rot = (lane >> 1) & 3;
+            const int rl = (lane % LPR) * 4;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int e = (j + rot) & 3;
-                    const float x = pick(v, e);
-                    const uint32_t o = off + (uint32_t)e * 16;
-                    if (precise) {
-                        const float h = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
-                        *reinterpret_cast<float*>(hi + o) = h;
-                        *reinterpret_cast<float*>(lo + o) = x - h;
-                    } else {
-                        *reinterpret_cast<float*>(hi + o) = x;
+            for (int u = 0; u < ROUNDS; ++u) {
+                const int c = tcol(u);
+                if (c < kChunks) {
+                    const float4 k0 = r[4 * u], k1 = r[4 * u + 1], k2 = r[4 * u + 2], k3 = r[4 * u + 3];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int e = (j + rot) & 3;       // row rl + e gets (k0[e], k1[e], k2[e], k3[e])
+                        const float4 v = make_float4(pick(k0, e), pick(k1, e), pick(k2, e), pick(k3, e));
+                        put<PRECISE>(hi, lo, (uint32_t)c * LBO + (uint32_t)(rl + e) * 16, v);
                     }
                 }
             }
@@ -217,18 +226,19 @@ struct OperandLoader {
 };
 
 // NT = column tile / 16 (B operand rows per CTA = 16 * NT <= 128); A_K / B_K: operand contiguous
-// along k in memory; VEC: both operands allow 128-bit loads.
+// along k in memory; VEC: both operands allow 128-bit loads; PRECISE: three split MMAs per product.
 // Grid: (ceil(M/128), ceil(N/(16 NT)), nodes).
-template <int NT, bool A_K, bool B_K, bool VEC>
-__global__ void __launch_bounds__(kThreads, NT <= 4 ? 4 : 2)
+template <int NT, bool A_K, bool B_K, bool VEC, bool PRECISE>
+__global__ void __launch_bounds__(kThreads, (PRECISE || NT > 4) ? 2 : 3)
 tc_gemm_kernel(Args g) {
     constexpr int ROWS_A = kTileM, ROWS_B = 16 * NT;
-    constexpr uint32_t A_BYTES = ROWS_A * kBlockK * 4, B_BYTES = ROWS_B * kBlockK * 4;
-    constexpr int TA = ROWS_A / 16, TB = ROWS_B / 16;          // 16-byte chunks per loader thread
+    constexpr uint32_t A_BYTES = tile_bytes(ROWS_A), B_BYTES = tile_bytes(ROWS_B);
+    constexpr uint32_t A_LBO = tile_lbo(ROWS_A), B_LBO = tile_lbo(ROWS_B);
     constexpr uint32_t TMEM_COLS = ROWS_B <= 32 ? 32 : (ROWS_B <= 64 ? 64 : 128);
     extern __shared__ __align__(1024) unsigned char smem[];
-    // per stage: A hi | A lo | B hi | B lo
-    constexpr uint32_t STAGE = 2 * A_BYTES + 2 * B_BYTES;
+    // stage: A hi | A lo | B hi | B lo   (the lo tiles only when PRECISE)
+    constexpr uint32_t NCOPY = PRECISE ? 2 : 1;
+    constexpr uint32_t STAGE = NCOPY * (A_BYTES + B_BYTES);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * STAGE);
     uint64_t* empty = full + kStages;
     uint64_t* accum = empty + kStages;
@@ -256,14 +266,16 @@ tc_gemm_kernel(Args g) {
 
     if (warp < 4) {
         // ------------------------------ loaders ------------------------------
-        OperandLoader<ROWS_A, A_K, VEC> la;
-        OperandLoader<ROWS_B, B_K, VEC> lb;
+        using LoaderA = OperandLoader<ROWS_A, A_K, VEC>;
+        using LoaderB = OperandLoader<ROWS_B, B_K, VEC>;
+        LoaderA la;
+        LoaderB lb;
         la.init(g.A + (int64_t)node * g.a_node, g.a_pitch, warp, lane, m0, g.M, g.K);
         lb.init(g.B + (int64_t)node * g.b_node, g.b_pitch, warp, lane, n0, g.N, g.K);
         // One k-block per thread in flight: the proxy fence below also waits for the thread's
         // outstanding global loads, so deeper register prefetch would not overlap anything.  Memory
         // parallelism comes from the CTAs that share the SM.
-        float4 ra[TA], rb[TB];
+        float4 ra[LoaderA::T], rb[LoaderB::T];
         bool ok = true;
         la.fetch(0, ra); lb.fetch(0, rb);
         for (int kb = 0; kb < KB; ++kb) {
@@ -271,8 +283,8 @@ tc_gemm_kernel(Args g) {
             const uint32_t fill = (uint32_t)(kb / kStages);
             if (!mbar_wait(empty + s, (fill & 1u) ^ 1u)) { ok = false; break; }
             unsigned char* base = smem + s * STAGE;
-            la.store(base, base + A_BYTES, ra, g.precise);
-            lb.store(base + 2 * A_BYTES, base + 2 * A_BYTES + B_BYTES, rb, g.precise);
+            la.template store<PRECISE>(base, base + A_BYTES, ra);
+            lb.template store<PRECISE>(base + NCOPY * A_BYTES, base + NCOPY * A_BYTES + B_BYTES, rb);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             mbar_arrive(full + s);
             if (kb + 1 < KB) { la.fetch(kb + 1, ra); lb.fetch(kb + 1, rb); }
@@ -312,8 +324,6 @@ tc_gemm_kernel(Args g) {
         // instruction descriptor: fp32 accumulate, TF32 x TF32, both operands K-major, N, M
         const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(ROWS_B >> 3) << 17) |
                                ((uint32_t)(kTileM >> 4) << 24);
-        const uint32_t a_lbo = ROWS_A * 16, b_lbo = ROWS_B * 16;      // next 4 k: one 16-byte chunk column further
-        const uint32_t a_step = 2 * a_lbo, b_step = 2 * b_lbo;        // one MMA consumes k = 8 = two chunks
         bool ok = true;
         uint32_t acc = 0;
         for (int kb = 0; kb < KB; ++kb) {
@@ -322,12 +332,14 @@ tc_gemm_kernel(Args g) {
             if (!mbar_wait(full + s, fill & 1u)) { ok = false; break; }
             tc_fence_after();
             const uint32_t a_hi = smem_u32(smem + s * STAGE), a_lo = a_hi + A_BYTES;
-            const uint32_t b_hi = a_hi + 2 * A_BYTES, b_lo = b_hi + B_BYTES;
+            const uint32_t b_hi = a_hi + NCOPY * A_BYTES, b_lo = b_hi + B_BYTES;
 #pragma unroll
-            for (int kk = 0; kk < kBlockK / 8; ++kk) {
-                const uint64_t dah = smem_desc(a_hi + kk * a_step, a_lbo, 128), dbh = smem_desc(b_hi + kk * b_step, b_lbo, 128);
-                if (g.precise) {
-                    const uint64_t dal = smem_desc(a_lo + kk * a_step, a_lbo, 128), dbl = smem_desc(b_lo + kk * b_step, b_lbo, 128);
+            for (int kk = 0; kk < kBlockK / 8; ++kk) {       // one MMA consumes k = 8 = two chunk columns
+                const uint64_t dah = smem_desc(a_hi + kk * 2 * A_LBO, A_LBO, 128);
+                const uint64_t dbh = smem_desc(b_hi + kk * 2 * B_LBO, B_LBO, 128);
+                if (PRECISE) {
+                    const uint64_t dal = smem_desc(a_lo + kk * 2 * A_LBO, A_LBO, 128);
+                    const uint64_t dbl = smem_desc(b_lo + kk * 2 * B_LBO, B_LBO, 128);
                     mma_tf32(tmem_base, dal, dbh, idesc, acc); acc = 1;
                     mma_tf32(tmem_base, dah, dbl, idesc, acc);
                 }
@@ -345,9 +357,9 @@ tc_gemm_kernel(Args g) {
     }
 }
 
-template <int NT>
+template <int NT, bool PRECISE>
 constexpr size_t smem_bytes() {
-    return (size_t)kStages * (2 * kTileM * kBlockK * 4 + 2 * 16 * NT * kBlockK * 4) + (2 * kStages + 1) * 8 + 16;
+    return (size_t)kStages * (PRECISE ? 2 : 1) * (tile_bytes(kTileM) + tile_bytes(16 * NT)) + (2 * kStages + 1) * 8 + 16;
 }
 
 }  // namespace tc
