@@ -188,13 +188,13 @@ template <int NT, bool A_K, bool B_K, bool VEC, bool PRECISE>
 cudaError_t launch_tc_inst(dpsgd_ctx* c, const tc::Args& a, int n_tiles) {
     static bool attr_set = false;
     auto kernel = tc::tc_gemm_kernel<NT, A_K, B_K, VEC, PRECISE>;
-    constexpr size_t smem = tc::smem_bytes<NT, PRECISE>();
+    constexpr size_t smem = tc::smem_bytes<NT, A_K, B_K, PRECISE>();
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    dim3 grid((a.M + tc::kTileM - 1) / tc::kTileM, n_tiles, c->n);
+    dim3 grid((a.M + tc::kTileM - 1) / tc::kTileM, (n_tiles + a.n_per_cta - 1) / a.n_per_cta, c->n);
     kernel<<<grid, tc::kThreads, smem, c->stream>>>(a);
     c->launches++;
     return cudaGetLastError();
@@ -227,6 +227,7 @@ cudaError_t run_tc(dpsgd_ctx* c, tc::Args a, int max_tile) {
                      vec_ok(a.B, a.b_pitch, a.b_node, a.b_kcontig ? a.K : a.N);
     a.a_vec = a.b_vec = vec;
     a.precise = c->mlp_precision == 0;
+    a.n_per_cta = 8;            // matters for the weight-gradient product only (many column tiles)
     a.status = &c->d_result->status;
     const int want = a.N < max_tile ? a.N : max_tile;
     if (vec) {

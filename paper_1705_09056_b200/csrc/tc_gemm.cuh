@@ -11,12 +11,11 @@
 // or 128 bytes of each of four k-rows (operand contiguous along m / n): measured on B200, 64-byte
 // pieces reach 2.5 TB/s, full 128-byte lines 3.5 and 256-byte runs 5.1.  The values are split in
 // registers and written as hi / lo copies to shared memory directly in the no-swizzle K-major
-// layout the MMA descriptors describe: element (r,k) at (k/4)*LBO + (r/8)*128 + (r%8)*16 + (k%4)*4.
-// The descriptor arithmetic is linear in LBO, so LBO carries 16 bytes of padding per chunk column
-// and the 128-bit stores of lanes that run along k fall into different banks.  An operand that is
-// contiguous along m / n is transposed on the way: each lane scatters the four elements of its load
-// to four rows, in an order rotated per lane so that a warp's 32 scalar stores hit 32 banks.
-// (tcgen05 has no no-swizzle MN-major mode for 32-bit operands.)  One thread of a fifth warp
+// layout the MMA descriptors describe: element (r,k) at (k/4)*LBO + (r/8)*SBO + (r%8)*16 + (k%4)*4.
+// The descriptor arithmetic is linear in its two strides, so they carry 16 bytes of padding that
+// spreads the loaders' 128-bit stores over the banks.  An operand that is contiguous along m / n is
+// transposed on the way, 4x4 blocks at a time in registers.  (tcgen05 has no no-swizzle MN-major
+// mode for 32-bit operands.)  One thread of a fifth warp
 // issues the MMAs; tcgen05.commit releases a stage back to the loaders; the loader warps then
 // read the accumulator with tcgen05.ld and apply the epilogue with coalesced stores (m contiguous).
 // Every mbarrier wait is bounded; a wait that runs out raises the status word, and the CTA still
@@ -44,6 +43,7 @@ struct Args {
     float* C; int64_t c_node; int64_t c_pitch;                                   // C[n*c_pitch + m]
     const float* aux; int64_t aux_node; int64_t aux_pitch;                       // bias[m] or mask[n*aux_pitch + m]
     int M, N, K;
+    int n_per_cta;     // column tiles one CTA walks through (the A tile is kept when K fits one k-block)
     int epi;
     int precise;       // 1: three split MMAs per product, 0: one TF32 MMA
     int* status;
@@ -110,13 +110,16 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
     for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
 }
 
-__device__ __forceinline__ float pick(float4 v, int e) {
-    return e == 0 ? v.x : (e == 1 ? v.y : (e == 2 ? v.z : v.w));
+// Shared-memory layout of a ROWS-row operand tile: element (r,k) at
+//     (k/4)*LBO + (r/8)*SBO + (r%8)*16 + (k%4)*4.
+// The descriptor arithmetic is linear, so both strides can carry padding that spreads the loader's
+// 128-bit stores over the banks: a k-contiguous operand is stored by lanes that run along k (pad LBO
+// by 16 bytes), a transposed one by lanes that run along rows, four rows apart (pad SBO by 16 bytes).
+__host__ __device__ constexpr uint32_t tile_sbo(bool kc) { return kc ? 128u : 144u; }
+__host__ __device__ constexpr uint32_t tile_lbo(int rows, bool kc) {
+    return kc ? (uint32_t)rows * 16 + 16 : (uint32_t)(rows / 8) * 144;
 }
-
-// Byte distance between consecutive 16-byte chunk columns of a ROWS-row operand tile.
-__host__ __device__ constexpr uint32_t tile_lbo(int rows) { return (uint32_t)rows * 16 + 16; }
-__host__ __device__ constexpr uint32_t tile_bytes(int rows) { return kChunks * tile_lbo(rows); }
+__host__ __device__ constexpr uint32_t tile_bytes(int rows, bool kc) { return kChunks * tile_lbo(rows, kc); }
 
 // One loader thread's share of an operand tile (ROWS x 64 k) as 16-byte chunks, i.e. four
 // consecutive elements along the operand's contiguous direction.
@@ -126,8 +129,7 @@ __host__ __device__ constexpr uint32_t tile_bytes(int rows) { return kChunks * t
 //   !KC : it is contiguous along its row index (element (r,k) at k*pitch + r) and is transposed on
 //         the way to shared memory.  ROWS/4 lanes cover all rows of one k (512 bytes for 128 rows);
 //         a thread loads the same four rows at four consecutive k, transposes the 4x4 block in
-//         registers (free) and stores four chunks, one per row, in an order rotated per lane so
-//         that the 128-bit stores of a quarter warp fall into different banks.
+//         registers (free) and stores four chunks, one per row.
 //   VEC : 128-bit loads are legal (16-byte aligned rows, extent of the contiguous direction a
 //         multiple of 4); otherwise the four elements are loaded and bounds-checked one by one.
 // Loads are predicated, never branched around, so that all of a thread's loads are in flight together.
@@ -137,7 +139,7 @@ struct OperandLoader {
     static constexpr int G = 32 / LPR;                         // !KC: chunk columns per warp instruction
     static constexpr int ROUNDS = (kChunks + 4 * G - 1) / (4 * G);
     static constexpr int T = KC ? ROWS / 8 : 4 * ROUNDS;
-    static constexpr uint32_t LBO = tile_lbo(ROWS);
+    static constexpr uint32_t LBO = tile_lbo(ROWS, KC), SBO = tile_sbo(KC);
     const float* src;
     int64_t pitch;
     int row_base, rows, K, warp, lane;
@@ -206,19 +208,19 @@ struct OperandLoader {
             for (int t = 0; t < T; ++t)
                 put<PRECISE>(hi, lo, (uint32_t)(lane & 15) * LBO + (uint32_t)krow(t) * 16, r[t]);
         } else {
-            const int rot = (lane >> 1) & 3;
+            // rows rl .. rl+3 lie inside one 8-row group; lanes are 4 rows (64 + 8 pad bytes) apart
             const int rl = (lane % LPR) * 4;
+            const uint32_t roff = (uint32_t)(rl >> 3) * SBO + (uint32_t)(rl & 7) * 16;
 #pragma unroll
             for (int u = 0; u < ROUNDS; ++u) {
                 const int c = tcol(u);
                 if (c < kChunks) {
                     const float4 k0 = r[4 * u], k1 = r[4 * u + 1], k2 = r[4 * u + 2], k3 = r[4 * u + 3];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int e = (j + rot) & 3;       // row rl + e gets (k0[e], k1[e], k2[e], k3[e])
-                        const float4 v = make_float4(pick(k0, e), pick(k1, e), pick(k2, e), pick(k3, e));
-                        put<PRECISE>(hi, lo, (uint32_t)c * LBO + (uint32_t)(rl + e) * 16, v);
-                    }
+                    const uint32_t off = (uint32_t)c * LBO + roff;      // 4x4 transpose in registers
+                    put<PRECISE>(hi, lo, off, make_float4(k0.x, k1.x, k2.x, k3.x));
+                    put<PRECISE>(hi, lo, off + 16, make_float4(k0.y, k1.y, k2.y, k3.y));
+                    put<PRECISE>(hi, lo, off + 32, make_float4(k0.z, k1.z, k2.z, k3.z));
+                    put<PRECISE>(hi, lo, off + 48, make_float4(k0.w, k1.w, k2.w, k3.w));
                 }
             }
         }
@@ -227,30 +229,33 @@ struct OperandLoader {
 
 // NT = column tile / 16 (B operand rows per CTA = 16 * NT <= 128); A_K / B_K: operand contiguous
 // along k in memory; VEC: both operands allow 128-bit loads; PRECISE: three split MMAs per product.
-// Grid: (ceil(M/128), ceil(N/(16 NT)), nodes).
+// Grid: (ceil(M/128), ceil(N/(16 NT * n_per_cta)), nodes).
 template <int NT, bool A_K, bool B_K, bool VEC, bool PRECISE>
 __global__ void __launch_bounds__(kThreads, (PRECISE || NT > 4) ? 2 : 3)
 tc_gemm_kernel(Args g) {
     constexpr int ROWS_A = kTileM, ROWS_B = 16 * NT;
-    constexpr uint32_t A_BYTES = tile_bytes(ROWS_A), B_BYTES = tile_bytes(ROWS_B);
-    constexpr uint32_t A_LBO = tile_lbo(ROWS_A), B_LBO = tile_lbo(ROWS_B);
+    constexpr uint32_t A_BYTES = tile_bytes(ROWS_A, A_K), B_BYTES = tile_bytes(ROWS_B, B_K);
+    constexpr uint32_t A_LBO = tile_lbo(ROWS_A, A_K), B_LBO = tile_lbo(ROWS_B, B_K);
+    constexpr uint32_t A_SBO = tile_sbo(A_K), B_SBO = tile_sbo(B_K);
     constexpr uint32_t TMEM_COLS = ROWS_B <= 32 ? 32 : (ROWS_B <= 64 ? 64 : 128);
     extern __shared__ __align__(1024) unsigned char smem[];
     // stage: A hi | A lo | B hi | B lo   (the lo tiles only when PRECISE)
     constexpr uint32_t NCOPY = PRECISE ? 2 : 1;
     constexpr uint32_t STAGE = NCOPY * (A_BYTES + B_BYTES);
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * STAGE);
-    uint64_t* empty = full + kStages;
-    uint64_t* accum = empty + kStages;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGE);      // one stage per CTA
+    uint64_t* empty = full + 1;
+    uint64_t* accum = empty + 1;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int node = blockIdx.z;
-    const int m0 = blockIdx.x * kTileM, n0 = blockIdx.y * ROWS_B;
+    const int m0 = blockIdx.x * kTileM;
+    const int tile0 = blockIdx.y * g.n_per_cta;
+    const int n_tiles = min(g.n_per_cta, (g.N + ROWS_B - 1) / ROWS_B - tile0);
     const int KB = (g.K + kBlockK - 1) / kBlockK;
 
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(full + s, kLoaderThreads); mbar_init(empty + s, 1); }
+        mbar_init(full, kLoaderThreads); mbar_init(empty, 1);
         mbar_init(accum, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -271,84 +276,99 @@ tc_gemm_kernel(Args g) {
         LoaderA la;
         LoaderB lb;
         la.init(g.A + (int64_t)node * g.a_node, g.a_pitch, warp, lane, m0, g.M, g.K);
-        lb.init(g.B + (int64_t)node * g.b_node, g.b_pitch, warp, lane, n0, g.N, g.K);
         // One k-block per thread in flight: the proxy fence below also waits for the thread's
         // outstanding global loads, so deeper register prefetch would not overlap anything.  Memory
         // parallelism comes from the CTAs that share the SM.
         float4 ra[LoaderA::T], rb[LoaderB::T];
+        const int m = m0 + warp * 32 + lane;
+        float* C = g.C + (int64_t)node * g.c_node;
+        const float* aux = g.aux ? g.aux + (int64_t)node * g.aux_node : nullptr;
+        const float bias = (g.epi <= EPI_BIAS && m < g.M) ? __ldg(aux + m) : 0.f;
         bool ok = true;
+        uint32_t q = 0;                                     // k-blocks pushed so far (stage phase)
+        lb.init(g.B + (int64_t)node * g.b_node, g.b_pitch, warp, lane, tile0 * ROWS_B, g.N, g.K);
         la.fetch(0, ra); lb.fetch(0, rb);
-        for (int kb = 0; kb < KB; ++kb) {
-            const int s = kb % kStages;
-            const uint32_t fill = (uint32_t)(kb / kStages);
-            if (!mbar_wait(empty + s, (fill & 1u) ^ 1u)) { ok = false; break; }
-            unsigned char* base = smem + s * STAGE;
-            la.template store<PRECISE>(base, base + A_BYTES, ra);
-            lb.template store<PRECISE>(base + NCOPY * A_BYTES, base + NCOPY * A_BYTES + B_BYTES, rb);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            mbar_arrive(full + s);
-            if (kb + 1 < KB) { la.fetch(kb + 1, ra); lb.fetch(kb + 1, rb); }
-        }
-        // ------------------------------ epilogue ------------------------------
-        if (ok && !mbar_wait(accum, 0)) ok = false;
-        ok = __all_sync(0xffffffffu, ok);      // tcgen05.ld below needs the whole warp
-        if (!ok) {
-            if (lane == 0) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
-        } else {
+        for (int it = 0; it < n_tiles && ok; ++it) {
+            const int n0 = (tile0 + it) * ROWS_B;
+            const bool keep_a = (KB == 1 && it > 0);        // the A tile of the only k-block is already staged
+            for (int kb = 0; kb < KB; ++kb, ++q) {
+                if (!mbar_wait(empty, (q & 1u) ^ 1u)) { ok = false; break; }
+                if (!keep_a) la.template store<PRECISE>(smem, smem + A_BYTES, ra);
+                lb.template store<PRECISE>(smem + NCOPY * A_BYTES, smem + NCOPY * A_BYTES + B_BYTES, rb);
+                tc_fence_before();                          // orders this thread's earlier tcgen05.ld (previous tile)
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(full);
+                if (kb + 1 < KB) { la.fetch(kb + 1, ra); lb.fetch(kb + 1, rb); }
+                else if (it + 1 < n_tiles) {                // first k-block of the next column tile
+                    lb.row_base = n0 + ROWS_B;
+                    if (KB > 1) la.fetch(0, ra);
+                    lb.fetch(0, rb);
+                }
+            }
+            // ------------------------------ epilogue of this column tile ------------------------------
+            if (ok && !mbar_wait(accum, (uint32_t)it & 1u)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);               // tcgen05.ld below needs the whole warp
+            if (!ok) break;
             tc_fence_after();
-            const int m = m0 + warp * 32 + lane;
-            float* C = g.C + (int64_t)node * g.c_node;
-            const float* aux = g.aux ? g.aux + (int64_t)node * g.aux_node : nullptr;
-            const float bias = (g.epi <= EPI_BIAS && m < g.M) ? __ldg(aux + m) : 0.f;
 #pragma unroll 1
             for (int c0 = 0; c0 < ROWS_B; c0 += 16) {
                 float v[16];
                 tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
-                if (m < g.M) {
+                const int nb = n0 + c0;
+                const int cnt = m < g.M ? min(16, g.N - nb) : 0;      // columns of this group inside the matrix
+                float* out = C + (int64_t)nb * g.c_pitch + m;
+                if (g.epi == EPI_STORE) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) if (j < cnt) out[(int64_t)j * g.c_pitch] = v[j];
+                } else if (g.epi == EPI_MASK) {
+                    const float* mk = aux + (int64_t)nb * g.aux_pitch + m;
+                    float gate[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) gate[j] = j < cnt ? __ldg(mk + (int64_t)j * g.aux_pitch) : 0.f;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) if (j < cnt) out[(int64_t)j * g.c_pitch] = gate[j] > 0.f ? v[j] : 0.f;
+                } else {
+                    const bool relu = g.epi == EPI_BIAS_RELU;
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        const int n = n0 + c0 + j;
-                        if (n < g.N) {
-                            float x = v[j];
-                            if (g.epi == EPI_BIAS_RELU) { x += bias; x = x > 0.f ? x : 0.f; }
-                            else if (g.epi == EPI_BIAS) x += bias;
-                            else if (g.epi == EPI_MASK) x = __ldg(aux + (int64_t)n * g.aux_pitch + m) > 0.f ? x : 0.f;
-                            C[(int64_t)n * g.c_pitch + m] = x;
-                        }
+                        const float x = v[j] + bias;
+                        if (j < cnt) out[(int64_t)j * g.c_pitch] = (relu && x < 0.f) ? 0.f : x;
                     }
                 }
             }
         }
+        if (!ok && lane == 0) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
     } else if (lane == 0) {
         // ------------------------------ MMA issuer ------------------------------
         // instruction descriptor: fp32 accumulate, TF32 x TF32, both operands K-major, N, M
         const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(ROWS_B >> 3) << 17) |
                                ((uint32_t)(kTileM >> 4) << 24);
         bool ok = true;
-        uint32_t acc = 0;
-        for (int kb = 0; kb < KB; ++kb) {
-            const int s = kb % kStages;
-            const uint32_t fill = (uint32_t)(kb / kStages);
-            if (!mbar_wait(full + s, fill & 1u)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t a_hi = smem_u32(smem + s * STAGE), a_lo = a_hi + A_BYTES;
-            const uint32_t b_hi = a_hi + NCOPY * A_BYTES, b_lo = b_hi + B_BYTES;
+        uint32_t q = 0;
+        for (int it = 0; it < n_tiles && ok; ++it) {
+            uint32_t acc = 0;                               // the first MMA of a column tile overwrites the accumulator
+            for (int kb = 0; kb < KB; ++kb, ++q) {
+                if (!mbar_wait(full, q & 1u)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t a_hi = smem_u32(smem), a_lo = a_hi + A_BYTES;
+                const uint32_t b_hi = a_hi + NCOPY * A_BYTES, b_lo = b_hi + B_BYTES;
 #pragma unroll
-            for (int kk = 0; kk < kBlockK / 8; ++kk) {       // one MMA consumes k = 8 = two chunk columns
-                const uint64_t dah = smem_desc(a_hi + kk * 2 * A_LBO, A_LBO, 128);
-                const uint64_t dbh = smem_desc(b_hi + kk * 2 * B_LBO, B_LBO, 128);
-                if (PRECISE) {
-                    const uint64_t dal = smem_desc(a_lo + kk * 2 * A_LBO, A_LBO, 128);
-                    const uint64_t dbl = smem_desc(b_lo + kk * 2 * B_LBO, B_LBO, 128);
-                    mma_tf32(tmem_base, dal, dbh, idesc, acc); acc = 1;
-                    mma_tf32(tmem_base, dah, dbl, idesc, acc);
+                for (int kk = 0; kk < kBlockK / 8; ++kk) {       // one MMA consumes k = 8 = two chunk columns
+                    const uint64_t dah = smem_desc(a_hi + kk * 2 * A_LBO, A_LBO, A_SBO);
+                    const uint64_t dbh = smem_desc(b_hi + kk * 2 * B_LBO, B_LBO, B_SBO);
+                    if (PRECISE) {
+                        const uint64_t dal = smem_desc(a_lo + kk * 2 * A_LBO, A_LBO, A_SBO);
+                        const uint64_t dbl = smem_desc(b_lo + kk * 2 * B_LBO, B_LBO, B_SBO);
+                        mma_tf32(tmem_base, dal, dbh, idesc, acc); acc = 1;
+                        mma_tf32(tmem_base, dah, dbl, idesc, acc);
+                    }
+                    mma_tf32(tmem_base, dah, dbh, idesc, acc); acc = 1;
                 }
-                mma_tf32(tmem_base, dah, dbh, idesc, acc); acc = 1;
+                mma_commit(empty);      // frees the stage once these MMAs have read it
             }
-            mma_commit(empty + s);      // frees the stage once these MMAs have read it
+            if (ok) mma_commit(accum);  // accumulator of this column tile complete
         }
-        if (ok) mma_commit(accum);      // accumulator complete
-        else atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
+        if (!ok) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
     }
     tc_fence_before();
     __syncthreads();
@@ -357,9 +377,9 @@ tc_gemm_kernel(Args g) {
     }
 }
 
-template <int NT, bool PRECISE>
+template <int NT, bool A_K, bool B_K, bool PRECISE>
 constexpr size_t smem_bytes() {
-    return (size_t)kStages * (PRECISE ? 2 : 1) * (tile_bytes(kTileM) + tile_bytes(16 * NT)) + (2 * kStages + 1) * 8 + 16;
+    return (size_t)(PRECISE ? 2 : 1) * (tile_bytes(kTileM, A_K) + tile_bytes(16 * NT, B_K)) + 3 * 8 + 16;
 }
 
 }  // namespace tc
