@@ -59,7 +59,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "25"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -128,6 +128,22 @@ def workload_config(topology):
             "n": N_NODES, "N": N_PARAMS, "topology": topology, "gamma": GAMMA,
             "l2": "no flush needed: 19.2 GB touched per step >> 126 MB L2",
             "parallelism": "replicas only (one GPU per independent replica)"}
+
+
+def max_over_ranks(seconds_or_ms: float, device) -> float:
+    """Slowest rank's time.  A timing reduction only: the replicas exchange no data."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(seconds_or_ms)
+    t = torch.tensor([seconds_or_ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(replicas_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job replica-steps/s of `world` independent replicas timed by the slowest rank."""
+    return world * replicas_per_rank / (ms_per_step * 1e-3)
 
 
 def time_steps(ctx, steps, warmup, torch):
@@ -206,10 +222,7 @@ def run_ours(args):
             launches = ctx.launch_count() - l0
             if rank == 0:
                 clocks = sampler.stop(t0, t1)
-            if world > 1:
-                t = torch.tensor([ms], device=dev, dtype=torch.float64)
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                ms = float(t.item())
+            ms = max_over_ranks(ms, dev)
         gbs = bytes_per_launch / (ms * 1e-3) / 1e9
         results[topo] = {"kernel": kind, "ms_per_step": ms, "replica_steps_per_s": n / (ms * 1e-3),
                          "GBps": gbs, "frac_of_measured_peak": gbs / peak,
@@ -232,10 +245,7 @@ def run_ours(args):
                 ring_ctx.mix_update_host(Gh)
             torch.cuda.synchronize()
             dt = (time.perf_counter() - t0) / k_e2e
-            if world > 1:
-                t = torch.tensor([dt], device=dev, dtype=torch.float64)
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                dt = float(t.item())
+            dt = max_over_ranks(dt, dev)
             e2e = {"value": world * n / dt, "unit": "replica-steps/s", "h2d_bytes_per_step": 4 * n * N,
                    "d2h_bytes_per_step": 8, "steps": k_e2e, "ms_per_step": dt * 1e3,
                    "call": "dpsgd_mix_update_host (pinned host G -> device, mix+update, consensus distance -> host)"}
@@ -268,7 +278,7 @@ def run_ours(args):
 
     ring = results["ring"]
     line = {
-        "metric": METRIC, "value": world * ring["replica_steps_per_s"], "unit": "replica-steps/s",
+        "metric": METRIC, "value": aggregate_throughput(n, world, ring["ms_per_step"]), "unit": "replica-steps/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ring["ms_per_step"],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic", "config": workload_config("ring"),
