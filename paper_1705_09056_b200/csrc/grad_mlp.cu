@@ -227,9 +227,15 @@ cudaError_t run_tc(dpsgd_ctx* c, tc::Args a, int max_tile) {
                      vec_ok(a.B, a.b_pitch, a.b_node, a.b_kcontig ? a.K : a.N);
     a.a_vec = a.b_vec = vec;
     a.precise = c->mlp_precision == 0;
-    a.n_per_cta = 8;            // matters for the weight-gradient product only (many column tiles)
     a.status = &c->d_result->status;
     const int want = a.N < max_tile ? a.N : max_tile;
+    {   // column tiles per CTA: up to 8 (keeps the A tile staged), but never so many that the grid
+        // falls under about four CTAs per CTA slot of the device
+        const int tile = want <= 16 ? 16 : (want <= 32 ? 32 : (want <= 64 ? 64 : 128));
+        const long long tiles = (long long)((a.M + tc::kTileM - 1) / tc::kTileM) * ((a.N + tile - 1) / tile) * c->n;
+        const long long per = tiles / (4LL * 2 * 148);
+        a.n_per_cta = (int)(per < 1 ? 1 : (per > 8 ? 8 : per));
+    }
     if (vec) {
         if (want <= 16) return launch_tc_nt<1, true>(c, a, (a.N + 15) / 16);
         if (want <= 32) return launch_tc_nt<2, true>(c, a, (a.N + 31) / 32);
