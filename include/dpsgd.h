@@ -133,6 +133,25 @@ DPSGD_API dpsgd_status dpsgd_grad(dpsgd_ctx* ctx, uint64_t k);
  */
 DPSGD_API dpsgd_status dpsgd_mix_update(dpsgd_ctx* ctx);
 
+/*
+ * Footnote c of Algorithm 1: with update_then_mix != 0 every later gossip step first applies the
+ * local gradient and then averages, X_next <- W (X_cur - gamma G); 0 restores the printed order.
+ * With W = 1 1^T / n the swapped order is exactly centralized minibatch SGD on every row.
+ */
+DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* ctx, int32_t update_then_mix);
+
+/*
+ * dpsgd_mix_update() that also writes sum_i ||xbar - x_i||^2 of the NEW X (Theorem 4, Eq. 10) to
+ * one double in device memory, asynchronously on the stream.  For ring and uniform-dense W the
+ * sum is accumulated inside the gossip kernel (no second pass over HBM); otherwise a consensus
+ * pass over the new X follows.  consensus_out_dev: device, 8-byte aligned, caller-owned.
+ */
+DPSGD_API dpsgd_status dpsgd_mix_update_consensus(dpsgd_ctx* ctx, double* consensus_out_dev);
+
+/* dpsgd_grad(k) followed by dpsgd_mix_update_consensus(): an iteration that logs its consensus
+ * distance (as the 112-node experiments of Section 5 would, per step). */
+DPSGD_API dpsgd_status dpsgd_step_consensus(dpsgd_ctx* ctx, uint64_t k, double* consensus_out_dev);
+
 /* One full iteration k of Algorithm 1: dpsgd_grad(k) followed by dpsgd_mix_update(). */
 DPSGD_API dpsgd_status dpsgd_step(dpsgd_ctx* ctx, uint64_t k);
 

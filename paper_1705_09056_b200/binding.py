@@ -37,6 +37,9 @@ SIGNATURES = {
     "dpsgd_grad": [_vp, _u64],
     "dpsgd_mix_update": [_vp],
     "dpsgd_step": [_vp, _u64],
+    "dpsgd_set_order": [_vp, _i32],
+    "dpsgd_mix_update_consensus": [_vp, _vp],
+    "dpsgd_step_consensus": [_vp, _u64, _vp],
     "dpsgd_consensus_dist": [_vp, ctypes.POINTER(ctypes.c_double)],
     "dpsgd_average": [_vp, _vp],
     "dpsgd_mix_update_host": [_vp, _vp, _i64, ctypes.POINTER(ctypes.c_double)],
@@ -184,6 +187,19 @@ class Dpsgd:
 
     def step(self, k: int):
         self._check(self._lib.dpsgd_step(self._h, k))
+
+    def set_order(self, update_then_mix: bool):
+        """Footnote c of Algorithm 1: apply the local gradient first, then average."""
+        self._check(self._lib.dpsgd_set_order(self._h, 1 if update_then_mix else 0))
+
+    def mix_update_consensus(self, out: torch.Tensor):
+        """Gossip step that also writes the new consensus distance into `out` (one float64 on the device)."""
+        assert out.is_cuda and out.dtype == torch.float64 and out.numel() >= 1
+        self._check(self._lib.dpsgd_mix_update_consensus(self._h, _ptr(out)))
+
+    def step_consensus(self, k: int, out: torch.Tensor):
+        assert out.is_cuda and out.dtype == torch.float64 and out.numel() >= 1
+        self._check(self._lib.dpsgd_step_consensus(self._h, k, _ptr(out)))
 
     def consensus_dist(self) -> float:
         out = ctypes.c_double()

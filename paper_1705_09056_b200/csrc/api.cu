@@ -143,6 +143,7 @@ dpsgd_status need_model(dpsgd_ctx* c) {
 cudaError_t run_mix(dpsgd_ctx* c) {
     const float* X = c->X[c->cur];
     float* Xn = c->X[c->cur ^ 1];
+    if (c->swapped && c->mix_kind != DPSGD_MIX_TILED_CSR) return launch_mix_variant(c, X, c->G, Xn, true, nullptr);
     switch (c->mix_kind) {
         case DPSGD_MIX_RING: return launch_mix_ring(c, X, c->G, Xn);
         case DPSGD_MIX_UNIFORM_DENSE: return launch_mix_uniform(c, X, c->G, Xn);
@@ -333,6 +334,45 @@ DPSGD_API dpsgd_status dpsgd_mix_update(dpsgd_ctx* c) {
     if (e != cudaSuccess) return cuda_fail(c, e, "mix_update kernel");
     c->cur ^= 1;
     return DPSGD_OK;
+}
+
+// Gossip step that also leaves the consensus distance of the new X in *out_dev.
+dpsgd_status mix_with_consensus(dpsgd_ctx* c, double* out_dev) {
+    const float* X = c->X[c->cur];
+    float* Xn = c->X[c->cur ^ 1];
+    cudaError_t e = launch_mix_variant(c, X, c->G, Xn, c->swapped, out_dev);
+    if (e == cudaErrorNotSupported) {       // no fused kernel for this W: mix, then one pass over the new X
+        e = run_mix(c);
+        if (e == cudaSuccess) e = launch_consensus(c, Xn, out_dev);
+    }
+    if (e != cudaSuccess) return cuda_fail(c, e, "mix_update with consensus");
+    c->cur ^= 1;
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* c, int32_t update_then_mix) {
+    if (!c) return DPSGD_ERR_ARG;
+    c->swapped = update_then_mix != 0;
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_mix_update_consensus(dpsgd_ctx* c, double* out_dev) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    if (!out_dev) return fail(c, DPSGD_ERR_ARG, "consensus_out_dev is NULL");
+    if (!aligned(out_dev, 8)) return fail(c, DPSGD_ERR_ALIGN, "consensus_out_dev must be 8-byte aligned");
+    return mix_with_consensus(c, out_dev);
+}
+
+DPSGD_API dpsgd_status dpsgd_step_consensus(dpsgd_ctx* c, uint64_t k, double* out_dev) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    if ((s = need_model(c)) != DPSGD_OK) return s;
+    if (!out_dev) return fail(c, DPSGD_ERR_ARG, "consensus_out_dev is NULL");
+    if (!aligned(out_dev, 8)) return fail(c, DPSGD_ERR_ALIGN, "consensus_out_dev must be 8-byte aligned");
+    cudaError_t e = run_grad(c, k);
+    if (e != cudaSuccess) return cuda_fail(c, e, "gradient kernels");
+    return mix_with_consensus(c, out_dev);
 }
 
 DPSGD_API dpsgd_status dpsgd_step(dpsgd_ctx* c, uint64_t k) {

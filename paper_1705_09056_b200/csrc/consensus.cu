@@ -99,17 +99,32 @@ average_kernel(const float4* __restrict__ X, int n, int64_t ld4, float4* __restr
 
 }  // namespace
 
+// Grows the per-CTA partial-sum buffer of the context to at least `count` doubles.
+cudaError_t ensure_partials(dpsgd_ctx* c, int count) {
+    if (count <= c->partials_cap) return cudaSuccess;
+    cudaError_t e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) return e;
+    cudaFree(c->d_partials);
+    c->d_partials = nullptr; c->partials_cap = 0;
+    e = cudaMalloc(&c->d_partials, sizeof(double) * (size_t)count);
+    if (e != cudaSuccess) return e;
+    c->partials_cap = count;
+    return cudaSuccess;
+}
+
+// Adds the first `count` partials of the context in a fixed order into *result_dev.
+cudaError_t launch_consensus_final(dpsgd_ctx* c, int count, double* result_dev) {
+    consensus_final_kernel<<<1, kThreads, 0, c->stream>>>(c->d_partials, count, result_dev);
+    c->launches++;
+    return cudaGetLastError();
+}
+
 cudaError_t launch_consensus(dpsgd_ctx* c, const float* X, double* result_dev) {
     const int64_t ld4 = c->ld / 4;
     const int grid = (int)((ld4 + kThreads - 1) / kThreads);
-    if (grid > c->partials_cap) {
-        cudaError_t e = cudaStreamSynchronize(c->stream);
+    {
+        cudaError_t e = ensure_partials(c, grid);
         if (e != cudaSuccess) return e;
-        cudaFree(c->d_partials);
-        c->d_partials = nullptr; c->partials_cap = 0;
-        e = cudaMalloc(&c->d_partials, sizeof(double) * (size_t)grid);
-        if (e != cudaSuccess) return e;
-        c->partials_cap = grid;
     }
     consensus_partial_kernel<8><<<grid, kThreads, 0, c->stream>>>(
         reinterpret_cast<const float4*>(X), c->n, ld4, c->d_partials);

@@ -54,6 +54,7 @@ struct dpsgd_ctx {
     dpsgd::MixW W;
     void* d_w_blob = nullptr;  // one allocation holding row_ptr | col | val | band
     int mix_kind = DPSGD_MIX_GATHER_CSR;
+    bool swapped = false;      // footnote c of Algorithm 1: update locally, then average
     bool can_ring = false, can_uniform = false, can_tiled = false;
 
     // bound buffers
@@ -103,6 +104,10 @@ bool mix_tiled_supported(const dpsgd_ctx* c);
 void mix_tiled_release(dpsgd_ctx* c);
 
 cudaError_t launch_consensus(dpsgd_ctx* c, const float* X, double* result_dev);
+cudaError_t ensure_partials(dpsgd_ctx* c, int count);
+cudaError_t launch_consensus_final(dpsgd_ctx* c, int count, double* result_dev);
+cudaError_t launch_mix_variant(dpsgd_ctx* c, const float* X, const float* G, float* Xn, bool swapped,
+                               double* stats_out);
 cudaError_t launch_average(dpsgd_ctx* c, const float* X, float* xbar);
 
 cudaError_t launch_sample(dpsgd_ctx* c, uint64_t k, int32_t* idx);

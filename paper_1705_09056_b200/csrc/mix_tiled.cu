@@ -45,6 +45,7 @@ struct TiledState {
     int grid = 0;
     int csr_in_smem = 0;
     int x_tma = 1;
+    int swapped = 0;
     int* d_status = nullptr;
     PackedNz* d_nz = nullptr;
 };
@@ -98,7 +99,9 @@ __device__ __forceinline__ void cp_async_arrive(uint64_t* bar) {
 // row_ptr and of the packed nonzeros so that the gather loop never leaves the SM.
 // X arrives by TMA (one box per tile) or, with X_TMA = false, by per-thread 16-byte async copies
 // like G always does; each stage's mbarrier counts the TMA transaction plus one arrival per thread.
-template <int T, int S, bool X_TMA>
+// SWAPPED (footnote c of Algorithm 1): the staged X tile is first turned into X - gamma G in place,
+// then gathered: X_next[i] = sum_j W_ij (X[j] - gamma G[j]).
+template <int T, int S, bool X_TMA, bool SWAPPED>
 __global__ void __launch_bounds__(kThreads)
 mix_tiled_kernel(const __grid_constant__ CUtensorMap mapX, const float4* __restrict__ X,
                  const float4* __restrict__ G, float4* __restrict__ Xn, const int32_t* row_ptr,
@@ -166,9 +169,20 @@ mix_tiled_kernel(const __grid_constant__ CUtensorMap mapX, const float4* __restr
             }
             return;
         }
-        const unsigned char* xs = smem_raw + (size_t)s * stage_bytes + cg * 16;   // this thread's column group
+        unsigned char* xs = smem_raw + (size_t)s * stage_bytes + cg * 16;   // this thread's column group
         const unsigned char* gs = xs + tile_bytes;
         const int64_t c4 = (first + it * step) * kGroups + cg;
+        if (SWAPPED) {
+            for (int i = r0; i < n; i += kRowStep) {
+                float4* xp = reinterpret_cast<float4*>(xs + (uint32_t)i * (T * 4u));
+                const float4 g = *reinterpret_cast<const float4*>(gs + (uint32_t)i * (T * 4u));
+                float4 v = *xp;
+                v.x = fmaf(ngamma, g.x, v.x); v.y = fmaf(ngamma, g.y, v.y);
+                v.z = fmaf(ngamma, g.z, v.z); v.w = fmaf(ngamma, g.w, v.w);
+                *xp = v;
+            }
+            __syncthreads();
+        }
         if (c4 < ld4) {
             float4* out = Xn + c4;
             for (int i = r0; i < n; i += kRowStep) {
@@ -180,9 +194,11 @@ mix_tiled_kernel(const __grid_constant__ CUtensorMap mapX, const float4* __restr
                     a.x = fmaf(e.w, v.x, a.x); a.y = fmaf(e.w, v.y, a.y);
                     a.z = fmaf(e.w, v.z, a.z); a.w = fmaf(e.w, v.w, a.w);
                 }
-                const float4 g = *reinterpret_cast<const float4*>(gs + (uint32_t)i * (T * 4u));
-                a.x = fmaf(ngamma, g.x, a.x); a.y = fmaf(ngamma, g.y, a.y);
-                a.z = fmaf(ngamma, g.z, a.z); a.w = fmaf(ngamma, g.w, a.w);
+                if (!SWAPPED) {
+                    const float4 g = *reinterpret_cast<const float4*>(gs + (uint32_t)i * (T * 4u));
+                    a.x = fmaf(ngamma, g.x, a.x); a.y = fmaf(ngamma, g.y, a.y);
+                    a.z = fmaf(ngamma, g.z, a.z); a.w = fmaf(ngamma, g.w, a.w);
+                }
                 __stcs(out + (int64_t)i * ld4, a);
             }
         }
@@ -244,11 +260,11 @@ bool pick_shape(int n, int nnz, int* T_out, int* S_out, int* ctas_out) {
     return false;
 }
 
-template <int T, int S, bool X_TMA>
+template <int T, int S, bool X_TMA, bool SWAPPED>
 cudaError_t launch_tsx(dpsgd_ctx* c, TiledState* st, int which, const float* G, float* Xn) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(mix_tiled_kernel<T, S, X_TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(mix_tiled_kernel<T, S, X_TMA, SWAPPED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)(kSmemPerSm - kSmemPerCtaReserve));
         if (e != cudaSuccess) return e;
         attr_set = true;
@@ -256,7 +272,7 @@ cudaError_t launch_tsx(dpsgd_ctx* c, TiledState* st, int which, const float* G, 
     const int64_t ld4 = c->ld / 4;
     const int64_t tiles = (c->ld + T - 1) / T;
     const int grid = (int)std::min<int64_t>(tiles, st->grid);
-    mix_tiled_kernel<T, S, X_TMA><<<grid, kThreads, st->smem, c->stream>>>(
+    mix_tiled_kernel<T, S, X_TMA, SWAPPED><<<grid, kThreads, st->smem, c->stream>>>(
         st->mapX[which], reinterpret_cast<const float4*>(c->X[which]), reinterpret_cast<const float4*>(G),
         reinterpret_cast<float4*>(Xn), c->W.row_ptr, st->d_nz, c->n, ld4, tiles, -c->gamma, st->csr_in_smem,
         st->d_status);
@@ -265,7 +281,9 @@ cudaError_t launch_tsx(dpsgd_ctx* c, TiledState* st, int which, const float* G, 
 
 template <int T, int S>
 cudaError_t launch_ts(dpsgd_ctx* c, TiledState* st, int which, const float* G, float* Xn) {
-    return st->x_tma ? launch_tsx<T, S, true>(c, st, which, G, Xn) : launch_tsx<T, S, false>(c, st, which, G, Xn);
+    if (st->swapped)
+        return st->x_tma ? launch_tsx<T, S, true, true>(c, st, which, G, Xn) : launch_tsx<T, S, false, true>(c, st, which, G, Xn);
+    return st->x_tma ? launch_tsx<T, S, true, false>(c, st, which, G, Xn) : launch_tsx<T, S, false, false>(c, st, which, G, Xn);
 }
 
 template <int T>
@@ -326,6 +344,7 @@ cudaError_t launch_mix_tiled(dpsgd_ctx* c, const float* X, const float* G, float
         c->tma_state = st;
     }
     const int which = (X == c->X[0]) ? 0 : 1;
+    st->swapped = c->swapped ? 1 : 0;
     cudaError_t e;
     switch (st->T) {
         case 128: e = launch_t<128>(c, st, which, G, Xn); break;

@@ -22,6 +22,8 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=1)
     ap.add_argument("--consensus", action="store_true", help="also run the consensus reduction")
+    ap.add_argument("--fused", action="store_true", help="time the gossip step that also returns the consensus distance")
+    ap.add_argument("--swapped", action="store_true", help="footnote c: update locally, then average")
     args = ap.parse_args()
 
     build.build()
@@ -34,13 +36,17 @@ def main():
     ctx.bind(X0, X1, G)
     if args.kind >= 0:
         ctx.mix_kind(args.kind)
+    if args.swapped:
+        ctx.set_order(True)
+    out = torch.zeros(1, dtype=torch.float64, device=dev)
+    step = (lambda: ctx.mix_update_consensus(out)) if args.fused else ctx.mix_update
     for _ in range(args.warmup):
-        ctx.mix_update()
+        step()
     torch.cuda.synchronize()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record()
     for _ in range(args.steps):
-        ctx.mix_update()
+        step()
     b.record()
     torch.cuda.synchronize()
     ms = a.elapsed_time(b) / max(1, args.steps)

@@ -24,6 +24,9 @@ def main():
     ap.add_argument("--topology", default="")
     ap.add_argument("--precision", type=int, default=0, help="MLP: 0 fp32-faithful, 1 single TF32 pass")
     ap.add_argument("--consensus", action="store_true", help="evaluate the consensus distance every step")
+    ap.add_argument("--fused-consensus", action="store_true",
+                    help="log the consensus distance every step from inside the gossip kernel")
+    ap.add_argument("--swapped", action="store_true", help="footnote c: update locally, then average")
     args = ap.parse_args()
 
     build.build()
@@ -56,7 +59,13 @@ def main():
     for k in range(args.warmup):
         ctx.step(k)
     l0 = ctx.launch_count()
-    if args.consensus:
+    if args.swapped:
+        ctx.set_order(True)
+    log = torch.zeros(args.steps + args.warmup + 8, dtype=torch.float64, device=dev)
+    if args.fused_consensus:
+        def whole(k):
+            ctx.step_consensus(args.warmup + k, log[k:k + 1])
+    elif args.consensus:
         def whole(k):
             ctx.step(args.warmup + k)
             ctx.consensus_dist()
