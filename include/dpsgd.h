@@ -141,6 +141,16 @@ DPSGD_API dpsgd_status dpsgd_mix_update(dpsgd_ctx* ctx);
 DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* ctx, int32_t update_then_mix);
 
 /*
+ * Momentum as used for both algorithms in the Torch experiments (Section 5.3: learning rate 0.1,
+ * momentum 0.9).  The paper prints no formula; the reading is the heavy-ball update of the
+ * framework it used, kept per node: v_i <- beta v_i + g_i, then the gossip step with v_i in place
+ * of g_i.  V_dev: device, fp32 [n][ld], 128-byte aligned, caller-owned, zero before the first
+ * step, distinct from X0/X1/G; 0 <= beta < 1.  V_dev = NULL switches momentum off.  Call after
+ * dpsgd_bind (rebinding switches it off).
+ */
+DPSGD_API dpsgd_status dpsgd_set_momentum(dpsgd_ctx* ctx, float beta, float* V_dev);
+
+/*
  * dpsgd_mix_update() that also writes sum_i ||xbar - x_i||^2 of the NEW X (Theorem 4, Eq. 10) to
  * one double in device memory, asynchronously on the stream.  For ring and uniform-dense W the
  * sum is accumulated inside the gossip kernel (no second pass over HBM); otherwise a consensus

@@ -18,6 +18,7 @@ Pins (see tests/test_oracle_*.py):
   mix_update ............ brute-force dense W @ X, mean preservation, sqrt(rho) contraction,
                           W = I, gamma = 0, closed-form ring spectrum
   consensus_dist ........ ||X||_F^2 - n ||xbar||^2 identity, zero at identical rows
+  momentum .............. beta = 0 reduces to mix_update; constant-gradient closed form
   step / run ............ least-squares gradient descent closed form; dense-W reduction to
                           centralized minibatch SGD
   MLP trajectories ...... parity unpinned beyond the per-step pins above (non-convex, no
@@ -242,6 +243,22 @@ def mix_update_swapped(X, G, row_ptr, col, val, gamma):
             acc += np.float64(val[p]) * (X[j].astype(np.float64) - g64 * G[j].astype(np.float64))
         out[i] = acc.astype(np.float32)
     return out
+
+
+def momentum_buffer(V, G, beta):
+    """Heavy-ball momentum of the Torch runs of Section 5.3 (learning rate 0.1, momentum 0.9), kept
+    per node: v_{k+1,i} = beta v_{k,i} + g_i.  fp64 arithmetic, one rounding to fp32."""
+    b64 = np.float64(np.float32(beta))
+    return (b64 * V.astype(np.float64) + G.astype(np.float64)).astype(np.float32)
+
+
+def mix_update_momentum(X, V, G, row_ptr, col, val, gamma, beta, swapped=False):
+    """D-PSGD iteration with the momentum buffer in place of the raw gradient:
+    V' = beta V + G, then X' = W X - gamma V' (or W (X - gamma V') in footnote c's order).
+    Returns (X', V')."""
+    Vn = momentum_buffer(V, G, beta)
+    f = mix_update_swapped if swapped else mix_update
+    return f(X, Vn, row_ptr, col, val, gamma), Vn
 
 
 def node_average(X):

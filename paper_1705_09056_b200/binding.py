@@ -38,6 +38,7 @@ SIGNATURES = {
     "dpsgd_mix_update": [_vp],
     "dpsgd_step": [_vp, _u64],
     "dpsgd_set_order": [_vp, _i32],
+    "dpsgd_set_momentum": [_vp, _f32, _vp],
     "dpsgd_mix_update_consensus": [_vp, _vp],
     "dpsgd_step_consensus": [_vp, _u64, _vp],
     "dpsgd_consensus_dist": [_vp, ctypes.POINTER(ctypes.c_double)],
@@ -191,6 +192,13 @@ class Dpsgd:
     def set_order(self, update_then_mix: bool):
         """Footnote c of Algorithm 1: apply the local gradient first, then average."""
         self._check(self._lib.dpsgd_set_order(self._h, 1 if update_then_mix else 0))
+
+    def set_momentum(self, beta: float, V: Optional[torch.Tensor]):
+        """Heavy-ball momentum (Section 5.3): V is an n x ld fp32 CUDA tensor, zero at the start; None = off."""
+        if V is not None:
+            assert V.is_cuda and V.dtype == torch.float32 and V.is_contiguous() and V.shape == self._keep[0].shape
+        self._check(self._lib.dpsgd_set_momentum(self._h, beta, _ptr(V)))
+        self._momentum_keep = V
 
     def mix_update_consensus(self, out: torch.Tensor):
         """Gossip step that also writes the new consensus distance into `out` (one float64 on the device)."""

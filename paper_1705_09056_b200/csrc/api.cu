@@ -140,15 +140,26 @@ dpsgd_status need_model(dpsgd_ctx* c) {
     return DPSGD_OK;
 }
 
+// The buffer the gossip step subtracts: the gradients, or the momentum buffers after their update.
+cudaError_t step_direction(dpsgd_ctx* c, const float** dir) {
+    *dir = c->G;
+    if (!c->V) return cudaSuccess;
+    *dir = c->V;
+    return launch_momentum(c, c->V, c->G);
+}
+
 cudaError_t run_mix(dpsgd_ctx* c) {
     const float* X = c->X[c->cur];
     float* Xn = c->X[c->cur ^ 1];
-    if (c->swapped && c->mix_kind != DPSGD_MIX_TILED_CSR) return launch_mix_variant(c, X, c->G, Xn, true, nullptr);
+    const float* D = nullptr;
+    cudaError_t e = step_direction(c, &D);
+    if (e != cudaSuccess) return e;
+    if (c->swapped && c->mix_kind != DPSGD_MIX_TILED_CSR) return launch_mix_variant(c, X, D, Xn, true, nullptr);
     switch (c->mix_kind) {
-        case DPSGD_MIX_RING: return launch_mix_ring(c, X, c->G, Xn);
-        case DPSGD_MIX_UNIFORM_DENSE: return launch_mix_uniform(c, X, c->G, Xn);
-        case DPSGD_MIX_TILED_CSR: return launch_mix_tiled(c, X, c->G, Xn);
-        default: return launch_mix_gather(c, X, c->G, Xn);
+        case DPSGD_MIX_RING: return launch_mix_ring(c, X, D, Xn);
+        case DPSGD_MIX_UNIFORM_DENSE: return launch_mix_uniform(c, X, D, Xn);
+        case DPSGD_MIX_TILED_CSR: return launch_mix_tiled(c, X, D, Xn);
+        default: return launch_mix_gather(c, X, D, Xn);
     }
 }
 
@@ -246,6 +257,7 @@ DPSGD_API dpsgd_status dpsgd_bind(dpsgd_ctx* c, float* X0, float* X1, float* G, 
     c->X[0] = X0; c->X[1] = X1; c->G = G; c->cur = 0; c->ld = ld;
     c->stream = static_cast<cudaStream_t>(stream);
     c->bound = true;
+    c->V = nullptr; c->beta = 0.f;    // momentum buffers belong to the previous binding
     mix_tiled_release(c);  // tensor maps depend on the bound pointers
     return DPSGD_OK;
 }
@@ -340,8 +352,13 @@ DPSGD_API dpsgd_status dpsgd_mix_update(dpsgd_ctx* c) {
 dpsgd_status mix_with_consensus(dpsgd_ctx* c, double* out_dev) {
     const float* X = c->X[c->cur];
     float* Xn = c->X[c->cur ^ 1];
-    cudaError_t e = launch_mix_variant(c, X, c->G, Xn, c->swapped, out_dev);
-    if (e == cudaErrorNotSupported) {       // no fused kernel for this W: mix, then one pass over the new X
+    const bool fused = c->mix_kind == DPSGD_MIX_RING || c->mix_kind == DPSGD_MIX_UNIFORM_DENSE;
+    cudaError_t e;
+    if (fused) {
+        const float* D = nullptr;
+        e = step_direction(c, &D);
+        if (e == cudaSuccess) e = launch_mix_variant(c, X, D, Xn, c->swapped, out_dev);
+    } else {                                // no fused kernel for this W: mix, then one pass over the new X
         e = run_mix(c);
         if (e == cudaSuccess) e = launch_consensus(c, Xn, out_dev);
     }
@@ -353,6 +370,20 @@ dpsgd_status mix_with_consensus(dpsgd_ctx* c, double* out_dev) {
 DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* c, int32_t update_then_mix) {
     if (!c) return DPSGD_ERR_ARG;
     c->swapped = update_then_mix != 0;
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_set_momentum(dpsgd_ctx* c, float beta, float* V_dev) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    if (!V_dev) { c->V = nullptr; c->beta = 0.f; return DPSGD_OK; }
+    if (!(beta >= 0.f && beta < 1.f)) return fail(c, DPSGD_ERR_ARG, "momentum must be in [0, 1)");
+    if (!aligned(V_dev, 128)) return fail(c, DPSGD_ERR_ALIGN, "V_dev must be 128-byte aligned");
+    const uintptr_t bytes = (uintptr_t)c->n * (uintptr_t)c->ld * sizeof(float);
+    const uintptr_t v = (uintptr_t)V_dev, p[3] = {(uintptr_t)c->X[0], (uintptr_t)c->X[1], (uintptr_t)c->G};
+    for (int a = 0; a < 3; ++a)
+        if (v < p[a] + bytes && p[a] < v + bytes) return fail(c, DPSGD_ERR_ARG, "V_dev overlaps a bound buffer");
+    c->V = V_dev; c->beta = beta;
     return DPSGD_OK;
 }
 

@@ -55,6 +55,8 @@ struct dpsgd_ctx {
     void* d_w_blob = nullptr;  // one allocation holding row_ptr | col | val | band
     int mix_kind = DPSGD_MIX_GATHER_CSR;
     bool swapped = false;      // footnote c of Algorithm 1: update locally, then average
+    float beta = 0.f;          // momentum coefficient
+    float* V = nullptr;        // momentum buffers [n][ld] (caller-owned), NULL = plain SGD
     bool can_ring = false, can_uniform = false, can_tiled = false;
 
     // bound buffers
@@ -106,6 +108,7 @@ void mix_tiled_release(dpsgd_ctx* c);
 cudaError_t launch_consensus(dpsgd_ctx* c, const float* X, double* result_dev);
 cudaError_t ensure_partials(dpsgd_ctx* c, int count);
 cudaError_t launch_consensus_final(dpsgd_ctx* c, int count, double* result_dev);
+cudaError_t launch_momentum(dpsgd_ctx* c, float* V, const float* G);
 cudaError_t launch_mix_variant(dpsgd_ctx* c, const float* X, const float* G, float* Xn, bool swapped,
                                double* stats_out);
 cudaError_t launch_average(dpsgd_ctx* c, const float* X, float* xbar);

@@ -221,7 +221,23 @@ mix_gather_swapped_kernel(const float4* __restrict__ X, const float4* __restrict
     }
 }
 
+// Momentum buffer of the Torch experiments (Section 5.3): V <- beta V + G, in place.
+__global__ void __launch_bounds__(kThreads)
+momentum_kernel(float4* __restrict__ V, const float4* __restrict__ G, int64_t total4, float beta) {
+    const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (t >= total4) return;
+    st_stream(V + t, axpy4(beta, ld_stream(V + t), ld_stream(G + t)));
+}
+
 }  // namespace
+
+cudaError_t launch_momentum(dpsgd_ctx* c, float* V, const float* G) {
+    const int64_t total4 = (int64_t)c->n * c->ld / 4;
+    momentum_kernel<<<(unsigned)((total4 + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(
+        reinterpret_cast<float4*>(V), reinterpret_cast<const float4*>(G), total4, c->beta);
+    c->launches++;
+    return cudaGetLastError();
+}
 
 // stats_out != nullptr: also leave the consensus distance of X_next in *stats_out (device).
 // Returns cudaErrorNotSupported when this W has no fused-statistics kernel (the caller then runs

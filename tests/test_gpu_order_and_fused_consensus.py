@@ -118,3 +118,43 @@ def test_step_consensus_trajectory_on_a_small_mlp():
         assert np.allclose(got, ref, rtol=5e-3, atol=1e-12)
         assert row_rel_err(run.x(), o.X) <= TOL_TRAJ
         run.close()
+
+
+@pytest.mark.parametrize("topo,n,N,swapped", [("ring", 8, 3001, False), ("ring", 64, 20011, True),
+                                              ("dense", 8, 999, False), ("torus", 16, 1234, False),
+                                              ("torus", 16, 1234, True), ("ring+antipode", 8, 515, False)])
+def test_momentum_steps_match_oracle(topo, n, N, swapped):
+    """v <- beta v + g per node, then the gossip step with v (Section 5.3: momentum 0.9)."""
+    rng = np.random.default_rng(N + 1)
+    csr = wl.topology(topo, n)
+    X = _rand(rng, n, N)
+    gamma, beta = 0.1, 0.9
+    run = GpuRun(n, N, csr, gamma, X=X)
+    V = torch.zeros_like(run.X0)
+    run.ctx.set_momentum(beta, V)
+    run.ctx.set_order(swapped)
+    Xr, Vr = X.copy(), np.zeros_like(X)
+    out = torch.zeros(1, dtype=torch.float64, device="cuda")
+    for k in range(6):
+        G = _rand(rng, n, N)
+        run.set_g(G)
+        if k % 2 == 0:
+            run.ctx.mix_update()
+        else:
+            run.ctx.mix_update_consensus(out)
+        Xr, Vr = orc.mix_update_momentum(Xr, Vr, G, *csr, gamma, beta, swapped=swapped)
+        if k % 2 == 1:
+            c_ref = orc.consensus_dist(Xr)
+            assert abs(float(out.item()) - c_ref) <= 1e-4 * c_ref + 1e-9
+    assert row_rel_err(run.x(), Xr) <= 1e-5
+    assert row_rel_err(V[:, :N].cpu().numpy(), Vr) <= 1e-5
+    assert float(V[:, N:].abs().max()) == 0.0 if run.ld > N else True
+    run.check_pads()
+    # switching momentum off restores the plain step
+    run.ctx.set_momentum(0.0, None)
+    G = _rand(rng, n, N)
+    run.set_g(G)
+    run.ctx.mix_update()
+    f = orc.mix_update_swapped if swapped else orc.mix_update
+    assert row_rel_err(run.x(), f(Xr, G, *csr, gamma)) <= TOL_STEP
+    run.close()

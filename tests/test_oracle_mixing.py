@@ -326,3 +326,47 @@ def test_oracle_step_is_grad_then_mix_with_pre_mix_gradient():
     G = orc.gradients(X0, orc.MODEL_LSQ, (d,), A, y, idx)
     expect = orc.mix_update(X0, G, rp, col, val, 0.1)
     assert np.array_equal(o.step(3), expect)
+
+
+# ---- momentum (Section 5.3: learning rate 0.1, momentum 0.9) ---------------------------------
+
+def test_momentum_zero_beta_is_the_plain_step():
+    rng = np.random.default_rng(20)
+    n, N = 6, 11
+    rp, col, val = wl.ring(n)
+    X, V, G = _rand(rng, n, N), _rand(rng, n, N), _rand(rng, n, N)
+    Xn, Vn = orc.mix_update_momentum(X, V, G, rp, col, val, 0.2, 0.0)
+    assert np.array_equal(Vn, G)
+    assert np.array_equal(Xn, orc.mix_update(X, G, rp, col, val, 0.2))
+
+
+def test_momentum_constant_gradient_closed_form():
+    """W = I and a constant gradient g: v_k = g (1 - beta^k)/(1 - beta) and
+    x_k = x_0 - gamma g (k - beta (1 - beta^k)/(1 - beta)) / (1 - beta)."""
+    n, N, K = 3, 5, 30
+    rng = np.random.default_rng(21)
+    X0, g = _rand(rng, n, N), _rand(rng, n, N)
+    beta, gamma = 0.5, 0.25            # exact in fp32
+    X, V = X0.copy(), np.zeros_like(X0)
+    for _ in range(K):
+        X, V = orc.mix_update_momentum(X, V, g, *wl.identity(n), gamma, beta)
+    g64 = g.astype(np.float64)
+    v_K = g64 * (1 - beta ** K) / (1 - beta)
+    x_K = X0 - gamma * g64 * (K - beta * (1 - beta ** K) / (1 - beta)) / (1 - beta)
+    assert np.allclose(V, v_K, rtol=1e-6)
+    assert np.allclose(X, x_K, rtol=0, atol=2e-5)
+
+
+def test_momentum_matches_brute_force_and_both_orders():
+    rng = np.random.default_rng(22)
+    n, N = 4, 6
+    rp, col, val = wl.random_symmetric_doubly_stochastic(n, 5)
+    W = wl.csr_to_dense(n, rp, col, val)
+    X, V, G = _rand(rng, n, N), _rand(rng, n, N), _rand(rng, n, N)
+    gamma, beta = np.float32(0.1), np.float32(0.9)
+    Vb = float(beta) * V.astype(np.float64) + G
+    Xn, Vn = orc.mix_update_momentum(X, V, G, rp, col, val, gamma, beta)
+    assert np.allclose(Vn, Vb, rtol=1e-7)
+    assert np.allclose(Xn, W @ X.astype(np.float64) - float(gamma) * Vn.astype(np.float64), rtol=1e-6, atol=1e-7)
+    Xs, _ = orc.mix_update_momentum(X, V, G, rp, col, val, gamma, beta, swapped=True)
+    assert np.allclose(Xs, W @ (X.astype(np.float64) - float(gamma) * Vn.astype(np.float64)), rtol=1e-6, atol=1e-7)
