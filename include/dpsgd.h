@@ -141,6 +141,14 @@ DPSGD_API dpsgd_status dpsgd_mix_update(dpsgd_ctx* ctx);
 DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* ctx, int32_t update_then_mix);
 
 /*
+ * A local iteration without communication (Section 5.3, last paragraph: a node may run more than
+ * one minibatch before it synchronises): samples xi_{k,i}, computes g_i at x_{k,i} and updates
+ * x_i <- x_i - gamma g_i in place (the gossip step with W = I), momentum included when set.  Call it
+ * tau - 1 times with distinct k between two dpsgd_step() calls for tau local steps per exchange.
+ */
+DPSGD_API dpsgd_status dpsgd_local_step(dpsgd_ctx* ctx, uint64_t k);
+
+/*
  * Momentum as used for both algorithms in the Torch experiments (Section 5.3: learning rate 0.1,
  * momentum 0.9).  The paper prints no formula; the reading is the heavy-ball update of the
  * framework it used, kept per node: v_i <- beta v_i + g_i, then the gossip step with v_i in place

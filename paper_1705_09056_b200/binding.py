@@ -37,6 +37,7 @@ SIGNATURES = {
     "dpsgd_grad": [_vp, _u64],
     "dpsgd_mix_update": [_vp],
     "dpsgd_step": [_vp, _u64],
+    "dpsgd_local_step": [_vp, _u64],
     "dpsgd_set_order": [_vp, _i32],
     "dpsgd_set_momentum": [_vp, _f32, _vp],
     "dpsgd_mix_update_consensus": [_vp, _vp],
@@ -188,6 +189,10 @@ class Dpsgd:
 
     def step(self, k: int):
         self._check(self._lib.dpsgd_step(self._h, k))
+
+    def local_step(self, k: int):
+        """Gradient step without communication (several minibatches between exchanges)."""
+        self._check(self._lib.dpsgd_local_step(self._h, k))
 
     def set_order(self, update_then_mix: bool):
         """Footnote c of Algorithm 1: apply the local gradient first, then average."""

@@ -373,6 +373,17 @@ DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* c, int32_t update_then_mix) {
     return DPSGD_OK;
 }
 
+DPSGD_API dpsgd_status dpsgd_local_step(dpsgd_ctx* c, uint64_t k) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    if ((s = need_model(c)) != DPSGD_OK) return s;
+    cudaError_t e = run_grad(c, k);
+    const float* D = nullptr;
+    if (e == cudaSuccess) e = step_direction(c, &D);
+    if (e == cudaSuccess) e = launch_local_update(c, c->X[c->cur], D);
+    return e == cudaSuccess ? DPSGD_OK : cuda_fail(c, e, "local step");
+}
+
 DPSGD_API dpsgd_status dpsgd_set_momentum(dpsgd_ctx* c, float beta, float* V_dev) {
     dpsgd_status s = need_bound(c);
     if (s != DPSGD_OK) return s;

@@ -109,6 +109,7 @@ cudaError_t launch_consensus(dpsgd_ctx* c, const float* X, double* result_dev);
 cudaError_t ensure_partials(dpsgd_ctx* c, int count);
 cudaError_t launch_consensus_final(dpsgd_ctx* c, int count, double* result_dev);
 cudaError_t launch_momentum(dpsgd_ctx* c, float* V, const float* G);
+cudaError_t launch_local_update(dpsgd_ctx* c, float* X, const float* D);
 cudaError_t launch_mix_variant(dpsgd_ctx* c, const float* X, const float* G, float* Xn, bool swapped,
                                double* stats_out);
 cudaError_t launch_average(dpsgd_ctx* c, const float* X, float* xbar);

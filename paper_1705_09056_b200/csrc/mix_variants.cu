@@ -229,7 +229,23 @@ momentum_kernel(float4* __restrict__ V, const float4* __restrict__ G, int64_t to
     st_stream(V + t, axpy4(beta, ld_stream(V + t), ld_stream(G + t)));
 }
 
+// Local SGD step without communication: X <- X - gamma D, in place (W = I).
+__global__ void __launch_bounds__(kThreads)
+local_update_kernel(float4* __restrict__ X, const float4* __restrict__ D, int64_t total4, float ngamma) {
+    const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (t >= total4) return;
+    st_stream(X + t, axpy4(ngamma, ld_stream(D + t), ld_stream(X + t)));
+}
+
 }  // namespace
+
+cudaError_t launch_local_update(dpsgd_ctx* c, float* X, const float* D) {
+    const int64_t total4 = (int64_t)c->n * c->ld / 4;
+    local_update_kernel<<<(unsigned)((total4 + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(
+        reinterpret_cast<float4*>(X), reinterpret_cast<const float4*>(D), total4, -c->gamma);
+    c->launches++;
+    return cudaGetLastError();
+}
 
 cudaError_t launch_momentum(dpsgd_ctx* c, float* V, const float* G) {
     const int64_t total4 = (int64_t)c->n * c->ld / 4;

@@ -159,3 +159,27 @@ def test_checkpoint_resume_is_bit_identical():
         c.ctx.step(k)
     assert np.array_equal(a.x(), c.x())
     a.close(); c.close()
+
+
+def test_local_steps_between_exchanges_match_oracle():
+    """tau = 3: two iterations without communication (the gossip step with W = I), then one with the
+    ring, repeated; every step uses its own k for the sampler."""
+    w = wl.logistic_workload(n=6, d=40, m=64, batch=8, gamma=0.2, l2_lambda=1e-3, seed=33)
+    A, y = w.A.numpy(), w.y.numpy()
+    csr = w.csr()
+    seed = 8
+    run = GpuRun(w.n, w.N, csr, w.gamma, seed=seed, X=np.zeros((w.n, w.N), np.float32))
+    _attach(run, w, A, y)
+    o = orc.Oracle(w.n, w.N, *csr, w.gamma, seed, w.model, w.dims, w.batch, w.l2_lambda, A, y)
+    ident = wl.identity(w.n)
+    for k in range(18):
+        G = o.grad(k)
+        if k % 3 == 2:
+            run.ctx.step(k)
+            o.mix_update(G)
+        else:
+            run.ctx.local_step(k)
+            o.X = orc.mix_update(o.X, G, *ident, w.gamma)
+    assert row_rel_err(run.x(), o.X) <= 1e-5
+    run.check_pads()
+    run.close()
