@@ -221,7 +221,9 @@ DPSGD_API dpsgd_status dpsgd_current(dpsgd_ctx* ctx, float** X_cur_dev);
 DPSGD_API dpsgd_status dpsgd_set_gamma(dpsgd_ctx* ctx, float gamma);
 
 /* Which DPSGD_MIX_* kernel the structure of W selected; force >= 0 overrides it when the
- * requested kernel can handle W (else DPSGD_ERR_UNSUPPORTED).  Pass force = -1 to query. */
+ * requested kernel can handle W (else DPSGD_ERR_UNSUPPORTED).  Pass force = -1 to query.
+ * Unless a kernel was forced, problems of at most 8 MB per matrix (latency-bound) take a
+ * one-thread-per-output kernel instead, whatever the structure of W. */
 DPSGD_API dpsgd_status dpsgd_mix_kind(dpsgd_ctx* ctx, int32_t force, int32_t* kind_out);
 
 /* Number of kernels this context has launched so far (for launch accounting). */

@@ -154,6 +154,7 @@ cudaError_t run_mix(dpsgd_ctx* c) {
     const float* D = nullptr;
     cudaError_t e = step_direction(c, &D);
     if (e != cudaSuccess) return e;
+    if (!c->kind_forced && mix_is_small(c)) return launch_mix_rowpar(c, X, D, Xn);   // latency-bound sizes
     if (c->swapped && c->mix_kind != DPSGD_MIX_TILED_CSR) return launch_mix_variant(c, X, D, Xn, true, nullptr);
     switch (c->mix_kind) {
         case DPSGD_MIX_RING: return launch_mix_ring(c, X, D, Xn);
@@ -491,6 +492,7 @@ DPSGD_API dpsgd_status dpsgd_mix_kind(dpsgd_ctx* c, int32_t force, int32_t* kind
                         force == DPSGD_MIX_GATHER_CSR;
         if (!ok) return fail(c, DPSGD_ERR_UNSUPPORTED, "this W cannot use the requested mixing kernel");
         c->mix_kind = force;
+        c->kind_forced = true;
     }
     if (kind_out) *kind_out = c->mix_kind;
     return DPSGD_OK;

@@ -58,6 +58,7 @@ struct dpsgd_ctx {
     float beta = 0.f;          // momentum coefficient
     float* V = nullptr;        // momentum buffers [n][ld] (caller-owned), NULL = plain SGD
     bool can_ring = false, can_uniform = false, can_tiled = false;
+    bool kind_forced = false;  // dpsgd_mix_kind(force) was used: no automatic small-problem kernel
 
     // bound buffers
     float* X[2] = {nullptr, nullptr};
@@ -101,6 +102,8 @@ namespace dpsgd {
 cudaError_t launch_mix_ring(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
 cudaError_t launch_mix_uniform(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
 cudaError_t launch_mix_gather(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
+cudaError_t launch_mix_rowpar(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
+bool mix_is_small(const dpsgd_ctx* c);
 cudaError_t launch_mix_tiled(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
 bool mix_tiled_supported(const dpsgd_ctx* c);
 void mix_tiled_release(dpsgd_ctx* c);

@@ -5,9 +5,9 @@
 //   logistic      : F = log(1 + exp(-y (a.w + c)))  g_w = (1/B) sum_b -y_b s_b a_b + l2 w,
 //                   x = [w | c]                     g_c = (1/B) sum_b -y_b s_b,  s_b = sigma(-y_b z_b)
 //
-// Two kernels: a batched GEMV "forward" (one warp per (node, sample): draw the index, dot the
+// Two kernels: a batched GEMV "forward" (one CTA per (node, sample): draw the index, dot the
 // gathered data row with the node's parameters by warp shuffles, turn it into the per-sample
-// coefficient) and a rank-B "backward" (G_i = sum_b coef_b a_b).  All reductions run in a
+// coefficient) and a rank-B "backward" (G_i = sum_b coef_b a_b, eight interleaved slices of the minibatch added in a fixed order).  All reductions run in a
 // fixed order, so results are bit-reproducible.
 #include "ctx.h"
 #include "philox.cuh"
@@ -15,7 +15,7 @@
 namespace dpsgd {
 namespace {
 
-constexpr int kFwdWarps = 8;
+constexpr int kFwdThreads = 256;
 
 __device__ __forceinline__ float warp_allsum(float v) {
 #pragma unroll
@@ -23,14 +23,15 @@ __device__ __forceinline__ float warp_allsum(float v) {
     return v;
 }
 
+// One CTA per (node, sample): all loads of the 16 KB data row are in flight at once (four 128-bit
+// loads per thread at d = 4096), then a shuffle + shared-memory reduction in a fixed order.
 template <int VEC>
-__global__ void __launch_bounds__(kFwdWarps * 32)
+__global__ void __launch_bounds__(kFwdThreads)
 glm_forward_kernel(const float* __restrict__ X, int64_t ld, const float* __restrict__ A,
                    const float* __restrict__ y, int64_t m, int d, int B, int n, uint64_t seed,
                    uint64_t k, int model, int32_t* __restrict__ idx, float* __restrict__ coef) {
-    const int w = blockIdx.x * kFwdWarps + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (w >= n * B) return;
+    __shared__ float part[kFwdThreads / 32];
+    const int w = blockIdx.x;
     const int node = w / B, b = w - node * B;
     const int32_t j = sample_index(seed, k, (uint32_t)node, (uint32_t)b, (uint32_t)m);
     const float* row = A + ((int64_t)node * m + j) * d;
@@ -39,16 +40,33 @@ glm_forward_kernel(const float* __restrict__ X, int64_t ld, const float* __restr
     if (VEC == 4) {
         const float4* r4 = reinterpret_cast<const float4*>(row);
         const float4* x4 = reinterpret_cast<const float4*>(x);
-        for (int c = lane; c < d / 4; c += 32) {
-            const float4 a = __ldg(r4 + c), v = __ldg(x4 + c);
+        const int d4 = d / 4;
+        int c = threadIdx.x;
+        for (; c + 3 * kFwdThreads < d4; c += 4 * kFwdThreads) {
+            float4 a[4], v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { a[u] = __ldcs(r4 + c + u * kFwdThreads); v[u] = __ldg(x4 + c + u * kFwdThreads); }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                acc = fmaf(a[u].x, v[u].x, acc); acc = fmaf(a[u].y, v[u].y, acc);
+                acc = fmaf(a[u].z, v[u].z, acc); acc = fmaf(a[u].w, v[u].w, acc);
+            }
+        }
+        for (; c < d4; c += kFwdThreads) {
+            const float4 a = __ldcs(r4 + c), v = __ldg(x4 + c);
             acc = fmaf(a.x, v.x, acc); acc = fmaf(a.y, v.y, acc);
             acc = fmaf(a.z, v.z, acc); acc = fmaf(a.w, v.w, acc);
         }
     } else {
-        for (int c = lane; c < d; c += 32) acc = fmaf(__ldg(row + c), __ldg(x + c), acc);
+        for (int c = threadIdx.x; c < d; c += kFwdThreads) acc = fmaf(__ldg(row + c), __ldg(x + c), acc);
     }
-    const float dot = warp_allsum(acc);
-    if (lane == 0) {
+    acc = warp_allsum(acc);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float dot = 0.f;
+#pragma unroll
+        for (int t = 0; t < kFwdThreads / 32; ++t) dot += part[t];
         const float yv = __ldg(y + (int64_t)node * m + j);
         float cf;
         if (model == DPSGD_MODEL_LSQ) {
@@ -63,16 +81,16 @@ glm_forward_kernel(const float* __restrict__ X, int64_t ld, const float* __restr
     }
 }
 
-// blockDim = (64, 4): 64 column groups x 4 interleaved slices of the minibatch.
+// blockDim = (32, 8): 32 column groups x 8 interleaved slices of the minibatch.
 template <int VEC>
 __global__ void __launch_bounds__(256)
 glm_backward_kernel(const float* __restrict__ X, float* __restrict__ G, int64_t ld,
                     const float* __restrict__ A, int64_t m, int d, int B, int model, float l2,
                     const int32_t* __restrict__ idx, const float* __restrict__ coef) {
-    __shared__ float red[4][64][VEC];
+    __shared__ float red[8][32][VEC];
     const int node = blockIdx.y;
     const int tx = threadIdx.x, ty = threadIdx.y;
-    const int col = (blockIdx.x * 64 + tx) * VEC;       // first of VEC columns
+    const int col = (blockIdx.x * 32 + tx) * VEC;       // first of VEC columns
     const bool live = col < d;
     float acc[VEC];
 #pragma unroll
@@ -81,7 +99,8 @@ glm_backward_kernel(const float* __restrict__ X, float* __restrict__ G, int64_t 
     const float* cf = coef + (int64_t)node * B;
     if (live) {
         const float* base = A + (int64_t)node * m * d + col;
-        for (int b = ty; b < B; b += 4) {
+#pragma unroll 8
+        for (int b = ty; b < B; b += 8) {
             const float w = __ldg(cf + b);
             const float* row = base + (int64_t)__ldg(ix + b) * d;
             if (VEC == 4) {
@@ -101,14 +120,16 @@ glm_backward_kernel(const float* __restrict__ X, float* __restrict__ G, int64_t 
         const float* x = X + (int64_t)node * ld + col;
 #pragma unroll
         for (int v = 0; v < VEC; ++v) {
-            float s = ((red[0][tx][v] + red[1][tx][v]) + red[2][tx][v]) + red[3][tx][v];
+            float s = red[0][tx][v];
+#pragma unroll
+            for (int t = 1; t < 8; ++t) s += red[t][tx][v];
             if (model == DPSGD_MODEL_LOGISTIC) s = fmaf(l2, __ldg(x + v), s);
             g[v] = s;
         }
     }
     // bias gradient (logistic) and zero padding: columns [d, ld)
     if (blockIdx.x == 0 && ty == 1) {
-        for (int64_t c = d + tx; c < ld; c += 64) {
+        for (int64_t c = d + tx; c < ld; c += 32) {
             float s = 0.f;
             if (model == DPSGD_MODEL_LOGISTIC && c == d)
                 for (int b = 0; b < B; ++b) s += __ldg(cf + b);
@@ -122,16 +143,16 @@ glm_backward_kernel(const float* __restrict__ X, float* __restrict__ G, int64_t 
 cudaError_t launch_grad_linear(dpsgd_ctx* c, uint64_t k, const float* X, float* G) {
     const int n = c->n, B = c->batch, d = c->d;
     const float* y = static_cast<const float*>(c->y);
-    const int fwd_grid = (n * B + kFwdWarps - 1) / kFwdWarps;
+    const int fwd_grid = n * B;
     const bool vec = (d % 4 == 0);
     if (vec)
-        glm_forward_kernel<4><<<fwd_grid, kFwdWarps * 32, 0, c->stream>>>(
+        glm_forward_kernel<4><<<fwd_grid, kFwdThreads, 0, c->stream>>>(
             X, c->ld, c->A, y, c->m, d, B, n, c->seed, k, c->model, c->d_idx, c->d_coef);
     else
-        glm_forward_kernel<1><<<fwd_grid, kFwdWarps * 32, 0, c->stream>>>(
+        glm_forward_kernel<1><<<fwd_grid, kFwdThreads, 0, c->stream>>>(
             X, c->ld, c->A, y, c->m, d, B, n, c->seed, k, c->model, c->d_idx, c->d_coef);
     const int vw = vec ? 4 : 1;
-    dim3 grid((d + 64 * vw - 1) / (64 * vw), n), block(64, 4);
+    dim3 grid((d + 32 * vw - 1) / (32 * vw), n), block(32, 8);
     if (vec)
         glm_backward_kernel<4><<<grid, block, 0, c->stream>>>(X, G, c->ld, c->A, c->m, d, B, c->model,
                                                               c->l2, c->d_idx, c->d_coef);

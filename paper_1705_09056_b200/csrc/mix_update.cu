@@ -150,7 +150,54 @@ mix_gather_kernel(const float4* __restrict__ X, const float4* __restrict__ G, fl
     }
 }
 
+// Small problems (X fits L2 many times over): one thread per OUTPUT group of 4 columns instead of
+// one per column walking all rows, so the step is a single load-compute-store latency deep.  The
+// neighbour rows are re-read through L1/L2, which costs nothing at this size.
+__global__ void __launch_bounds__(128)
+mix_rowpar_kernel(const float4* __restrict__ X, const float4* __restrict__ G, float4* __restrict__ Xn,
+                  const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col,
+                  const float* __restrict__ val, int n, int64_t ld4, float ngamma, int swapped) {
+    const int64_t c = (int64_t)blockIdx.x * 128 + threadIdx.x;
+    const int i = blockIdx.y;
+    if (c >= ld4) return;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int pe = __ldg(row_ptr + i + 1);
+    for (int p = __ldg(row_ptr + i); p < pe; ++p) {
+        const float w = __ldg(val + p);
+        const int64_t j = __ldg(col + p);
+        float4 v = __ldg(X + j * ld4 + c);
+        if (swapped) {
+            const float4 g = __ldg(G + j * ld4 + c);
+            v.x = fmaf(ngamma, g.x, v.x); v.y = fmaf(ngamma, g.y, v.y);
+            v.z = fmaf(ngamma, g.z, v.z); v.w = fmaf(ngamma, g.w, v.w);
+        }
+        a.x = fmaf(w, v.x, a.x); a.y = fmaf(w, v.y, a.y);
+        a.z = fmaf(w, v.z, a.z); a.w = fmaf(w, v.w, a.w);
+    }
+    if (!swapped) {
+        const float4 g = __ldg(G + (int64_t)i * ld4 + c);
+        a.x = fmaf(ngamma, g.x, a.x); a.y = fmaf(ngamma, g.y, a.y);
+        a.z = fmaf(ngamma, g.z, a.z); a.w = fmaf(ngamma, g.w, a.w);
+    }
+    Xn[(int64_t)i * ld4 + c] = a;
+}
+
 }  // namespace
+
+bool mix_is_small(const dpsgd_ctx* c) {
+    return (int64_t)c->n * c->ld * (int64_t)sizeof(float) <= (int64_t(8) << 20) && c->n <= 65535 &&
+           (int64_t)c->W.nnz <= (int64_t)c->n * 32;
+}
+
+cudaError_t launch_mix_rowpar(dpsgd_ctx* c, const float* X, const float* G, float* Xn) {
+    const int64_t ld4 = c->ld / 4;
+    dim3 grid((unsigned)((ld4 + 127) / 128), (unsigned)c->n);
+    mix_rowpar_kernel<<<grid, 128, 0, c->stream>>>(
+        reinterpret_cast<const float4*>(X), reinterpret_cast<const float4*>(G), reinterpret_cast<float4*>(Xn),
+        c->W.row_ptr, c->W.col, c->W.val, c->n, ld4, -c->gamma, c->swapped ? 1 : 0);
+    c->launches++;
+    return cudaGetLastError();
+}
 
 cudaError_t launch_mix_ring(dpsgd_ctx* c, const float* X, const float* G, float* Xn) {
     const int64_t ld4 = c->ld / 4;
