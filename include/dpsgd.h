@@ -173,6 +173,13 @@ DPSGD_API dpsgd_status dpsgd_step_consensus(dpsgd_ctx* ctx, uint64_t k, double* 
 /* One full iteration k of Algorithm 1: dpsgd_grad(k) followed by dpsgd_mix_update(). */
 DPSGD_API dpsgd_status dpsgd_step(dpsgd_ctx* ctx, uint64_t k);
 
+/* The loop of Algorithm 1: iterations k_first, k_first + 1, ... (dpsgd_step each), enqueued in one
+ * call.  For launch-bound sizes (linear models, matrices of at most 8 MB, at least 8 iterations) a
+ * pair of iterations is captured once into a CUDA graph that reads the iteration number from
+ * device memory, and replayed; results are identical to repeated dpsgd_step calls.  The bound
+ * stream must not be used by other threads during the call. */
+DPSGD_API dpsgd_status dpsgd_run(dpsgd_ctx* ctx, uint64_t k_first, int64_t iterations);
+
 /*
  * sum_i || xbar - x_i ||^2 over the current X (sum_i Q_{k,i} of Eq. 10; divide by n for M_k
  * of Eq. 13), accumulated in fp64.  Waits for the stream and writes one double to host memory.

@@ -34,7 +34,7 @@ MODEL_MLP = 2
 
 # ------------------------------------------------------------------------------------------
 # Algorithm 1, step "randomly sample xi_{k,i} from local data of node i".
-# The paper fixes no generator; this build uses the counter-based Philox4x32-10 of Salmon,
+# The paper fixes no generator; this implementation uses the counter-based Philox4x32-10 of Salmon,
 # Moraes, Dror and Shaw (SC'11), keyed by the run seed, with the counter holding
 # (draw block, node, iteration).
 # ------------------------------------------------------------------------------------------

@@ -37,6 +37,7 @@ SIGNATURES = {
     "dpsgd_grad": [_vp, _u64],
     "dpsgd_mix_update": [_vp],
     "dpsgd_step": [_vp, _u64],
+    "dpsgd_run": [_vp, _u64, _i64],
     "dpsgd_local_step": [_vp, _u64],
     "dpsgd_set_order": [_vp, _i32],
     "dpsgd_set_momentum": [_vp, _f32, _vp],
@@ -213,6 +214,10 @@ class Dpsgd:
     def step_consensus(self, k: int, out: torch.Tensor):
         assert out.is_cuda and out.dtype == torch.float64 and out.numel() >= 1
         self._check(self._lib.dpsgd_step_consensus(self._h, k, _ptr(out)))
+
+    def run(self, k_first: int, iterations: int):
+        """Iterations k_first .. k_first + iterations - 1 of Algorithm 1, enqueued by one call."""
+        self._check(self._lib.dpsgd_run(self._h, k_first, iterations))
 
     def consensus_dist(self) -> float:
         out = ctypes.c_double()

@@ -106,6 +106,11 @@ void classify_w(dpsgd_ctx* c) {
     else c->mix_kind = DPSGD_MIX_GATHER_CSR;
 }
 
+// Anything baked into a captured graph changed: drop it.
+void drop_graph(dpsgd_ctx* c) {
+    if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
+}
+
 float band_entry(const dpsgd_ctx* c, int i, int j) {
     for (int p = c->h_row_ptr[i]; p < c->h_row_ptr[i + 1]; ++p)
         if (c->h_col[p] == j) return c->h_val[p];
@@ -117,6 +122,9 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) %
 void release(dpsgd_ctx* c) {
     if (!c) return;
     mix_tiled_release(c);
+    drop_graph(c);
+    if (c->capture_stream) cudaStreamDestroy(c->capture_stream);
+    cudaFree(c->d_k);
     cudaFree(c->d_w_blob);
     cudaFree(c->d_idx);
     cudaFree(c->d_coef);
@@ -257,6 +265,7 @@ DPSGD_API dpsgd_status dpsgd_bind(dpsgd_ctx* c, float* X0, float* X1, float* G, 
                 return fail(c, DPSGD_ERR_ARG, "X0, X1 and G must not overlap");
     c->X[0] = X0; c->X[1] = X1; c->G = G; c->cur = 0; c->ld = ld;
     c->stream = static_cast<cudaStream_t>(stream);
+    drop_graph(c);
     c->bound = true;
     c->V = nullptr; c->beta = 0.f;    // momentum buffers belong to the previous binding
     mix_tiled_release(c);  // tensor maps depend on the bound pointers
@@ -297,6 +306,7 @@ DPSGD_API dpsgd_status dpsgd_set_model(dpsgd_ctx* c, int32_t kind, const int32_t
         return fail(c, DPSGD_ERR_ARG, buf);
     }
     if (c->bound) cudaStreamSynchronize(c->stream);
+    drop_graph(c);
     cudaFree(c->d_idx); cudaFree(c->d_coef); cudaFree(c->d_act); cudaFree(c->d_delta);
     c->d_idx = nullptr; c->d_coef = nullptr; c->d_act = nullptr; c->d_delta = nullptr;
     c->model = kind; c->d = dims[0]; c->batch = batch; c->l2 = l2_lambda; c->mlp = shape;
@@ -320,6 +330,7 @@ DPSGD_API dpsgd_status dpsgd_set_data(dpsgd_ctx* c, const float* A, const void* 
     if (m < 1 || m >= (int64_t(1) << 31)) return fail(c, DPSGD_ERR_ARG, "m_per_node must be in [1, 2^31)");
     if (d != c->d) return fail(c, DPSGD_ERR_ARG, "d does not match the model's input width");
     if (!aligned(A, 16) || !aligned(y, 16)) return fail(c, DPSGD_ERR_ALIGN, "A and y must be 16-byte aligned");
+    drop_graph(c);
     c->A = A; c->y = y; c->m = m; c->have_data = true;
     return DPSGD_OK;
 }
@@ -370,6 +381,7 @@ dpsgd_status mix_with_consensus(dpsgd_ctx* c, double* out_dev) {
 
 DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* c, int32_t update_then_mix) {
     if (!c) return DPSGD_ERR_ARG;
+    drop_graph(c);
     c->swapped = update_then_mix != 0;
     return DPSGD_OK;
 }
@@ -388,6 +400,7 @@ DPSGD_API dpsgd_status dpsgd_local_step(dpsgd_ctx* c, uint64_t k) {
 DPSGD_API dpsgd_status dpsgd_set_momentum(dpsgd_ctx* c, float beta, float* V_dev) {
     dpsgd_status s = need_bound(c);
     if (s != DPSGD_OK) return s;
+    drop_graph(c);
     if (!V_dev) { c->V = nullptr; c->beta = 0.f; return DPSGD_OK; }
     if (!(beta >= 0.f && beta < 1.f)) return fail(c, DPSGD_ERR_ARG, "momentum must be in [0, 1)");
     if (!aligned(V_dev, 128)) return fail(c, DPSGD_ERR_ALIGN, "V_dev must be 128-byte aligned");
@@ -427,6 +440,77 @@ DPSGD_API dpsgd_status dpsgd_step(dpsgd_ctx* c, uint64_t k) {
     e = run_mix(c);
     if (e != cudaSuccess) return cuda_fail(c, e, "mix_update kernel");
     c->cur ^= 1;
+    return DPSGD_OK;
+}
+
+// Captures two iterations (the X buffers swap back) that read the iteration number from device
+// memory and advance it, so that one graph can be replayed for any k.
+dpsgd_status capture_pair(dpsgd_ctx* c) {
+    cudaError_t e = cudaSuccess;
+    if (!c->d_k) e = cudaMalloc(&c->d_k, sizeof(uint64_t));
+    if (e != cudaSuccess) return cuda_fail(c, e, "iteration counter");
+    // record on a private stream (the bound one may be the legacy default stream, which cannot
+    // capture); the instantiated graph is launched on the bound stream
+    if (!c->capture_stream) e = cudaStreamCreateWithFlags(&c->capture_stream, cudaStreamNonBlocking);
+    if (e != cudaSuccess) return cuda_fail(c, e, "capture stream");
+    const int cur0 = c->cur;
+    const int64_t launches0 = c->launches;
+    cudaStream_t bound_stream = c->stream;
+    e = cudaStreamBeginCapture(c->capture_stream, cudaStreamCaptureModeThreadLocal);
+    if (e != cudaSuccess) return cuda_fail(c, e, "begin capture");
+    c->stream = c->capture_stream;
+    c->k_dev_active = c->d_k;
+    dpsgd_status s = DPSGD_OK;
+    for (int t = 0; t < 2 && s == DPSGD_OK; ++t) {
+        s = dpsgd_step(c, 0);
+        if (s == DPSGD_OK && launch_advance_k(c) != cudaSuccess) s = DPSGD_ERR_CUDA;
+    }
+    c->k_dev_active = nullptr;
+    c->stream = bound_stream;
+    cudaGraph_t graph = nullptr;
+    e = cudaStreamEndCapture(c->capture_stream, &graph);
+    c->cur = cur0;                                // nothing ran: the capture only recorded
+    c->graph_launches = c->launches - launches0;
+    c->launches = launches0;
+    if (s != DPSGD_OK || e != cudaSuccess || !graph) {
+        if (graph) cudaGraphDestroy(graph);
+        return s != DPSGD_OK ? s : cuda_fail(c, e, "end capture");
+    }
+    e = cudaGraphInstantiate(&c->graph_exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess) { c->graph_exec = nullptr; return cuda_fail(c, e, "graph instantiate"); }
+    c->graph_cur = cur0;
+    return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_run(dpsgd_ctx* c, uint64_t k_first, int64_t iterations) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    if ((s = need_model(c)) != DPSGD_OK) return s;
+    if (iterations < 0) return fail(c, DPSGD_ERR_ARG, "iterations must be >= 0");
+    int64_t t = 0;
+    // Launch-bound sizes only: replay a captured pair of iterations.  The first two iterations always
+    // run directly, which also completes any first-use set-up before a capture starts.
+    const bool small = mix_is_small(c) && c->model != DPSGD_MODEL_MLP && iterations >= 8;
+    if (small) {
+        for (; t < 2; ++t)
+            if ((s = dpsgd_step(c, k_first + (uint64_t)t)) != DPSGD_OK) return s;
+        if (!c->graph_exec && capture_pair(c) != DPSGD_OK) drop_graph(c);
+        if (c->graph_exec) {
+            if (c->cur != c->graph_cur) {           // bring the buffer parity to the captured one
+                if ((s = dpsgd_step(c, k_first + (uint64_t)t)) != DPSGD_OK) return s;
+                ++t;
+            }
+            cudaError_t e = launch_set_k(c, k_first + (uint64_t)t);
+            for (; e == cudaSuccess && t + 2 <= iterations; t += 2) {
+                e = cudaGraphLaunch(c->graph_exec, c->stream);
+                c->launches += c->graph_launches;
+            }
+            if (e != cudaSuccess) return cuda_fail(c, e, "graph replay");
+        }
+    }
+    for (; t < iterations; ++t)
+        if ((s = dpsgd_step(c, k_first + (uint64_t)t)) != DPSGD_OK) return s;
     return DPSGD_OK;
 }
 
@@ -479,6 +563,7 @@ DPSGD_API dpsgd_status dpsgd_current(dpsgd_ctx* c, float** X_cur) {
 DPSGD_API dpsgd_status dpsgd_set_gamma(dpsgd_ctx* c, float gamma) {
     if (!c) return DPSGD_ERR_ARG;
     if (!(gamma == gamma)) return fail(c, DPSGD_ERR_ARG, "gamma is NaN");
+    drop_graph(c);
     c->gamma = gamma;
     return DPSGD_OK;
 }
@@ -491,6 +576,7 @@ DPSGD_API dpsgd_status dpsgd_mix_kind(dpsgd_ctx* c, int32_t force, int32_t* kind
                         (force == DPSGD_MIX_TILED_CSR && c->can_tiled) ||
                         force == DPSGD_MIX_GATHER_CSR;
         if (!ok) return fail(c, DPSGD_ERR_UNSUPPORTED, "this W cannot use the requested mixing kernel");
+        drop_graph(c);
         c->mix_kind = force;
         c->kind_forced = true;
     }

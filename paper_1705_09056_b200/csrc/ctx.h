@@ -92,6 +92,14 @@ struct dpsgd_ctx {
     dpsgd::ResultBlock* h_result = nullptr;  // pinned
     void* tma_state = nullptr;     // tensor maps for the tiled mixing kernel
 
+    // graph replay of pairs of iterations (small, launch-bound problems)
+    uint64_t* d_k = nullptr;                 // device iteration counter
+    const uint64_t* k_dev_active = nullptr;  // non-NULL only while a graph is captured
+    cudaGraphExec_t graph_exec = nullptr;
+    cudaStream_t capture_stream = nullptr;   // private stream the pair is recorded on
+    int graph_cur = 0;                       // value of `cur` the graph was captured at
+    int64_t graph_launches = 0;              // kernels in one replay
+
     int64_t launches = 0;
     std::string err;
 };
@@ -118,6 +126,8 @@ cudaError_t launch_mix_variant(dpsgd_ctx* c, const float* X, const float* G, flo
 cudaError_t launch_average(dpsgd_ctx* c, const float* X, float* xbar);
 
 cudaError_t launch_sample(dpsgd_ctx* c, uint64_t k, int32_t* idx);
+cudaError_t launch_set_k(dpsgd_ctx* c, uint64_t v);
+cudaError_t launch_advance_k(dpsgd_ctx* c);
 cudaError_t launch_grad_linear(dpsgd_ctx* c, uint64_t k, const float* X, float* G);
 cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G);
 size_t mlp_act_floats(const dpsgd_ctx* c);

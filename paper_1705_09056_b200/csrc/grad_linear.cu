@@ -29,10 +29,12 @@ template <int VEC>
 __global__ void __launch_bounds__(kFwdThreads)
 glm_forward_kernel(const float* __restrict__ X, int64_t ld, const float* __restrict__ A,
                    const float* __restrict__ y, int64_t m, int d, int B, int n, uint64_t seed,
-                   uint64_t k, int model, int32_t* __restrict__ idx, float* __restrict__ coef) {
+                   uint64_t k, const uint64_t* __restrict__ k_ptr, int model, int32_t* __restrict__ idx,
+                   float* __restrict__ coef) {
     __shared__ float part[kFwdThreads / 32];
     const int w = blockIdx.x;
     const int node = w / B, b = w - node * B;
+    if (k_ptr) k = *k_ptr;        // iteration counter kept on the device (graph replay)
     const int32_t j = sample_index(seed, k, (uint32_t)node, (uint32_t)b, (uint32_t)m);
     const float* row = A + ((int64_t)node * m + j) * d;
     const float* x = X + (int64_t)node * ld;
@@ -147,10 +149,10 @@ cudaError_t launch_grad_linear(dpsgd_ctx* c, uint64_t k, const float* X, float* 
     const bool vec = (d % 4 == 0);
     if (vec)
         glm_forward_kernel<4><<<fwd_grid, kFwdThreads, 0, c->stream>>>(
-            X, c->ld, c->A, y, c->m, d, B, n, c->seed, k, c->model, c->d_idx, c->d_coef);
+            X, c->ld, c->A, y, c->m, d, B, n, c->seed, k, c->k_dev_active, c->model, c->d_idx, c->d_coef);
     else
         glm_forward_kernel<1><<<fwd_grid, kFwdThreads, 0, c->stream>>>(
-            X, c->ld, c->A, y, c->m, d, B, n, c->seed, k, c->model, c->d_idx, c->d_coef);
+            X, c->ld, c->A, y, c->m, d, B, n, c->seed, k, c->k_dev_active, c->model, c->d_idx, c->d_coef);
     const int vw = vec ? 4 : 1;
     dim3 grid((d + 32 * vw - 1) / (32 * vw), n), block(32, 8);
     if (vec)

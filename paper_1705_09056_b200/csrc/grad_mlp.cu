@@ -44,7 +44,8 @@ MlpPlan make_plan(const dpsgd_ctx* c) {
 // h_0[node][b][:] = A[node][idx][:] with idx drawn for (iteration k, node, b).
 __global__ void __launch_bounds__(128)
 mlp_gather_kernel(const float* __restrict__ A, int64_t m, int d, int B, uint64_t seed, uint64_t k,
-                  int32_t* __restrict__ idx, float* __restrict__ h0) {
+                  const uint64_t* __restrict__ k_ptr, int32_t* __restrict__ idx, float* __restrict__ h0) {
+    if (k_ptr) k = *k_ptr;        // iteration counter kept on the device (graph replay)
     const int node = blockIdx.y, b = blockIdx.x;
     const int32_t j = sample_index(seed, k, (uint32_t)node, (uint32_t)b, (uint32_t)m);
     if (threadIdx.x == 0) idx[node * B + b] = j;
@@ -269,7 +270,7 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) 
     const int32_t* y = static_cast<const int32_t*>(c->y);
     const bool use_tc = c->mlp_precision != 2 && B <= 128;   // precision 2 = fp32 FMA kernel
 
-    mlp_gather_kernel<<<dim3(B, n), 128, 0, c->stream>>>(c->A, c->m, s.dims[0], B, c->seed, k, c->d_idx,
+    mlp_gather_kernel<<<dim3(B, n), 128, 0, c->stream>>>(c->A, c->m, s.dims[0], B, c->seed, k, c->k_dev_active, c->d_idx,
                                                          c->d_act + p.act_off[0]);
     c->launches++;
 

@@ -12,7 +12,22 @@ __global__ void sample_kernel(uint64_t seed, uint64_t k, int n, int B, uint32_t 
     idx[t] = sample_index(seed, k, (uint32_t)node, (uint32_t)b, m);
 }
 
+__global__ void set_k_kernel(uint64_t* k, uint64_t v) { *k = v; }
+__global__ void advance_k_kernel(uint64_t* k) { *k += 1; }
+
 }  // namespace
+
+cudaError_t launch_set_k(dpsgd_ctx* c, uint64_t v) {
+    set_k_kernel<<<1, 1, 0, c->stream>>>(c->d_k, v);
+    c->launches++;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_advance_k(dpsgd_ctx* c) {
+    advance_k_kernel<<<1, 1, 0, c->stream>>>(c->d_k);
+    c->launches++;
+    return cudaGetLastError();
+}
 
 cudaError_t launch_sample(dpsgd_ctx* c, uint64_t k, int32_t* idx) {
     const int total = c->n * c->batch;

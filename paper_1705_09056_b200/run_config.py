@@ -74,11 +74,19 @@ def main():
             ctx.step(args.warmup + k)
     ms_step = timed(whole, args.steps)
     launches = (ctx.launch_count() - l0) / args.steps
+    # the same iterations enqueued by one library call (no per-step binding overhead)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    ctx.run(args.warmup + args.steps, args.steps)
+    b.record()
+    torch.cuda.synchronize()
+    ms_run = a.elapsed_time(b) / args.steps
     ms_grad = timed(lambda k: ctx.grad(k), max(3, args.steps // 5))
     ms_mix = timed(lambda k: ctx.mix_update(), max(3, args.steps // 5))
     print(json.dumps({
         "workload": w.name, "n": w.n, "N": w.N, "dims": list(w.dims), "batch": w.batch, "topology": w.topology,
-        "mix_kernel": binding.MIX_NAMES[ctx.mix_kind()], "ms_per_step": ms_step,
+        "mix_kernel": binding.MIX_NAMES[ctx.mix_kind()], "ms_per_step": ms_step, "ms_per_step_one_call": ms_run,
         "replica_steps_per_s": w.n / (ms_step * 1e-3), "ms_grad": ms_grad, "ms_mix_update": ms_mix,
         "launches_per_step": launches, "consensus": ctx.consensus_dist()}))
     ctx.close()

@@ -183,3 +183,47 @@ def test_local_steps_between_exchanges_match_oracle():
     assert row_rel_err(run.x(), o.X) <= 1e-5
     run.check_pads()
     run.close()
+
+
+def test_run_equals_repeated_steps():
+    w = wl.lsq_workload(n=6, d=32, m=128, batch=8)
+    A, y = w.A.numpy(), w.y.numpy()
+    X0 = np.zeros((w.n, w.N), dtype=np.float32)
+    a = GpuRun(w.n, w.N, w.csr(), w.gamma, seed=5, X=X0)
+    _attach(a, w, A, y)
+    for k in range(3, 33):
+        a.ctx.step(k)
+    b = GpuRun(w.n, w.N, w.csr(), w.gamma, seed=5, X=X0)
+    _attach(b, w, A, y)
+    b.ctx.run(3, 30)
+    assert np.array_equal(a.x(), b.x())
+    a.close(); b.close()
+
+
+@pytest.mark.parametrize("model", [binding.MODEL_LSQ, binding.MODEL_LOGISTIC])
+def test_graph_replayed_run_is_bit_identical_to_steps(model):
+    """dpsgd_run replays a captured pair of iterations for small problems; odd counts, several
+    calls in a row and a change of gamma in between must all equal plain stepping."""
+    w = _linear_workload(model, 8, 64, 256, 16)
+    A, y = w.A.numpy(), w.y.numpy()
+    X0 = np.zeros((w.n, w.N), dtype=np.float32)
+    a = GpuRun(w.n, w.N, w.csr(), w.gamma, seed=5, X=X0)
+    _attach(a, w, A, y)
+    b = GpuRun(w.n, w.N, w.csr(), w.gamma, seed=5, X=X0)
+    _attach(b, w, A, y)
+    k = 0
+    for count, gamma in ((9, w.gamma), (20, w.gamma), (3, w.gamma), (31, 0.5 * w.gamma), (8, 0.5 * w.gamma)):
+        a.ctx.set_gamma(gamma); b.ctx.set_gamma(gamma)
+        for t in range(count):
+            a.ctx.step(k + t)
+        b.ctx.run(k, count)
+        k += count
+        assert np.array_equal(a.x(), b.x()), (count, gamma)
+    o = orc.Oracle(w.n, w.N, *w.csr(), w.gamma, 5, w.model, w.dims, w.batch, w.l2_lambda, A, y)
+    for t in range(29):
+        o.step(t)
+    c = GpuRun(w.n, w.N, w.csr(), w.gamma, seed=5, X=X0)
+    _attach(c, w, A, y)
+    c.ctx.run(0, 29)
+    assert row_rel_err(c.x(), o.X) <= TOL_TRAJ
+    a.close(); b.close(); c.close()
