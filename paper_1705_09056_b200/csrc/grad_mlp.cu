@@ -187,14 +187,11 @@ void run_gemm(dpsgd_ctx* c, const GemmArgs& g) {
 
 template <int NT, bool A_K, bool B_K, bool VEC, bool PRECISE>
 cudaError_t launch_tc_inst(dpsgd_ctx* c, const tc::Args& a, int n_tiles) {
-    static bool attr_set = false;
     auto kernel = tc::tc_gemm_kernel<NT, A_K, B_K, VEC, PRECISE>;
     constexpr size_t smem = tc::smem_bytes<NT, A_K, B_K, PRECISE>();
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    // per device and cheap: set on every launch rather than remembered in a process-wide flag
+    cudaError_t ea = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (ea != cudaSuccess) return ea;
     dim3 grid((a.M + tc::kTileM - 1) / tc::kTileM, (n_tiles + a.n_per_cta - 1) / a.n_per_cta, c->n);
     kernel<<<grid, tc::kThreads, smem, c->stream>>>(a);
     c->launches++;

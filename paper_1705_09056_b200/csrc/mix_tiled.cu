@@ -262,13 +262,11 @@ bool pick_shape(int n, int nnz, int* T_out, int* S_out, int* ctas_out) {
 
 template <int T, int S, bool X_TMA, bool SWAPPED>
 cudaError_t launch_tsx(dpsgd_ctx* c, TiledState* st, int which, const float* G, float* Xn) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(mix_tiled_kernel<T, S, X_TMA, SWAPPED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)(kSmemPerSm - kSmemPerCtaReserve));
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    // per device and cheap: set on every launch rather than remembered in a process-wide flag
+    cudaError_t ea = cudaFuncSetAttribute(mix_tiled_kernel<T, S, X_TMA, SWAPPED>,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)(kSmemPerSm - kSmemPerCtaReserve));
+    if (ea != cudaSuccess) return ea;
     const int64_t ld4 = c->ld / 4;
     const int64_t tiles = (c->ld + T - 1) / T;
     const int grid = (int)std::min<int64_t>(tiles, st->grid);
