@@ -156,14 +156,21 @@ cudaError_t step_direction(dpsgd_ctx* c, const float** dir) {
     return launch_momentum(c, c->V, c->G);
 }
 
+// Ring and uniform W have kernels that update the momentum buffers inside the gossip pass.
+bool momentum_fuses(const dpsgd_ctx* c) {
+    return c->V && (c->mix_kind == DPSGD_MIX_RING || c->mix_kind == DPSGD_MIX_UNIFORM_DENSE);
+}
+
 cudaError_t run_mix(dpsgd_ctx* c) {
     const float* X = c->X[c->cur];
     float* Xn = c->X[c->cur ^ 1];
+    const bool small = !c->kind_forced && mix_is_small(c);
+    if (!small && momentum_fuses(c)) return launch_mix_variant(c, X, c->G, Xn, c->swapped, nullptr, c->V);
     const float* D = nullptr;
     cudaError_t e = step_direction(c, &D);
     if (e != cudaSuccess) return e;
-    if (!c->kind_forced && mix_is_small(c)) return launch_mix_rowpar(c, X, D, Xn);   // latency-bound sizes
-    if (c->swapped && c->mix_kind != DPSGD_MIX_TILED_CSR) return launch_mix_variant(c, X, D, Xn, true, nullptr);
+    if (small) return launch_mix_rowpar(c, X, D, Xn);   // latency-bound sizes
+    if (c->swapped && c->mix_kind != DPSGD_MIX_TILED_CSR) return launch_mix_variant(c, X, D, Xn, true, nullptr, nullptr);
     switch (c->mix_kind) {
         case DPSGD_MIX_RING: return launch_mix_ring(c, X, D, Xn);
         case DPSGD_MIX_UNIFORM_DENSE: return launch_mix_uniform(c, X, D, Xn);
@@ -367,9 +374,7 @@ dpsgd_status mix_with_consensus(dpsgd_ctx* c, double* out_dev) {
     const bool fused = c->mix_kind == DPSGD_MIX_RING || c->mix_kind == DPSGD_MIX_UNIFORM_DENSE;
     cudaError_t e;
     if (fused) {
-        const float* D = nullptr;
-        e = step_direction(c, &D);
-        if (e == cudaSuccess) e = launch_mix_variant(c, X, D, Xn, c->swapped, out_dev);
+        e = launch_mix_variant(c, X, c->G, Xn, c->swapped, out_dev, c->V);   // V, when set, updated in the pass
     } else {                                // no fused kernel for this W: mix, then one pass over the new X
         e = run_mix(c);
         if (e == cudaSuccess) e = launch_consensus(c, Xn, out_dev);

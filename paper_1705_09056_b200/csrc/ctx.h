@@ -122,7 +122,7 @@ cudaError_t launch_consensus_final(dpsgd_ctx* c, int count, double* result_dev);
 cudaError_t launch_momentum(dpsgd_ctx* c, float* V, const float* G);
 cudaError_t launch_local_update(dpsgd_ctx* c, float* X, const float* D);
 cudaError_t launch_mix_variant(dpsgd_ctx* c, const float* X, const float* G, float* Xn, bool swapped,
-                               double* stats_out);
+                               double* stats_out, float* V);
 cudaError_t launch_average(dpsgd_ctx* c, const float* X, float* xbar);
 
 cudaError_t launch_sample(dpsgd_ctx* c, uint64_t k, int32_t* idx);

@@ -8,7 +8,11 @@
 //            over HBM.  Per column the new rows are shifted by the first one and sum d, sum d^2 are
 //            kept in fp64; per-CTA partials are added in a fixed order by consensus_final.
 //
-// Same traffic as the plain kernels: X and G read once, X_next written once.
+//   MOM      the momentum buffers of the Section 5.3 runs, updated in the same pass: where row j of G is
+//            loaded, d_j = beta V[j] + G[j] is formed, written back to V[j] and used in place of G[j]
+//            (20 bytes per replica-parameter instead of 24 with a separate momentum pass).
+//
+// Same traffic as the plain kernels otherwise: X and G read once, X_next written once.
 #include "ctx.h"
 
 namespace dpsgd {
@@ -74,11 +78,11 @@ struct ColumnStats {
 
 // Ring (Theorem 3).  v_j = X[j] (Algorithm 1 order) or X[j] - gamma G[j] (footnote c); a rolling
 // register window (prev, cur, next) over v walks down the column, rows 0 and n-1 kept for the wrap.
-template <bool SWAPPED, bool STATS>
+template <bool SWAPPED, bool STATS, bool MOM>
 __global__ void __launch_bounds__(kThreads)
 mix_ring_x_kernel(const float4* __restrict__ X, const float4* __restrict__ G, float4* __restrict__ Xn,
-                  const float* __restrict__ band, int n, int64_t ld4, float ngamma,
-                  double* __restrict__ partials) {
+                  float4* __restrict__ V, float beta, const float* __restrict__ band, int n, int64_t ld4,
+                  float ngamma, double* __restrict__ partials) {
     __shared__ double red[kThreads / 32];
     const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     ColumnStats st;
@@ -87,21 +91,38 @@ mix_ring_x_kernel(const float4* __restrict__ X, const float4* __restrict__ G, fl
         const float4* x = X + c;
         const float4* g = G + c;
         float4* o = Xn + c;
+        float4* vb = MOM ? V + c : nullptr;
+        auto direction = [&](int j) {            // row j of G, or of the updated momentum buffers
+            const float4 gv = ld_stream(g + (int64_t)j * ld4);
+            if (!MOM) return gv;
+            const float4 d = axpy4(beta, ld_stream(vb + (int64_t)j * ld4), gv);
+            st_stream(vb + (int64_t)j * ld4, d);
+            return d;
+        };
         auto row_value = [&](int j) {            // v_j
             const float4 xv = ld_stream(x + (int64_t)j * ld4);
-            return SWAPPED ? axpy4(ngamma, ld_stream(g + (int64_t)j * ld4), xv) : xv;
+            return SWAPPED ? axpy4(ngamma, direction(j), xv) : xv;
         };
         const float4 first = row_value(0);
-        const float4 last = row_value(n - 1);
+        const float4 last = n > 1 ? row_value(n - 1) : first;   // each row's direction is formed once
         float4 prev = last, cur = first;
         constexpr int U = 4;
         int i = 0;
         for (; i + U <= n - 2; i += U) {          // rows whose lower neighbour i+1 <= n-2 comes from memory
-            float4 xn[U], gv[U];
+            float4 xn[U], gv[U], mv[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
+                const int64_t gr = (int64_t)(i + u + (SWAPPED ? 1 : 0)) * ld4;
                 xn[u] = ld_stream(x + (int64_t)(i + u + 1) * ld4);
-                gv[u] = ld_stream(g + (int64_t)(i + u + (SWAPPED ? 1 : 0)) * ld4);
+                gv[u] = ld_stream(g + gr);
+                if (MOM) mv[u] = ld_stream(vb + gr);
+            }
+            if (MOM) {
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    gv[u] = axpy4(beta, mv[u], gv[u]);
+                    st_stream(vb + (int64_t)(i + u + (SWAPPED ? 1 : 0)) * ld4, gv[u]);
+                }
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
@@ -122,7 +143,7 @@ mix_ring_x_kernel(const float4* __restrict__ X, const float4* __restrict__ G, fl
             else nx = row_value(i + 1);
             const float* w = band + 3 * i;
             float4 r = mix3(__ldg(w), prev, __ldg(w + 1), cur, __ldg(w + 2), nx);
-            if (!SWAPPED) r = axpy4(ngamma, ld_stream(g + (int64_t)i * ld4), r);
+            if (!SWAPPED) r = axpy4(ngamma, direction(i), r);
             st_stream(o + (int64_t)i * ld4, r);
             if (STATS) st.add(r);
             prev = cur;
@@ -137,10 +158,11 @@ mix_ring_x_kernel(const float4* __restrict__ X, const float4* __restrict__ G, fl
 
 // W = w 1 1^T.  Algorithm 1 order: x'_i = w sum_j x_j - gamma g_i.  Footnote c: every row becomes
 // w sum_j (x_j - gamma g_j), i.e. one centralized SGD step when w = 1/n.
-template <bool SWAPPED, bool STATS>
+template <bool SWAPPED, bool STATS, bool MOM>
 __global__ void __launch_bounds__(kThreads)
 mix_uniform_x_kernel(const float4* __restrict__ X, const float4* __restrict__ G, float4* __restrict__ Xn,
-                     int n, int64_t ld4, float w, float ngamma, double* __restrict__ partials) {
+                     float4* __restrict__ V, float beta, int n, int64_t ld4, float w, float ngamma,
+                     double* __restrict__ partials) {
     __shared__ double red[kThreads / 32];
     const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     ColumnStats st;
@@ -149,25 +171,38 @@ mix_uniform_x_kernel(const float4* __restrict__ X, const float4* __restrict__ G,
         const float4* x = X + c;
         const float4* g = G + c;
         float4* o = Xn + c;
+        float4* vb = MOM ? V + c : nullptr;
+        auto direction = [&](int j) {            // row j of G, or of the updated momentum buffers
+            const float4 gv = ld_stream(g + (int64_t)j * ld4);
+            if (!MOM) return gv;
+            const float4 d = axpy4(beta, ld_stream(vb + (int64_t)j * ld4), gv);
+            st_stream(vb + (int64_t)j * ld4, d);
+            return d;
+        };
         float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-        constexpr int U = 8;
+        constexpr int U = MOM ? 4 : 8;
         int i = 0;
         for (; i + U <= n; i += U) {
-            float4 v[U], gv[U];
+            float4 v[U], gv[U], mv[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 v[u] = ld_stream(x + (int64_t)(i + u) * ld4);
                 if (SWAPPED) gv[u] = ld_stream(g + (int64_t)(i + u) * ld4);
+                if (SWAPPED && MOM) mv[u] = ld_stream(vb + (int64_t)(i + u) * ld4);
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
+                if (SWAPPED && MOM) {
+                    gv[u] = axpy4(beta, mv[u], gv[u]);
+                    st_stream(vb + (int64_t)(i + u) * ld4, gv[u]);
+                }
                 const float4 t = SWAPPED ? axpy4(ngamma, gv[u], v[u]) : v[u];
                 s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
             }
         }
         for (; i < n; ++i) {
             float4 t = ld_stream(x + (int64_t)i * ld4);
-            if (SWAPPED) t = axpy4(ngamma, ld_stream(g + (int64_t)i * ld4), t);
+            if (SWAPPED) t = axpy4(ngamma, direction(i), t);
             s.x += t.x; s.y += t.y; s.z += t.z; s.w += t.w;
         }
         s.x *= w; s.y *= w; s.z *= w; s.w *= w;
@@ -177,18 +212,25 @@ mix_uniform_x_kernel(const float4* __restrict__ X, const float4* __restrict__ G,
         } else {
             i = 0;
             for (; i + U <= n; i += U) {
-                float4 gv[U];
-#pragma unroll
-                for (int u = 0; u < U; ++u) gv[u] = ld_stream(g + (int64_t)(i + u) * ld4);
+                float4 gv[U], mv[U];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
+                    gv[u] = ld_stream(g + (int64_t)(i + u) * ld4);
+                    if (MOM) mv[u] = ld_stream(vb + (int64_t)(i + u) * ld4);
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (MOM) {
+                        gv[u] = axpy4(beta, mv[u], gv[u]);
+                        st_stream(vb + (int64_t)(i + u) * ld4, gv[u]);
+                    }
                     const float4 r = axpy4(ngamma, gv[u], s);
                     st_stream(o + (int64_t)(i + u) * ld4, r);
                     if (STATS) st.add(r);
                 }
             }
             for (; i < n; ++i) {
-                const float4 r = axpy4(ngamma, ld_stream(g + (int64_t)i * ld4), s);
+                const float4 r = axpy4(ngamma, direction(i), s);
                 st_stream(o + (int64_t)i * ld4, r);
                 if (STATS) st.add(r);
             }
@@ -256,30 +298,58 @@ cudaError_t launch_momentum(dpsgd_ctx* c, float* V, const float* G) {
 }
 
 // stats_out != nullptr: also leave the consensus distance of X_next in *stats_out (device).
-// Returns cudaErrorNotSupported when this W has no fused-statistics kernel (the caller then runs
-// the separate consensus pass).
+// V != nullptr (ring and uniform W only): G holds the gradients, and the momentum buffers V are
+// updated in the same pass and used as the step direction.
+// Returns cudaErrorNotSupported when this W has no kernel for what is asked (the caller then runs
+// the separate passes).
+namespace {
+
+template <bool SWAPPED, bool STATS, bool MOM>
+void launch_ring_x(dpsgd_ctx* c, int grid, const float4* x4, const float4* g4, float4* o4, float4* v4) {
+    mix_ring_x_kernel<SWAPPED, STATS, MOM><<<grid, kThreads, 0, c->stream>>>(
+        x4, g4, o4, v4, c->beta, c->W.band, c->n, c->ld / 4, -c->gamma, c->d_partials);
+}
+template <bool SWAPPED, bool STATS, bool MOM>
+void launch_uniform_x(dpsgd_ctx* c, int grid, const float4* x4, const float4* g4, float4* o4, float4* v4) {
+    mix_uniform_x_kernel<SWAPPED, STATS, MOM><<<grid, kThreads, 0, c->stream>>>(
+        x4, g4, o4, v4, c->beta, c->n, c->ld / 4, c->W.uniform, -c->gamma, c->d_partials);
+}
+
+#define DPSGD_X_DISPATCH(fn, sw, st, mo, ...)                                   \
+    do {                                                                        \
+        const int key = ((sw) ? 4 : 0) | ((st) ? 2 : 0) | ((mo) ? 1 : 0);       \
+        switch (key) {                                                          \
+            case 0: fn<false, false, false>(__VA_ARGS__); break;                \
+            case 1: fn<false, false, true>(__VA_ARGS__); break;                 \
+            case 2: fn<false, true, false>(__VA_ARGS__); break;                 \
+            case 3: fn<false, true, true>(__VA_ARGS__); break;                  \
+            case 4: fn<true, false, false>(__VA_ARGS__); break;                 \
+            case 5: fn<true, false, true>(__VA_ARGS__); break;                  \
+            case 6: fn<true, true, false>(__VA_ARGS__); break;                  \
+            default: fn<true, true, true>(__VA_ARGS__); break;                  \
+        }                                                                       \
+    } while (0)
+
+}  // namespace
+
 cudaError_t launch_mix_variant(dpsgd_ctx* c, const float* X, const float* G, float* Xn, bool swapped,
-                               double* stats_out) {
+                               double* stats_out, float* V) {
     const int64_t ld4 = c->ld / 4;
     const int grid = (int)((ld4 + kThreads - 1) / kThreads);
     const float4* x4 = reinterpret_cast<const float4*>(X);
     const float4* g4 = reinterpret_cast<const float4*>(G);
     float4* o4 = reinterpret_cast<float4*>(Xn);
+    float4* v4 = reinterpret_cast<float4*>(V);
     const bool ring = c->mix_kind == DPSGD_MIX_RING, uniform = c->mix_kind == DPSGD_MIX_UNIFORM_DENSE;
-    if (stats_out && !(ring || uniform)) return cudaErrorNotSupported;
+    if ((stats_out || V) && !(ring || uniform)) return cudaErrorNotSupported;
     if (stats_out) {
         cudaError_t e = ensure_partials(c, grid);
         if (e != cudaSuccess) return e;
     }
-    double* part = c->d_partials;
     if (ring) {
-        if (swapped && stats_out) mix_ring_x_kernel<true, true><<<grid, kThreads, 0, c->stream>>>(x4, g4, o4, c->W.band, c->n, ld4, -c->gamma, part);
-        else if (swapped) mix_ring_x_kernel<true, false><<<grid, kThreads, 0, c->stream>>>(x4, g4, o4, c->W.band, c->n, ld4, -c->gamma, part);
-        else mix_ring_x_kernel<false, true><<<grid, kThreads, 0, c->stream>>>(x4, g4, o4, c->W.band, c->n, ld4, -c->gamma, part);
+        DPSGD_X_DISPATCH(launch_ring_x, swapped, stats_out != nullptr, V != nullptr, c, grid, x4, g4, o4, v4);
     } else if (uniform) {
-        if (swapped && stats_out) mix_uniform_x_kernel<true, true><<<grid, kThreads, 0, c->stream>>>(x4, g4, o4, c->n, ld4, c->W.uniform, -c->gamma, part);
-        else if (swapped) mix_uniform_x_kernel<true, false><<<grid, kThreads, 0, c->stream>>>(x4, g4, o4, c->n, ld4, c->W.uniform, -c->gamma, part);
-        else mix_uniform_x_kernel<false, true><<<grid, kThreads, 0, c->stream>>>(x4, g4, o4, c->n, ld4, c->W.uniform, -c->gamma, part);
+        DPSGD_X_DISPATCH(launch_uniform_x, swapped, stats_out != nullptr, V != nullptr, c, grid, x4, g4, o4, v4);
     } else {
         mix_gather_swapped_kernel<<<(unsigned)((ld4 + 127) / 128), 128, 0, c->stream>>>(
             x4, g4, o4, c->W.row_ptr, c->W.col, c->W.val, c->n, ld4, -c->gamma);

@@ -24,6 +24,7 @@ def main():
     ap.add_argument("--consensus", action="store_true", help="also run the consensus reduction")
     ap.add_argument("--fused", action="store_true", help="time the gossip step that also returns the consensus distance")
     ap.add_argument("--swapped", action="store_true", help="footnote c: update locally, then average")
+    ap.add_argument("--momentum", type=float, default=0.0, help="momentum of the Section 5.3 runs (one more matrix)")
     args = ap.parse_args()
 
     build.build()
@@ -38,6 +39,9 @@ def main():
         ctx.mix_kind(args.kind)
     if args.swapped:
         ctx.set_order(True)
+    if args.momentum > 0.0:
+        V = torch.zeros_like(X0)
+        ctx.set_momentum(args.momentum, V)
     out = torch.zeros(1, dtype=torch.float64, device=dev)
     step = (lambda: ctx.mix_update_consensus(out)) if args.fused else ctx.mix_update
     for _ in range(args.warmup):
@@ -52,7 +56,7 @@ def main():
     ms = a.elapsed_time(b) / max(1, args.steps)
     out = {"n": args.n, "N": args.N, "topology": args.topology,
            "kernel": binding.MIX_NAMES[ctx.mix_kind()], "ms_per_step": ms,
-           "GBps": 12.0 * args.n * args.N / (ms * 1e-3) / 1e9}
+           "GBps": (20.0 if args.momentum > 0.0 else 12.0) * args.n * args.N / (ms * 1e-3) / 1e9}
     if args.consensus:
         out["consensus"] = ctx.consensus_dist()
     print(json.dumps(out))

@@ -158,3 +158,42 @@ def test_momentum_steps_match_oracle(topo, n, N, swapped):
     f = orc.mix_update_swapped if swapped else orc.mix_update
     assert row_rel_err(run.x(), f(Xr, G, *csr, gamma)) <= TOL_STEP
     run.close()
+
+
+@pytest.mark.parametrize("swapped", [False, True])
+@pytest.mark.parametrize("topo,kind,n,N", [("ring", 0, 3, 40), ("ring", 0, 5, 1031), ("ring", 0, 6, 77),
+                                           ("ring", 0, 9, 4100), ("ring", 0, 64, 2051),
+                                           ("dense", 1, 1, 40), ("dense", 1, 2, 77), ("dense", 1, 5, 1031),
+                                           ("dense", 1, 9, 4100), ("dense", 1, 64, 2051)])
+def test_momentum_inside_the_gossip_pass(topo, kind, n, N, swapped):
+    """With the streaming kernel chosen (not the small-problem one), ring and uniform W update the
+    momentum buffers in the same pass as the gossip step; results as with separate passes."""
+    rng = np.random.default_rng(31 * n + N)
+    csr = wl.topology(topo, n)
+    X = _rand(rng, n, N)
+    gamma, beta = 0.05, 0.9
+    run = GpuRun(n, N, csr, gamma, X=X)
+    run.ctx.mix_kind(kind)
+    V0 = _rand(rng, n, N)
+    V = torch.zeros_like(run.X0)
+    V[:, :N] = torch.from_numpy(V0).cuda()
+    run.ctx.set_momentum(beta, V)
+    run.ctx.set_order(swapped)
+    Xr, Vr = X.copy(), V0.copy()
+    out = torch.zeros(1, dtype=torch.float64, device="cuda")
+    for k in range(4):
+        G = _rand(rng, n, N)
+        run.set_g(G)
+        if k % 2 == 0:
+            run.ctx.mix_update()
+        else:
+            run.ctx.mix_update_consensus(out)
+            torch.cuda.synchronize()
+        Xr, Vr = orc.mix_update_momentum(Xr, Vr, G, *csr, gamma, beta, swapped=swapped)
+        assert row_rel_err(run.x(), Xr) <= 1e-5
+        assert row_rel_err(V[:, :N].cpu().numpy(), Vr) <= 1e-5
+        if k % 2 == 1:
+            c_ref = orc.consensus_dist(Xr)
+            assert abs(float(out.item()) - c_ref) <= 1e-4 * c_ref + 1e-9
+    run.check_pads()
+    run.close()
