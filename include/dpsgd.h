@@ -149,6 +149,25 @@ DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* ctx, int32_t update_then_mix);
 DPSGD_API dpsgd_status dpsgd_local_step(dpsgd_ctx* ctx, uint64_t k);
 
 /*
+ * The same local iteration for some nodes only (Section 5.3, last paragraph: with machines of
+ * different speed, the faster ones may run more than one minibatch before the synchronisation).
+ * active_host: host, int32 [n]; node i takes the step when active_host[i] != 0, and otherwise its
+ * row of X (and of the momentum buffers) is left as it is.  The array is copied before the call
+ * returns.  n <= 65535.  Errors: DPSGD_ERR_ARG (NULL), DPSGD_ERR_STATE, DPSGD_ERR_UNSUPPORTED.
+ */
+DPSGD_API dpsgd_status dpsgd_local_step_nodes(dpsgd_ctx* ctx, uint64_t k, const int32_t* active_host);
+
+/*
+ * Per-node minibatch sizes (Section 5.3, last paragraph: different minibatch sizes compensate for
+ * machines of different speed).  batch_host: host, int32 [n], 1 <= B_i <= batch of dpsgd_set_model;
+ * node i then averages its gradient over its first B_i draws of the iteration (dpsgd_sample still
+ * returns all `batch` draws per node).  NULL restores the common size.  Synchronises the bound
+ * stream; a later dpsgd_set_model resets the sizes.  Errors: DPSGD_ERR_ARG (a size out of range),
+ * DPSGD_ERR_STATE (no model).
+ */
+DPSGD_API dpsgd_status dpsgd_set_node_batches(dpsgd_ctx* ctx, const int32_t* batch_host);
+
+/*
  * Momentum as used for both algorithms in the Torch experiments (Section 5.3: learning rate 0.1,
  * momentum 0.9).  The paper prints no formula; the reading is the heavy-ball update of the
  * framework it used, kept per node: v_i <- beta v_i + g_i, then the gossip step with v_i in place

@@ -39,6 +39,8 @@ SIGNATURES = {
     "dpsgd_step": [_vp, _u64],
     "dpsgd_run": [_vp, _u64, _i64],
     "dpsgd_local_step": [_vp, _u64],
+    "dpsgd_local_step_nodes": [_vp, _u64, _vp],
+    "dpsgd_set_node_batches": [_vp, _vp],
     "dpsgd_set_order": [_vp, _i32],
     "dpsgd_set_momentum": [_vp, _f32, _vp],
     "dpsgd_mix_update_consensus": [_vp, _vp],
@@ -194,6 +196,19 @@ class Dpsgd:
     def local_step(self, k: int):
         """Gradient step without communication (several minibatches between exchanges)."""
         self._check(self._lib.dpsgd_local_step(self._h, k))
+
+    def local_step_nodes(self, k: int, active):
+        """The local step for the nodes with a non-zero entry of `active` (length n) only."""
+        arr = (ctypes.c_int32 * self.n)(*[1 if a else 0 for a in active])
+        self._check(self._lib.dpsgd_local_step_nodes(self._h, k, arr))
+
+    def set_node_batches(self, sizes):
+        """Per-node minibatch sizes B_i <= batch (length n), or None for the common size."""
+        if sizes is None:
+            self._check(self._lib.dpsgd_set_node_batches(self._h, None))
+            return
+        arr = (ctypes.c_int32 * self.n)(*[int(b) for b in sizes])
+        self._check(self._lib.dpsgd_set_node_batches(self._h, arr))
 
     def set_order(self, update_then_mix: bool):
         """Footnote c of Algorithm 1: apply the local gradient first, then average."""

@@ -128,6 +128,8 @@ void release(dpsgd_ctx* c) {
     cudaFree(c->d_w_blob);
     cudaFree(c->d_idx);
     cudaFree(c->d_coef);
+    cudaFree(c->d_node_batch);
+    cudaFree(c->d_active);
     cudaFree(c->d_act);
     cudaFree(c->d_delta);
     cudaFree(c->d_partials);
@@ -149,11 +151,11 @@ dpsgd_status need_model(dpsgd_ctx* c) {
 }
 
 // The buffer the gossip step subtracts: the gradients, or the momentum buffers after their update.
-cudaError_t step_direction(dpsgd_ctx* c, const float** dir) {
+cudaError_t step_direction(dpsgd_ctx* c, const float** dir, const int32_t* active = nullptr) {
     *dir = c->G;
     if (!c->V) return cudaSuccess;
     *dir = c->V;
-    return launch_momentum(c, c->V, c->G);
+    return launch_momentum(c, c->V, c->G, active);
 }
 
 // Ring and uniform W have kernels that update the momentum buffers inside the gossip pass.
@@ -315,7 +317,9 @@ DPSGD_API dpsgd_status dpsgd_set_model(dpsgd_ctx* c, int32_t kind, const int32_t
     if (c->bound) cudaStreamSynchronize(c->stream);
     drop_graph(c);
     cudaFree(c->d_idx); cudaFree(c->d_coef); cudaFree(c->d_act); cudaFree(c->d_delta);
+    cudaFree(c->d_node_batch);
     c->d_idx = nullptr; c->d_coef = nullptr; c->d_act = nullptr; c->d_delta = nullptr;
+    c->d_node_batch = nullptr;             // per-node sizes belong to the model they were set for
     c->model = kind; c->d = dims[0]; c->batch = batch; c->l2 = l2_lambda; c->mlp = shape;
     c->mlp_precision = mlp_precision;
     cudaError_t e = cudaMalloc(&c->d_idx, sizeof(int32_t) * (size_t)c->n * batch);
@@ -391,15 +395,62 @@ DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* c, int32_t update_then_mix) {
     return DPSGD_OK;
 }
 
+namespace {
+dpsgd_status local_step(dpsgd_ctx* c, uint64_t k, const int32_t* active_dev) {
+    cudaError_t e = run_grad(c, k);
+    const float* D = nullptr;
+    if (e == cudaSuccess) e = step_direction(c, &D, active_dev);
+    if (e == cudaSuccess) e = launch_local_update(c, c->X[c->cur], D, active_dev);
+    return e == cudaSuccess ? DPSGD_OK : cuda_fail(c, e, "local step");
+}
+}  // namespace
+
 DPSGD_API dpsgd_status dpsgd_local_step(dpsgd_ctx* c, uint64_t k) {
     dpsgd_status s = need_bound(c);
     if (s != DPSGD_OK) return s;
     if ((s = need_model(c)) != DPSGD_OK) return s;
-    cudaError_t e = run_grad(c, k);
-    const float* D = nullptr;
-    if (e == cudaSuccess) e = step_direction(c, &D);
-    if (e == cudaSuccess) e = launch_local_update(c, c->X[c->cur], D);
-    return e == cudaSuccess ? DPSGD_OK : cuda_fail(c, e, "local step");
+    return local_step(c, k, nullptr);
+}
+
+DPSGD_API dpsgd_status dpsgd_local_step_nodes(dpsgd_ctx* c, uint64_t k, const int32_t* active_host) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    if ((s = need_model(c)) != DPSGD_OK) return s;
+    if (!active_host) return fail(c, DPSGD_ERR_ARG, "active_host is NULL");
+    if (c->n > 65535) return fail(c, DPSGD_ERR_UNSUPPORTED, "masked local steps need n <= 65535");
+    cudaError_t e = cudaSuccess;
+    if (!c->d_active) e = cudaMalloc(&c->d_active, sizeof(int32_t) * (size_t)c->n);
+    // pageable source: the copy is staged before the call returns, so the caller's array is free at once
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(c->d_active, active_host, sizeof(int32_t) * (size_t)c->n, cudaMemcpyHostToDevice,
+                            c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "dpsgd_local_step_nodes mask copy");
+    return local_step(c, k, c->d_active);
+}
+
+DPSGD_API dpsgd_status dpsgd_set_node_batches(dpsgd_ctx* c, const int32_t* batch_host) {
+    if (!c) return DPSGD_ERR_ARG;
+    if (c->model < 0) return fail(c, DPSGD_ERR_STATE, "call dpsgd_set_model before dpsgd_set_node_batches");
+    drop_graph(c);
+    cudaError_t e = cudaStreamSynchronize(c->stream);   // kernels in flight may still read the old sizes
+    if (e != cudaSuccess) return cuda_fail(c, e, "dpsgd_set_node_batches");
+    if (!batch_host) {
+        cudaFree(c->d_node_batch);
+        c->d_node_batch = nullptr;
+        return DPSGD_OK;
+    }
+    for (int i = 0; i < c->n; ++i)
+        if (batch_host[i] < 1 || batch_host[i] > c->batch)
+            return fail(c, DPSGD_ERR_ARG, "every per-node minibatch size must be in [1, batch]");
+    if (!c->d_node_batch) e = cudaMalloc(&c->d_node_batch, sizeof(int32_t) * (size_t)c->n);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(c->d_node_batch, batch_host, sizeof(int32_t) * (size_t)c->n, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        cudaFree(c->d_node_batch);
+        c->d_node_batch = nullptr;
+        return cuda_fail(c, e, "dpsgd_set_node_batches");
+    }
+    return DPSGD_OK;
 }
 
 DPSGD_API dpsgd_status dpsgd_set_momentum(dpsgd_ctx* c, float beta, float* V_dev) {

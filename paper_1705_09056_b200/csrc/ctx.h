@@ -83,6 +83,8 @@ struct dpsgd_ctx {
     // scratch (library-owned)
     int32_t* d_idx = nullptr;    // [n][B]
     float* d_coef = nullptr;     // [n][B] per-sample backward coefficients (linear models)
+    int32_t* d_node_batch = nullptr;  // [n] per-node minibatch sizes B_i <= B; NULL: every node uses B
+    int32_t* d_active = nullptr;      // [n] nodes that take part in a masked local step
     float* d_act = nullptr;      // MLP activations h_0..h_L  (see grad_mlp.cu for the layout)
     float* d_delta = nullptr;    // MLP back-propagated errors
     size_t act_floats = 0, delta_floats = 0;
@@ -119,8 +121,9 @@ void mix_tiled_release(dpsgd_ctx* c);
 cudaError_t launch_consensus(dpsgd_ctx* c, const float* X, double* result_dev);
 cudaError_t ensure_partials(dpsgd_ctx* c, int count);
 cudaError_t launch_consensus_final(dpsgd_ctx* c, int count, double* result_dev);
-cudaError_t launch_momentum(dpsgd_ctx* c, float* V, const float* G);
-cudaError_t launch_local_update(dpsgd_ctx* c, float* X, const float* D);
+// active: device [n], rows with 0 are left untouched; NULL: every row.
+cudaError_t launch_momentum(dpsgd_ctx* c, float* V, const float* G, const int32_t* active);
+cudaError_t launch_local_update(dpsgd_ctx* c, float* X, const float* D, const int32_t* active);
 cudaError_t launch_mix_variant(dpsgd_ctx* c, const float* X, const float* G, float* Xn, bool swapped,
                                double* stats_out, float* V);
 cudaError_t launch_average(dpsgd_ctx* c, const float* X, float* xbar);

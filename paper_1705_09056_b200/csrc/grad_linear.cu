@@ -30,12 +30,17 @@ __global__ void __launch_bounds__(kFwdThreads)
 glm_forward_kernel(const float* __restrict__ X, int64_t ld, const float* __restrict__ A,
                    const float* __restrict__ y, int64_t m, int d, int B, int n, uint64_t seed,
                    uint64_t k, const uint64_t* __restrict__ k_ptr, int model, int32_t* __restrict__ idx,
-                   float* __restrict__ coef) {
+                   float* __restrict__ coef, const int32_t* __restrict__ node_batch) {
     __shared__ float part[kFwdThreads / 32];
     const int w = blockIdx.x;
     const int node = w / B, b = w - node * B;
     if (k_ptr) k = *k_ptr;        // iteration counter kept on the device (graph replay)
     const int32_t j = sample_index(seed, k, (uint32_t)node, (uint32_t)b, (uint32_t)m);
+    const int Bi = node_batch ? __ldg(node_batch + node) : B;   // this node's minibatch size
+    if (b >= Bi) {                // draw beyond this node's minibatch: recorded, not used
+        if (threadIdx.x == 0) { idx[w] = j; coef[w] = 0.f; }
+        return;
+    }
     const float* row = A + ((int64_t)node * m + j) * d;
     const float* x = X + (int64_t)node * ld;
     float acc = 0.f;
@@ -72,11 +77,11 @@ glm_forward_kernel(const float* __restrict__ X, int64_t ld, const float* __restr
         const float yv = __ldg(y + (int64_t)node * m + j);
         float cf;
         if (model == DPSGD_MODEL_LSQ) {
-            cf = (dot - yv) / (float)B;
+            cf = (dot - yv) / (float)Bi;
         } else {
             const float z = dot + __ldg(x + d);
             const float s = 1.f / (1.f + expf(yv * z));
-            cf = -yv * s / (float)B;
+            cf = -yv * s / (float)Bi;
         }
         idx[w] = j;
         coef[w] = cf;
@@ -88,9 +93,11 @@ template <int VEC>
 __global__ void __launch_bounds__(256)
 glm_backward_kernel(const float* __restrict__ X, float* __restrict__ G, int64_t ld,
                     const float* __restrict__ A, int64_t m, int d, int B, int model, float l2,
-                    const int32_t* __restrict__ idx, const float* __restrict__ coef) {
+                    const int32_t* __restrict__ idx, const float* __restrict__ coef,
+                    const int32_t* __restrict__ node_batch) {
     __shared__ float red[8][32][VEC];
     const int node = blockIdx.y;
+    const int Bi = node_batch ? __ldg(node_batch + node) : B;
     const int tx = threadIdx.x, ty = threadIdx.y;
     const int col = (blockIdx.x * 32 + tx) * VEC;       // first of VEC columns
     const bool live = col < d;
@@ -102,7 +109,7 @@ glm_backward_kernel(const float* __restrict__ X, float* __restrict__ G, int64_t 
     if (live) {
         const float* base = A + (int64_t)node * m * d + col;
 #pragma unroll 8
-        for (int b = ty; b < B; b += 8) {
+        for (int b = ty; b < Bi; b += 8) {
             const float w = __ldg(cf + b);
             const float* row = base + (int64_t)__ldg(ix + b) * d;
             if (VEC == 4) {
@@ -134,7 +141,7 @@ glm_backward_kernel(const float* __restrict__ X, float* __restrict__ G, int64_t 
         for (int64_t c = d + tx; c < ld; c += 32) {
             float s = 0.f;
             if (model == DPSGD_MODEL_LOGISTIC && c == d)
-                for (int b = 0; b < B; ++b) s += __ldg(cf + b);
+                for (int b = 0; b < Bi; ++b) s += __ldg(cf + b);
             G[(int64_t)node * ld + c] = s;
         }
     }
@@ -149,18 +156,20 @@ cudaError_t launch_grad_linear(dpsgd_ctx* c, uint64_t k, const float* X, float* 
     const bool vec = (d % 4 == 0);
     if (vec)
         glm_forward_kernel<4><<<fwd_grid, kFwdThreads, 0, c->stream>>>(
-            X, c->ld, c->A, y, c->m, d, B, n, c->seed, k, c->k_dev_active, c->model, c->d_idx, c->d_coef);
+            X, c->ld, c->A, y, c->m, d, B, n, c->seed, k, c->k_dev_active, c->model, c->d_idx, c->d_coef,
+            c->d_node_batch);
     else
         glm_forward_kernel<1><<<fwd_grid, kFwdThreads, 0, c->stream>>>(
-            X, c->ld, c->A, y, c->m, d, B, n, c->seed, k, c->k_dev_active, c->model, c->d_idx, c->d_coef);
+            X, c->ld, c->A, y, c->m, d, B, n, c->seed, k, c->k_dev_active, c->model, c->d_idx, c->d_coef,
+            c->d_node_batch);
     const int vw = vec ? 4 : 1;
     dim3 grid((d + 32 * vw - 1) / (32 * vw), n), block(32, 8);
     if (vec)
         glm_backward_kernel<4><<<grid, block, 0, c->stream>>>(X, G, c->ld, c->A, c->m, d, B, c->model,
-                                                              c->l2, c->d_idx, c->d_coef);
+                                                              c->l2, c->d_idx, c->d_coef, c->d_node_batch);
     else
         glm_backward_kernel<1><<<grid, block, 0, c->stream>>>(X, G, c->ld, c->A, c->m, d, B, c->model,
-                                                              c->l2, c->d_idx, c->d_coef);
+                                                              c->l2, c->d_idx, c->d_coef, c->d_node_batch);
     c->launches += 2;
     return cudaGetLastError();
 }

@@ -135,14 +135,22 @@ bgemm_kernel(GemmArgs g) {
     }
 }
 
-// delta_L[b][:] = (softmax(logits[b]) - onehot(y[idx[b]])) / B; one warp per (node, sample).
+// delta_L[b][:] = (softmax(logits[b]) - onehot(y[idx[b]])) / B_i; one warp per (node, sample).
+// Columns b >= B_i (a node with a smaller minibatch) get delta = 0 and so drop out of every
+// product of the backward pass.
 __global__ void __launch_bounds__(128)
 softmax_ce_delta_kernel(const float* __restrict__ logits, const int32_t* __restrict__ y, int64_t m,
-                        const int32_t* __restrict__ idx, int n, int B, int C, float* __restrict__ delta) {
+                        const int32_t* __restrict__ idx, int n, int B, int C, float* __restrict__ delta,
+                        const int32_t* __restrict__ node_batch) {
     const int w = blockIdx.x * 4 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (w >= n * B) return;
     const int node = w / B;
+    const int Bi = node_batch ? __ldg(node_batch + node) : B;
+    if (w - node * B >= Bi) {
+        for (int c = lane; c < C; c += 32) delta[(int64_t)w * C + c] = 0.f;
+        return;
+    }
     const float* z = logits + (int64_t)w * C;
     float mx = -INFINITY;
     for (int c = lane; c < C; c += 32) mx = fmaxf(mx, z[c]);
@@ -153,7 +161,7 @@ softmax_ce_delta_kernel(const float* __restrict__ logits, const int32_t* __restr
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     const int label = __ldg(y + (int64_t)node * m + __ldg(idx + w));
-    const float inv = 1.f / s, invB = 1.f / (float)B;
+    const float inv = 1.f / s, invB = 1.f / (float)Bi;
     for (int c = lane; c < C; c += 32)
         delta[(int64_t)w * C + c] = (expf(z[c] - mx) * inv - (c == label ? 1.f : 0.f)) * invB;
 }
@@ -294,7 +302,8 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) 
     }
 
     softmax_ce_delta_kernel<<<(n * B + 3) / 4, 128, 0, c->stream>>>(
-        c->d_act + p.act_off[L], y, c->m, c->d_idx, n, B, s.dims[L], c->d_delta + p.delta_off[L]);
+        c->d_act + p.act_off[L], y, c->m, c->d_idx, n, B, s.dims[L], c->d_delta + p.delta_off[L],
+        c->d_node_batch);
     c->launches++;
 
     // backward

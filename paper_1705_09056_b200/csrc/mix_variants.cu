@@ -263,36 +263,46 @@ mix_gather_swapped_kernel(const float4* __restrict__ X, const float4* __restrict
     }
 }
 
-// Momentum buffer of the Torch experiments (Section 5.3): V <- beta V + G, in place.
+// Momentum buffer of the Torch experiments (Section 5.3): V <- beta V + G, in place.  blockIdx.y is
+// the node; a node whose entry of `active` is zero keeps its buffer.
 __global__ void __launch_bounds__(kThreads)
-momentum_kernel(float4* __restrict__ V, const float4* __restrict__ G, int64_t total4, float beta) {
-    const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    if (t >= total4) return;
+momentum_kernel(float4* __restrict__ V, const float4* __restrict__ G, int64_t ld4, float beta,
+                const int32_t* __restrict__ active) {
+    const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (c >= ld4 || (active && __ldg(active + blockIdx.y) == 0)) return;
+    const int64_t t = (int64_t)blockIdx.y * ld4 + c;
     st_stream(V + t, axpy4(beta, ld_stream(V + t), ld_stream(G + t)));
 }
 
-// Local SGD step without communication: X <- X - gamma D, in place (W = I).
+// Local SGD step without communication: X <- X - gamma D, in place (W = I), for the active nodes.
 __global__ void __launch_bounds__(kThreads)
-local_update_kernel(float4* __restrict__ X, const float4* __restrict__ D, int64_t total4, float ngamma) {
-    const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-    if (t >= total4) return;
+local_update_kernel(float4* __restrict__ X, const float4* __restrict__ D, int64_t ld4, float ngamma,
+                    const int32_t* __restrict__ active) {
+    const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (c >= ld4 || (active && __ldg(active + blockIdx.y) == 0)) return;
+    const int64_t t = (int64_t)blockIdx.y * ld4 + c;
     st_stream(X + t, axpy4(ngamma, ld_stream(D + t), ld_stream(X + t)));
 }
 
 }  // namespace
 
-cudaError_t launch_local_update(dpsgd_ctx* c, float* X, const float* D) {
-    const int64_t total4 = (int64_t)c->n * c->ld / 4;
-    local_update_kernel<<<(unsigned)((total4 + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(
-        reinterpret_cast<float4*>(X), reinterpret_cast<const float4*>(D), total4, -c->gamma);
+// Grids of (column blocks, node): gridDim.y <= 65535 bounds n here.
+cudaError_t launch_local_update(dpsgd_ctx* c, float* X, const float* D, const int32_t* active) {
+    if (c->n > 65535) return cudaErrorInvalidConfiguration;
+    const int64_t ld4 = c->ld / 4;
+    const dim3 grid((unsigned)((ld4 + kThreads - 1) / kThreads), (unsigned)c->n);
+    local_update_kernel<<<grid, kThreads, 0, c->stream>>>(
+        reinterpret_cast<float4*>(X), reinterpret_cast<const float4*>(D), ld4, -c->gamma, active);
     c->launches++;
     return cudaGetLastError();
 }
 
-cudaError_t launch_momentum(dpsgd_ctx* c, float* V, const float* G) {
-    const int64_t total4 = (int64_t)c->n * c->ld / 4;
-    momentum_kernel<<<(unsigned)((total4 + kThreads - 1) / kThreads), kThreads, 0, c->stream>>>(
-        reinterpret_cast<float4*>(V), reinterpret_cast<const float4*>(G), total4, c->beta);
+cudaError_t launch_momentum(dpsgd_ctx* c, float* V, const float* G, const int32_t* active) {
+    if (c->n > 65535) return cudaErrorInvalidConfiguration;
+    const int64_t ld4 = c->ld / 4;
+    const dim3 grid((unsigned)((ld4 + kThreads - 1) / kThreads), (unsigned)c->n);
+    momentum_kernel<<<grid, kThreads, 0, c->stream>>>(
+        reinterpret_cast<float4*>(V), reinterpret_cast<const float4*>(G), ld4, c->beta, active);
     c->launches++;
     return cudaGetLastError();
 }
