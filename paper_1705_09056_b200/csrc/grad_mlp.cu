@@ -12,9 +12,13 @@
 // tensor cores (tc_gemm.cuh: tcgen05 TF32 MMAs, three per product for fp32-faithful results) when
 // the minibatch fits a 128-column tile, and otherwise - or when asked - on the fp32 FMA kernel
 // below (exact fp32 products, fp32 accumulation in a fixed order).
+#include <algorithm>
+
 #include "ctx.h"
 #include "philox.cuh"
 #include "tc_gemm.cuh"
+#include "tc_stream.cuh"
+#include "tma_host.h"
 
 namespace dpsgd {
 namespace {
@@ -254,6 +258,86 @@ cudaError_t run_tc(dpsgd_ctx* c, tc::Args a, int max_tile) {
     return launch_tc_nt<8, false>(c, a, (a.N + 127) / 128);
 }
 
+// ---- weight-streaming kernel (tc_stream.cuh): forward and input-gradient products ----
+
+template <int NT, bool A_K, bool PRECISE>
+cudaError_t launch_tcs_inst(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap& mapB, const tcs::Args& a) {
+    auto kernel = tcs::tc_stream_kernel<NT, A_K, PRECISE>;
+    constexpr size_t smem = tcs::smem_bytes<NT, PRECISE>();
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                  cudaSharedmemCarveoutMaxShared)) != cudaSuccess) return e;
+    int sms = 0, dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    const int per_sm = NT <= 4 ? 2 : 1;                          // what the kernel's shared memory allows
+    const int grid = std::min(a.total_tiles, sms * per_sm);      // persistent CTAs
+    kernel<<<grid, tcs::kThreads, smem, c->stream>>>(mapA, mapB, a);
+    c->launches++;
+    return cudaGetLastError();
+}
+
+template <int NT>
+cudaError_t launch_tcs_nt(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap& mapB, const tcs::Args& a,
+                          bool a_kcontig, bool precise) {
+    if (a_kcontig) return precise ? launch_tcs_inst<NT, true, true>(c, mapA, mapB, a)
+                                  : launch_tcs_inst<NT, true, false>(c, mapA, mapB, a);
+    return precise ? launch_tcs_inst<NT, false, true>(c, mapA, mapB, a)
+                   : launch_tcs_inst<NT, false, false>(c, mapA, mapB, a);
+}
+
+// The TMA loads need 16-byte aligned bases and strides, B contiguous along k and one column tile
+// for the whole minibatch.
+bool stream_ok(const tc::Args& a) {
+    auto al = [](const float* p, int64_t pitch, int64_t node) {
+        return reinterpret_cast<uintptr_t>(p) % 16 == 0 && pitch % 4 == 0 && node % 4 == 0;
+    };
+    return a.b_kcontig && a.N <= 128 && al(a.A, a.a_pitch, a.a_node) && al(a.B, a.b_pitch, a.b_node);
+}
+
+// Returns cudaErrorNotSupported when the tensor maps cannot be built (the caller falls back).
+cudaError_t run_tcs(dpsgd_ctx* c, const tc::Args& t) {
+    const int rows_b = t.N <= 16 ? 16 : (t.N <= 32 ? 32 : (t.N <= 64 ? 64 : 128));
+    CUtensorMap mapA, mapB;
+    const uint64_t nodes = (uint64_t)c->n;
+    bool ok;
+    if (t.a_kcontig)     // A(m,k) at m*pitch + k
+        ok = make_map_3d(&mapA, t.A, (uint64_t)t.K, (uint64_t)t.M, nodes, (uint64_t)t.a_pitch * 4,
+                         (uint64_t)t.a_node * 4, tcs::kBK, tcs::kTileM, true);
+    else                 // A(m,k) at k*pitch + m
+        ok = make_map_3d(&mapA, t.A, (uint64_t)t.M, (uint64_t)t.K, nodes, (uint64_t)t.a_pitch * 4,
+                         (uint64_t)t.a_node * 4, tcs::kTileM, tcs::kBK, false);
+    ok = ok && make_map_3d(&mapB, t.B, (uint64_t)t.K, (uint64_t)t.N, nodes, (uint64_t)t.b_pitch * 4,
+                           (uint64_t)t.b_node * 4, tcs::kBK, (uint32_t)rows_b, true);
+    if (!ok) return cudaErrorNotSupported;
+    tcs::Args a{};
+    a.C = t.C; a.c_node = t.c_node; a.c_pitch = t.c_pitch;
+    a.aux = t.aux; a.aux_node = t.aux_node; a.aux_pitch = t.aux_pitch;
+    a.M = t.M; a.N = t.N; a.K = t.K;
+    a.m_tiles = (t.M + tcs::kTileM - 1) / tcs::kTileM;
+    a.total_tiles = a.m_tiles * c->n;
+    a.epi = t.epi;
+    a.status = &c->d_result->status;
+    const bool precise = c->mlp_precision == 0;
+    switch (rows_b) {
+        case 16: return launch_tcs_nt<1>(c, mapA, mapB, a, t.a_kcontig != 0, precise);
+        case 32: return launch_tcs_nt<2>(c, mapA, mapB, a, t.a_kcontig != 0, precise);
+        case 64: return launch_tcs_nt<4>(c, mapA, mapB, a, t.a_kcontig != 0, precise);
+        default: return launch_tcs_nt<8>(c, mapA, mapB, a, t.a_kcontig != 0, precise);
+    }
+}
+
+// Forward / input-gradient product: the streaming kernel when its loads are legal, else the
+// register-staged one.
+cudaError_t run_tc_weights(dpsgd_ctx* c, const tc::Args& a) {
+    if (stream_ok(a)) {
+        const cudaError_t e = run_tcs(c, a);
+        if (e != cudaErrorNotSupported) return e;
+    }
+    return run_tc(c, a, 128);
+}
+
 }  // namespace
 
 size_t mlp_act_floats(const dpsgd_ctx* c) {
@@ -295,7 +379,7 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) 
             a.C = g.C; a.c_node = g.c_node; a.c_pitch = dout;
             a.aux = g.aux; a.aux_node = g.aux_node; a.aux_pitch = 0;
             a.M = dout; a.N = B; a.K = din; a.epi = l < L ? tc::EPI_BIAS_RELU : tc::EPI_BIAS;
-            cudaError_t e = run_tc(c, a, 128);
+            cudaError_t e = run_tc_weights(c, a);
             if (e != cudaSuccess) return e;
         } else if (l < L) run_gemm<true, true, EPI_BIAS_RELU>(c, g);
         else run_gemm<true, true, EPI_BIAS>(c, g);
@@ -343,7 +427,7 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) 
                 a.C = g.C; a.c_node = g.c_node; a.c_pitch = din;
                 a.aux = g.aux; a.aux_node = g.aux_node; a.aux_pitch = din;
                 a.M = din; a.N = B; a.K = dout; a.epi = tc::EPI_MASK;
-                cudaError_t e = run_tc(c, a, 128);
+                cudaError_t e = run_tc_weights(c, a);
                 if (e != cudaSuccess) return e;
             } else run_gemm<true, false, EPI_MASK>(c, g);
         }

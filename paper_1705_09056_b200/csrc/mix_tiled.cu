@@ -19,6 +19,7 @@
 #include <vector>
 
 #include "ctx.h"
+#include "tma_host.h"
 
 namespace dpsgd {
 namespace {
@@ -208,25 +209,8 @@ mix_tiled_kernel(const __grid_constant__ CUtensorMap mapX, const float4* __restr
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (fn) return fn;
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-        return nullptr;
-    fn = reinterpret_cast<EncodeTiledFn>(p);
-    return fn;
-}
-
 bool make_map(CUtensorMap* map, const float* base, int n, int64_t ld, int T) {
-    EncodeTiledFn enc = encode_fn();
+    EncodeTiledFn enc = tensor_map_encoder();
     if (!enc) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)ld, (cuuint64_t)n};
     const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
