@@ -18,6 +18,7 @@
 #include "philox.cuh"
 #include "tc_gemm.cuh"
 #include "tc_stream.cuh"
+#include "tc_wgrad.cuh"
 #include "tma_host.h"
 
 namespace dpsgd {
@@ -328,6 +329,61 @@ cudaError_t run_tcs(dpsgd_ctx* c, const tc::Args& t) {
     }
 }
 
+// ---- weight-gradient kernel (tc_wgrad.cuh) ----
+
+template <int NT, bool PRECISE>
+cudaError_t launch_tcw_inst(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap& mapB, const CUtensorMap& mapC,
+                            tcw::Args a) {
+    auto kernel = tcw::tc_wgrad_kernel<NT, PRECISE>;
+    constexpr size_t smem = tcw::smem_bytes<NT, PRECISE>();
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int sms = 0, dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    // items = (node, 128-row block, run of column tiles): enough of them to balance the persistent CTAs
+    const long long blocks = (long long)c->n * a.m_tiles;
+    int chunks = (int)std::min<long long>(a.n_tiles, std::max<long long>(1, (12LL * sms + blocks - 1) / blocks));
+    a.chunk = (a.n_tiles + chunks - 1) / chunks;
+    a.chunks = (a.n_tiles + a.chunk - 1) / a.chunk;
+    a.total_items = (int)(blocks * a.chunks);
+    const int grid = std::min(a.total_items, sms);               // one persistent CTA per SM
+    kernel<<<grid, tcw::kThreads, smem, c->stream>>>(mapA, mapB, mapC, a);
+    c->launches++;
+    return cudaGetLastError();
+}
+
+// gW[o][k'] = sum_b delta[b][o] h[b][k'] for every node.  Returns cudaErrorNotSupported when the
+// shapes or alignments rule the TMA path out (the caller falls back).
+cudaError_t run_tcw(dpsgd_ctx* c, const float* h, int din, const float* delta, int dout, float* gW) {
+    const int B = c->batch;
+    auto al = [](const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; };
+    if (B > tcw::kMaxK || din % 4 != 0 || dout % 4 != 0 || !al(h) || !al(delta) || !al(gW) || c->ld % 4 != 0 ||
+        ((int64_t)B * din) % 4 != 0 || ((int64_t)B * dout) % 4 != 0)
+        return cudaErrorNotSupported;
+    const int rows_b = dout <= 16 ? 16 : (dout <= 32 ? 32 : 64);
+    const uint64_t nodes = (uint64_t)c->n;
+    CUtensorMap mapA, mapB, mapC;
+    bool ok = make_map_3d(&mapA, h, (uint64_t)din, (uint64_t)B, nodes, (uint64_t)din * 4, (uint64_t)B * din * 4,
+                          tcw::kTileM, tcw::kMaxK, false);
+    ok = ok && make_map_3d(&mapB, delta, (uint64_t)dout, (uint64_t)B, nodes, (uint64_t)dout * 4,
+                           (uint64_t)B * dout * 4, (uint32_t)rows_b, tcw::kMaxK, false);
+    ok = ok && make_map_3d(&mapC, gW, (uint64_t)din, (uint64_t)dout, nodes, (uint64_t)din * 4, (uint64_t)c->ld * 4,
+                           tcw::kTileM, (uint32_t)rows_b, false);
+    if (!ok) return cudaErrorNotSupported;
+    tcw::Args a{};
+    a.M = din; a.N = dout; a.K = B;
+    a.m_tiles = (din + tcw::kTileM - 1) / tcw::kTileM;
+    a.n_tiles = (dout + rows_b - 1) / rows_b;
+    a.status = &c->d_result->status;
+    const bool precise = c->mlp_precision == 0;
+    switch (rows_b) {
+        case 16: return precise ? launch_tcw_inst<1, true>(c, mapA, mapB, mapC, a) : launch_tcw_inst<1, false>(c, mapA, mapB, mapC, a);
+        case 32: return precise ? launch_tcw_inst<2, true>(c, mapA, mapB, mapC, a) : launch_tcw_inst<2, false>(c, mapA, mapB, mapC, a);
+        default: return precise ? launch_tcw_inst<4, true>(c, mapA, mapB, mapC, a) : launch_tcw_inst<4, false>(c, mapA, mapB, mapC, a);
+    }
+}
+
 // Forward / input-gradient product: the streaming kernel when its loads are legal, else the
 // register-staged one.
 cudaError_t run_tc_weights(dpsgd_ctx* c, const tc::Args& a) {
@@ -406,7 +462,8 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) 
                 a.B = delta; a.b_node = (int64_t)B * dout; a.b_pitch = dout; a.b_kcontig = 0;
                 a.C = g.C; a.c_node = c->ld; a.c_pitch = din;
                 a.M = din; a.N = dout; a.K = B; a.epi = tc::EPI_STORE;
-                cudaError_t e = run_tc(c, a, 64);
+                cudaError_t e = run_tcw(c, g.Bm, din, delta, dout, g.C);
+                if (e == cudaErrorNotSupported) e = run_tc(c, a, 64);
                 if (e != cudaSuccess) return e;
             } else run_gemm<false, false, EPI_STORE>(c, g);
         }

@@ -1,0 +1,311 @@
+// Weight-gradient product of the MLP (Algorithm 1 step 3), batched over the nodes:
+//
+//     gW[o][k'] = sum_b delta[b][o] * h[b][k']          K = minibatch <= 64, output din x dout per node
+//
+// i.e. C[n][m] = sum_k A(m,k) B(n,k) with m = k' (input unit), n = o (output unit), k = b, both
+// operands contiguous along their row index in memory (h is [b][k'], delta is [b][o]).  The product
+// is bound by WRITING the gradient (one pass over G), so the kernel is built around the output:
+//
+//   TMA warp        loads the raw h tile of a work item ([k][128 m], once per item) and, per column
+//                   tile, the raw delta tile ([k][N]) into a ring of stages.
+//   converter warps (4) split values into TF32 head and remainder (three MMAs per product, as in
+//                   tc_gemm.cuh).  The h tile goes to TENSOR MEMORY once per item (thread t owns row
+//                   t: column t of the raw tile, which transposes it) and serves every column tile
+//                   of the item; delta tiles go to shared memory in the K-major no-swizzle layout
+//                   (element (r,k) at (k/4)*LBO + (r/8)*128 + (r%8)*16 + (k%4)*4), double-buffered.
+//   MMA warp        one thread issues the MMAs of a column tile into one of two accumulators.
+//   epilogue warps  (4) read a finished accumulator with tcgen05.ld, lay it out in shared memory as
+//                   [n][128 m] and hand it to a TMA store (cp.async.bulk.tensor, shared -> global),
+//                   which writes whole lines asynchronously and clips at the matrix edge; two
+//                   staging buffers, so the store of one tile overlaps the next.
+//
+// One persistent CTA per SM; a work item is (node, 128-row block of m, run of column tiles).  Every
+// mbarrier wait is bounded; a wait that runs out raises the status word, the TMA thread waits
+// (bounded) for its loads in flight, outstanding stores are drained, and the CTA frees its TMEM
+// columns before it returns.
+#pragma once
+#include "tc_stream.cuh"
+
+namespace dpsgd {
+namespace tcw {
+
+using tc::mbar_arrive;
+using tc::mbar_init;
+using tc::mbar_wait;
+using tc::smem_u32;
+using tcs::lds32;
+using tcs::mbar_expect_tx;
+using tcs::tma_load_3d;
+
+constexpr int kThreads = 320;        // 4 epilogue warps, 4 converter warps, MMA warp, TMA warp
+constexpr int kTileM = 128;
+constexpr int kMaxK = 64;            // minibatch rows a raw tile holds
+constexpr int kStagesB = 3;
+constexpr uint32_t kAccStride = 64;  // TMEM columns per accumulator
+constexpr uint32_t kACols = 2 * kMaxK;   // heads, then remainders
+
+struct Args {
+    int M, N, K;                     // din, dout, minibatch
+    int m_tiles, n_tiles, chunk, chunks;   // column tiles per item, items per (node, m block)
+    int total_items;
+    int* status;
+};
+
+__host__ __device__ constexpr uint32_t a_raw_bytes() { return kMaxK * kTileM * 4; }
+__host__ __device__ constexpr uint32_t b_raw_bytes(int rows) { return (uint32_t)kMaxK * rows * 4; }
+__host__ __device__ constexpr uint32_t b_lbo(int rows) { return (uint32_t)rows * 16; }
+__host__ __device__ constexpr uint32_t b_conv_bytes(int rows) { return (kMaxK / 4) * b_lbo(rows); }
+__host__ __device__ constexpr uint32_t stage_bytes(int rows) { return (uint32_t)rows * kTileM * 4; }
+
+template <int NT, bool PRECISE>
+constexpr size_t smem_bytes() {
+    return 1024 + a_raw_bytes() + kStagesB * b_raw_bytes(16 * NT) + 2 * (PRECISE ? 2 : 1) * b_conv_bytes(16 * NT) +
+           2 * stage_bytes(16 * NT) + 256;
+}
+
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
+}
+__device__ __forceinline__ void sts32(uint32_t addr, float v) {
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+
+struct Item { int node, m0, t0, t1; };
+__device__ __forceinline__ Item decode(const Args& g, int item) {
+    const int per_node = g.m_tiles * g.chunks;
+    Item w;
+    w.node = item / per_node;
+    const int rem = item - w.node * per_node;
+    const int mt = rem / g.chunks, ch = rem - mt * g.chunks;
+    w.m0 = mt * kTileM;
+    w.t0 = ch * g.chunk;
+    w.t1 = min(g.n_tiles, w.t0 + g.chunk);
+    return w;
+}
+
+// NT = column tile / 16 (16, 32 or 64 output units per tile); PRECISE: three split MMAs per product.
+// mapA: h as (m, k, node), box 128 x 64.  mapB: delta as (n, k, node), box 16 NT x 64.  mapC: the
+// gradient block as (m, n, node), box 128 x 16 NT.
+//
+// Tensor memory columns: [0, 128) two accumulators, then two converted h tiles of 64 heads +
+// 64 remainders each.
+template <int NT, bool PRECISE>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                const __grid_constant__ CUtensorMap mapC, Args g) {
+    constexpr int ROWS_B = 16 * NT;
+    constexpr uint32_t A_RAW = a_raw_bytes(), B_RAW = b_raw_bytes(ROWS_B);
+    constexpr uint32_t B_CONV = b_conv_bytes(ROWS_B), B_LBO = b_lbo(ROWS_B), SBO = 128;
+    constexpr uint32_t NCOPY = PRECISE ? 2 : 1;
+    constexpr uint32_t CONV_BUF = NCOPY * B_CONV;
+    constexpr uint32_t STAGE = stage_bytes(ROWS_B);
+    constexpr uint32_t A_COL0 = 2 * kAccStride;
+    constexpr uint32_t TMEM_COLS = 512;
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t a_raw = base;
+    const uint32_t b_raw = a_raw + A_RAW;
+    const uint32_t b_conv = b_raw + kStagesB * B_RAW;
+    const uint32_t stage = b_conv + 2 * CONV_BUF;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + A_RAW + kStagesB * B_RAW + 2 * CONV_BUF + 2 * STAGE);
+    uint64_t* a_raw_full = bars;                 // 1
+    uint64_t* a_raw_empty = bars + 1;            // 1
+    uint64_t* a_conv_full = bars + 2;            // [2]
+    uint64_t* a_conv_empty = bars + 4;           // [2]
+    uint64_t* b_raw_full = bars + 6;             // [kStagesB]
+    uint64_t* b_raw_empty = b_raw_full + kStagesB;
+    uint64_t* b_conv_full = b_raw_empty + kStagesB;   // [2]
+    uint64_t* b_conv_empty = b_conv_full + 2;    // [2]
+    uint64_t* acc_full = b_conv_empty + 2;       // [2]
+    uint64_t* acc_empty = acc_full + 2;          // [2]
+    uint64_t* stage_free = acc_empty + 2;        // [2] the TMA store that last read the buffer is done reading
+    uint64_t* stage_ready = stage_free + 2;      // [2] all epilogue threads have written the buffer
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(stage_ready + 2);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int KS = (g.K + 7) / 8;                // MMAs (k = 8) per product and column tile
+
+    if (tid == 0) {
+        mbar_init(a_raw_full, 1); mbar_init(a_raw_empty, 128);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(a_conv_full + b, 128); mbar_init(a_conv_empty + b, 1);
+            mbar_init(b_conv_full + b, 128); mbar_init(b_conv_empty + b, 1);
+            mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, 128);
+            mbar_init(stage_free + b, 1); mbar_init(stage_ready + b, 128);
+        }
+        for (int s = 0; s < kStagesB; ++s) { mbar_init(b_raw_full + s, 1); mbar_init(b_raw_empty + s, 128); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 8) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    bool ok = true;
+
+    if (warp < 4) {
+        // ------------------------------ epilogue: TMEM -> shared memory -> TMA store ------------------------------
+        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+        uint32_t q = 0;
+        for (int item = blockIdx.x; item < g.total_items && ok; item += gridDim.x) {
+            const Item w = decode(g, item);
+            for (int t = w.t0; t < w.t1; ++t, ++q) {
+                const uint32_t ab = q & 1u, ph = (q >> 1) & 1u;
+                const uint32_t st = stage + ab * STAGE;
+                if (tid == 0) {     // the store issued two tiles ago has finished reading this staging buffer
+                    asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    mbar_arrive(stage_free + ab);
+                }
+                const bool go = mbar_wait(acc_full + ab, ph) && mbar_wait(stage_free + ab, ph);
+                if (!__all_sync(0xffffffffu, go)) { ok = false; break; }     // tcgen05.ld needs the whole warp
+                tc::tc_fence_after();
+#pragma unroll 1
+                for (int c0 = 0; c0 < ROWS_B; c0 += 16) {
+                    float v[16];
+                    tc::tmem_ld16(lane_base + ab * kAccStride + (uint32_t)c0, v);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) sts32(st + (uint32_t)(c0 + j) * (kTileM * 4) + (uint32_t)tid * 4, v[j]);
+                }
+                tc::tc_fence_before();
+                mbar_arrive(acc_empty + ab);                                 // the accumulator may be overwritten
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(stage_ready + ab);
+                if (tid == 0) {
+                    if (mbar_wait(stage_ready + ab, ph)) {
+                        tma_store_3d(&mapC, st, w.m0, t * ROWS_B, w.node);
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    } else {
+                        atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);     // tile not stored; the others run into their own limits
+                    }
+                }
+            }
+        }
+        if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores complete before exit
+        if (!ok && lane == 0) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
+    } else if (warp < 8) {
+        // ------------------------------ converters ------------------------------
+        const uint32_t ct = (uint32_t)tid - 128u, cw = (uint32_t)warp - 4u;
+        const uint32_t lane_base = tmem_base + ((cw * 32u) << 16);
+        uint32_t q = 0, it = 0;
+        for (int item = blockIdx.x; item < g.total_items && ok; item += gridDim.x, ++it) {
+            const Item w = decode(g, item);
+            const uint32_t abuf = it & 1u;
+            {   // h tile -> tensor memory: row ct of A is column ct of the raw [k][m] tile
+                const bool go = mbar_wait(a_raw_full, it & 1u) && mbar_wait(a_conv_empty + abuf, ((it >> 1) & 1u) ^ 1u);
+                if (!__all_sync(0xffffffffu, go)) { ok = false; break; }     // tcgen05.st needs the whole warp
+                tc::tc_fence_after();
+                const uint32_t a_cols = lane_base + A_COL0 + abuf * kACols;
+#pragma unroll 1
+                for (int k0 = 0; k0 < g.K; k0 += 16) {
+                    uint32_t hi[16], lo[16];
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        const float v = lds32(a_raw + (uint32_t)(k0 + k) * (kTileM * 4) + ct * 4);
+                        if (PRECISE) tcs::split(v, hi[k], lo[k]);
+                        else hi[k] = __float_as_uint(v);
+                    }
+                    tcs::tmem_st16(a_cols + (uint32_t)k0, hi);
+                    if (PRECISE) tcs::tmem_st16(a_cols + kMaxK + (uint32_t)k0, lo);
+                }
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                tc::tc_fence_before();
+                mbar_arrive(a_conv_full + abuf);
+                mbar_arrive(a_raw_empty);
+            }
+            for (int t = w.t0; t < w.t1; ++t, ++q) {
+                const uint32_t s = q % kStagesB, bb = q & 1u;
+                if (!mbar_wait(b_raw_full + s, (q / kStagesB) & 1u) || !mbar_wait(b_conv_empty + bb, ((q >> 1) & 1u) ^ 1u)) {
+                    ok = false;
+                    break;
+                }
+                const uint32_t rb = b_raw + s * B_RAW;
+                const uint32_t b_hi = b_conv + bb * CONV_BUF, b_lo = b_hi + B_CONV;
+#pragma unroll
+                for (uint32_t j = 0; j < (uint32_t)(ROWS_B * (kMaxK / 4)) / 128u; ++j) {
+                    const uint32_t idx = ct + j * 128u;
+                    const uint32_t n = idx % ROWS_B, c = idx / ROWS_B;      // output unit, 16-byte chunk (four k)
+                    const uint32_t src = rb + (4 * c) * (ROWS_B * 4) + n * 4;
+                    const float4 v = make_float4(lds32(src), lds32(src + ROWS_B * 4), lds32(src + 2 * ROWS_B * 4),
+                                                 lds32(src + 3 * ROWS_B * 4));
+                    tcs::put<PRECISE>(b_hi, b_lo, c * B_LBO + (n >> 3) * SBO + (n & 7) * 16, v);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(b_conv_full + bb);
+                mbar_arrive(b_raw_empty + s);
+            }
+        }
+        if (!ok && lane == 0) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
+    }
+    else if (warp == 8) {
+        if (lane == 0) {
+            // ------------------------------ MMA issuer ------------------------------
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(ROWS_B >> 3) << 17) |
+                                   ((uint32_t)(kTileM >> 4) << 24);
+            uint32_t q = 0, it = 0;
+            for (int item = blockIdx.x; item < g.total_items && ok; item += gridDim.x, ++it) {
+                const Item w = decode(g, item);
+                const uint32_t abuf = it & 1u;
+                if (!mbar_wait(a_conv_full + abuf, (it >> 1) & 1u)) { ok = false; break; }
+                const uint32_t a_hi = tmem_base + A_COL0 + abuf * kACols, a_lo = a_hi + kMaxK;
+                for (int t = w.t0; t < w.t1; ++t, ++q) {
+                    const uint32_t bb = q & 1u, ph = (q >> 1) & 1u;
+                    if (!mbar_wait(b_conv_full + bb, ph) || !mbar_wait(acc_empty + bb, ph ^ 1u)) { ok = false; break; }
+                    tc::tc_fence_after();
+                    const uint32_t d = tmem_base + bb * kAccStride;
+                    const uint32_t b_hi = b_conv + bb * CONV_BUF, b_lo = b_hi + B_CONV;
+                    uint32_t acc = 0;
+                    for (int ks = 0; ks < KS; ++ks) {
+                        const uint64_t dbh = tc::smem_desc(b_hi + (uint32_t)ks * 2 * B_LBO, B_LBO, SBO);
+                        if (PRECISE) {
+                            const uint64_t dbl = tc::smem_desc(b_lo + (uint32_t)ks * 2 * B_LBO, B_LBO, SBO);
+                            tcs::mma_tf32_ts(d, a_lo + (uint32_t)ks * 8, dbh, idesc, acc); acc = 1;
+                            tcs::mma_tf32_ts(d, a_hi + (uint32_t)ks * 8, dbl, idesc, acc);
+                        }
+                        tcs::mma_tf32_ts(d, a_hi + (uint32_t)ks * 8, dbh, idesc, acc); acc = 1;
+                    }
+                    tc::mma_commit(b_conv_empty + bb);
+                    tc::mma_commit(acc_full + bb);
+                }
+                if (ok) tc::mma_commit(a_conv_empty + abuf);     // every MMA that reads this h tile has been issued
+            }
+            if (!ok) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
+        }
+    } else if (lane == 0) {
+        // ------------------------------ TMA loads ------------------------------
+        uint32_t q = 0, it = 0;                  // delta tiles and h tiles issued so far
+        for (int item = blockIdx.x; item < g.total_items && ok; item += gridDim.x) {
+            const Item w = decode(g, item);
+            if (!mbar_wait(a_raw_empty, (it & 1u) ^ 1u)) { ok = false; break; }
+            mbar_expect_tx(a_raw_full, A_RAW);
+            tma_load_3d(a_raw, &mapA, w.m0, 0, w.node, a_raw_full);
+            ++it;
+            for (int t = w.t0; t < w.t1; ++t, ++q) {
+                const uint32_t s = q % kStagesB;
+                if (!mbar_wait(b_raw_empty + s, ((q / kStagesB) & 1u) ^ 1u)) { ok = false; break; }
+                mbar_expect_tx(b_raw_full + s, B_RAW);
+                tma_load_3d(b_raw + s * B_RAW, &mapB, t * ROWS_B, 0, w.node, b_raw_full + s);
+            }
+        }
+        // loads still in flight (only when somebody gave up): let them land before the CTA leaves
+        if (it > 0) mbar_wait(a_raw_full, (it - 1) & 1u);
+        for (uint32_t j = 0; j < (uint32_t)kStagesB && j < q; ++j) {
+            const uint32_t qq = q - 1 - j;
+            mbar_wait(b_raw_full + qq % kStagesB, (qq / kStagesB) & 1u);
+        }
+        if (!ok) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    if (warp == 8) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+}  // namespace tcw
+}  // namespace dpsgd
