@@ -30,8 +30,14 @@ struct MlpPlan {
     int B;
     int n;
     size_t act_off[kMaxLayers + 2];
-    size_t delta_off[kMaxLayers + 1];   // delta_l for l = 1..L, stored [l][node][B][d_l]
+    size_t delta_off[kMaxLayers + 1];   // delta_l for l = 1..L, stored [l][node][B][pitch_l]
+    int delta_pitch[kMaxLayers + 1];    // d_l; the output layer's rounded up to 4 floats (16-byte rows for TMA)
 };
+
+int delta_row_floats(const dpsgd_ctx* c, int l) {
+    const int d = c->mlp.dims[l];
+    return l == c->mlp.nlayers ? (d + 3) & ~3 : d;
+}
 
 MlpPlan make_plan(const dpsgd_ctx* c) {
     MlpPlan p{};
@@ -41,7 +47,8 @@ MlpPlan make_plan(const dpsgd_ctx* c) {
         p.act_off[l] = a;
         a += (size_t)c->n * c->batch * c->mlp.dims[l];
         p.delta_off[l] = d;
-        if (l >= 1) d += (size_t)c->n * c->batch * c->mlp.dims[l];
+        p.delta_pitch[l] = delta_row_floats(c, l);
+        if (l >= 1) d += (size_t)c->n * c->batch * p.delta_pitch[l];
     }
     return p;
 }
@@ -146,14 +153,14 @@ bgemm_kernel(GemmArgs g) {
 __global__ void __launch_bounds__(128)
 softmax_ce_delta_kernel(const float* __restrict__ logits, const int32_t* __restrict__ y, int64_t m,
                         const int32_t* __restrict__ idx, int n, int B, int C, float* __restrict__ delta,
-                        const int32_t* __restrict__ node_batch) {
+                        int dpitch, const int32_t* __restrict__ node_batch) {
     const int w = blockIdx.x * 4 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (w >= n * B) return;
     const int node = w / B;
     const int Bi = node_batch ? __ldg(node_batch + node) : B;
     if (w - node * B >= Bi) {
-        for (int c = lane; c < C; c += 32) delta[(int64_t)w * C + c] = 0.f;
+        for (int c = lane; c < C; c += 32) delta[(int64_t)w * dpitch + c] = 0.f;
         return;
     }
     const float* z = logits + (int64_t)w * C;
@@ -168,19 +175,19 @@ softmax_ce_delta_kernel(const float* __restrict__ logits, const int32_t* __restr
     const int label = __ldg(y + (int64_t)node * m + __ldg(idx + w));
     const float inv = 1.f / s, invB = 1.f / (float)Bi;
     for (int c = lane; c < C; c += 32)
-        delta[(int64_t)w * C + c] = (expf(z[c] - mx) * inv - (c == label ? 1.f : 0.f)) * invB;
+        delta[(int64_t)w * dpitch + c] = (expf(z[c] - mx) * inv - (c == label ? 1.f : 0.f)) * invB;
 }
 
 // gb[o] = sum_b delta[b][o], written into the gradient row; fixed order over b.
 __global__ void __launch_bounds__(128)
-bias_grad_kernel(const float* __restrict__ delta, int B, int D, float* __restrict__ G, int64_t ld,
+bias_grad_kernel(const float* __restrict__ delta, int B, int D, int dpitch, float* __restrict__ G, int64_t ld,
                  int64_t b_off) {
     const int node = blockIdx.y;
     const int o = blockIdx.x * 128 + threadIdx.x;
     if (o >= D) return;
-    const float* d = delta + (int64_t)node * B * D + o;
+    const float* d = delta + (int64_t)node * B * dpitch + o;
     float s = 0.f;
-    for (int b = 0; b < B; ++b) s += d[(int64_t)b * D];
+    for (int b = 0; b < B; ++b) s += d[(int64_t)b * dpitch];
     G[(int64_t)node * ld + b_off + o] = s;
 }
 
@@ -355,19 +362,18 @@ cudaError_t launch_tcw_inst(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtenso
 
 // gW[o][k'] = sum_b delta[b][o] h[b][k'] for every node.  Returns cudaErrorNotSupported when the
 // shapes or alignments rule the TMA path out (the caller falls back).
-cudaError_t run_tcw(dpsgd_ctx* c, const float* h, int din, const float* delta, int dout, float* gW) {
+cudaError_t run_tcw(dpsgd_ctx* c, const float* h, int din, const float* delta, int dout, int dpitch, float* gW) {
     const int B = c->batch;
     auto al = [](const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; };
-    if (B > tcw::kMaxK || din % 4 != 0 || dout % 4 != 0 || !al(h) || !al(delta) || !al(gW) || c->ld % 4 != 0 ||
-        ((int64_t)B * din) % 4 != 0 || ((int64_t)B * dout) % 4 != 0)
+    if (B > tcw::kMaxK || din % 4 != 0 || dpitch % 4 != 0 || !al(h) || !al(delta) || !al(gW) || c->ld % 4 != 0)
         return cudaErrorNotSupported;
     const int rows_b = dout <= 16 ? 16 : (dout <= 32 ? 32 : 64);
     const uint64_t nodes = (uint64_t)c->n;
     CUtensorMap mapA, mapB, mapC;
     bool ok = make_map_3d(&mapA, h, (uint64_t)din, (uint64_t)B, nodes, (uint64_t)din * 4, (uint64_t)B * din * 4,
                           tcw::kTileM, tcw::kMaxK, false);
-    ok = ok && make_map_3d(&mapB, delta, (uint64_t)dout, (uint64_t)B, nodes, (uint64_t)dout * 4,
-                           (uint64_t)B * dout * 4, (uint32_t)rows_b, tcw::kMaxK, false);
+    ok = ok && make_map_3d(&mapB, delta, (uint64_t)dout, (uint64_t)B, nodes, (uint64_t)dpitch * 4,
+                           (uint64_t)B * dpitch * 4, (uint32_t)rows_b, tcw::kMaxK, false);
     ok = ok && make_map_3d(&mapC, gW, (uint64_t)din, (uint64_t)dout, nodes, (uint64_t)din * 4, (uint64_t)c->ld * 4,
                            tcw::kTileM, (uint32_t)rows_b, false);
     if (!ok) return cudaErrorNotSupported;
@@ -404,7 +410,7 @@ size_t mlp_act_floats(const dpsgd_ctx* c) {
 
 size_t mlp_delta_floats(const dpsgd_ctx* c) {
     size_t a = 0;
-    for (int l = 1; l <= c->mlp.nlayers; ++l) a += (size_t)c->n * c->batch * c->mlp.dims[l];
+    for (int l = 1; l <= c->mlp.nlayers; ++l) a += (size_t)c->n * c->batch * delta_row_floats(c, l);
     return a;
 }
 
@@ -443,36 +449,37 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) 
 
     softmax_ce_delta_kernel<<<(n * B + 3) / 4, 128, 0, c->stream>>>(
         c->d_act + p.act_off[L], y, c->m, c->d_idx, n, B, s.dims[L], c->d_delta + p.delta_off[L],
-        c->d_node_batch);
+        p.delta_pitch[L], c->d_node_batch);
     c->launches++;
 
     // backward
     for (int l = L; l >= 1; --l) {
         const int din = s.dims[l - 1], dout = s.dims[l];
         const float* delta = c->d_delta + p.delta_off[l];
+        const int dp = p.delta_pitch[l];      // floats per sample in delta_l
         {   // gW_l[o][k] = sum_b delta[b][o] h_{l-1}[b][k]
             GemmArgs g{};
-            g.A = delta; g.a_node = (int64_t)B * dout; g.a_m = 1; g.a_k = dout;
+            g.A = delta; g.a_node = (int64_t)B * dp; g.a_m = 1; g.a_k = dp;
             g.Bm = c->d_act + p.act_off[l - 1]; g.b_node = (int64_t)B * din; g.b_n = 1; g.b_k = din;
             g.C = G + s.w_off[l - 1]; g.c_node = c->ld; g.c_m = din;
             g.M = dout; g.N = din; g.K = B;
             if (use_tc) {   // m = input unit k', n = output unit o: gW[o][k']
                 tc::Args a{};
                 a.A = g.Bm; a.a_node = g.b_node; a.a_pitch = din; a.a_kcontig = 0;
-                a.B = delta; a.b_node = (int64_t)B * dout; a.b_pitch = dout; a.b_kcontig = 0;
+                a.B = delta; a.b_node = (int64_t)B * dp; a.b_pitch = dp; a.b_kcontig = 0;
                 a.C = g.C; a.c_node = c->ld; a.c_pitch = din;
                 a.M = din; a.N = dout; a.K = B; a.epi = tc::EPI_STORE;
-                cudaError_t e = run_tcw(c, g.Bm, din, delta, dout, g.C);
+                cudaError_t e = run_tcw(c, g.Bm, din, delta, dout, dp, g.C);
                 if (e == cudaErrorNotSupported) e = run_tc(c, a, 64);
                 if (e != cudaSuccess) return e;
             } else run_gemm<false, false, EPI_STORE>(c, g);
         }
-        bias_grad_kernel<<<dim3((dout + 127) / 128, n), 128, 0, c->stream>>>(delta, B, dout, G, c->ld,
+        bias_grad_kernel<<<dim3((dout + 127) / 128, n), 128, 0, c->stream>>>(delta, B, dout, dp, G, c->ld,
                                                                                s.b_off[l - 1]);
         c->launches++;
         if (l > 1) {   // delta_{l-1}[b][k] = (sum_o delta[b][o] W_l[o][k]) * [h_{l-1}[b][k] > 0]
             GemmArgs g{};
-            g.A = delta; g.a_node = (int64_t)B * dout; g.a_m = dout; g.a_k = 1;
+            g.A = delta; g.a_node = (int64_t)B * dp; g.a_m = dp; g.a_k = 1;
             g.Bm = X + s.w_off[l - 1]; g.b_node = c->ld; g.b_n = 1; g.b_k = din;
             g.C = c->d_delta + p.delta_off[l - 1]; g.c_node = (int64_t)B * din; g.c_m = din;
             g.aux = c->d_act + p.act_off[l - 1]; g.aux_node = (int64_t)B * din; g.aux_m = din;
@@ -480,7 +487,7 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) 
             if (use_tc) {   // m = input unit k', n = sample: delta_{l-1}[b][k']
                 tc::Args a{};
                 a.A = g.Bm; a.a_node = c->ld; a.a_pitch = din; a.a_kcontig = 0;
-                a.B = delta; a.b_node = (int64_t)B * dout; a.b_pitch = dout; a.b_kcontig = 1;
+                a.B = delta; a.b_node = (int64_t)B * dp; a.b_pitch = dp; a.b_kcontig = 1;
                 a.C = g.C; a.c_node = g.c_node; a.c_pitch = din;
                 a.aux = g.aux; a.aux_node = g.aux_node; a.aux_pitch = din;
                 a.M = din; a.N = B; a.K = dout; a.epi = tc::EPI_MASK;

@@ -287,6 +287,7 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                     const uint32_t b_hi = conv + buf * CONV_BUF, b_lo = b_hi + B_CONV;
 #pragma unroll
                     for (uint32_t kk = 0; kk < kBK / 8; ++kk) {  // one MMA consumes k = 8: 8 columns of A, two chunk columns of B
+                        if ((int)(kb * kBK + kk * 8) >= g.K) break;   // nothing but zero fill from here on
                         const uint64_t dbh = tc::smem_desc(b_hi + kk * 2 * B_LBO, B_LBO, SBO);
                         if (PRECISE) {
                             const uint64_t dbl = tc::smem_desc(b_lo + kk * 2 * B_LBO, B_LBO, SBO);
