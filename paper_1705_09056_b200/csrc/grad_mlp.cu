@@ -16,6 +16,7 @@
 
 #include "ctx.h"
 #include "philox.cuh"
+#include "grad_mlp_narrow.cuh"
 #include "tc_gemm.cuh"
 #include "tc_stream.cuh"
 #include "tc_wgrad.cuh"
@@ -457,6 +458,28 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) 
         const int din = s.dims[l - 1], dout = s.dims[l];
         const float* delta = c->d_delta + p.delta_off[l];
         const int dp = p.delta_pitch[l];      // floats per sample in delta_l
+        if (use_tc && l == L && dout <= narrow::kMaxOut && (size_t)B * narrow::kMaxOut * sizeof(float) <= 32 * 1024) {
+            // classifier layer: weight gradient and the error passed on, in one pass over h_{l-1}
+            auto a16 = [](const void* q) { return reinterpret_cast<uintptr_t>(q) % 16 == 0; };
+            const float* hprev = c->d_act + p.act_off[l - 1];
+            float* dprev = l > 1 ? c->d_delta + p.delta_off[l - 1] : nullptr;
+            const size_t smem = (size_t)B * narrow::kMaxOut * sizeof(float);
+            const bool vec = din % 4 == 0 && s.w_off[l - 1] % 4 == 0 && a16(X) && a16(G) && a16(hprev) &&
+                             (!dprev || a16(dprev));
+            if (vec)
+                narrow::narrow_backward_kernel<4><<<dim3((din + 4 * narrow::kBwdThreads - 1) / (4 * narrow::kBwdThreads), n),
+                                                    narrow::kBwdThreads, smem, c->stream>>>(
+                    X, G, c->ld, s.w_off[l - 1], hprev, delta, dp, dprev, B, din, dout);
+            else
+                narrow::narrow_backward_kernel<1><<<dim3((din + narrow::kBwdThreads - 1) / narrow::kBwdThreads, n),
+                                                    narrow::kBwdThreads, smem, c->stream>>>(
+                    X, G, c->ld, s.w_off[l - 1], hprev, delta, dp, dprev, B, din, dout);
+            c->launches++;
+            bias_grad_kernel<<<dim3((dout + 127) / 128, n), 128, 0, c->stream>>>(delta, B, dout, dp, G, c->ld,
+                                                                                   s.b_off[l - 1]);
+            c->launches++;
+            continue;
+        }
         {   // gW_l[o][k] = sum_b delta[b][o] h_{l-1}[b][k]
             GemmArgs g{};
             g.A = delta; g.a_node = (int64_t)B * dp; g.a_m = 1; g.a_k = dp;
