@@ -9,9 +9,13 @@
 //     gW_l    = delta_l^T h_{l-1},   gb_l = sum_b delta_l[b],
 //     delta_{l-1} = (delta_l W_l) * [h_{l-1} > 0]                      (ReLU'(0) = 0)
 // All three products are batched GEMMs over the n nodes with per-node operands.  They run on the
-// tensor cores (tc_gemm.cuh: tcgen05 TF32 MMAs, three per product for fp32-faithful results) when
-// the minibatch fits a 128-column tile, and otherwise - or when asked - on the fp32 FMA kernel
-// below (exact fp32 products, fp32 accumulation in a fixed order).
+// tensor cores (tcgen05 TF32 MMAs, three per product for fp32-faithful results) when the minibatch
+// fits a 128-column tile: forward and input gradient on the weight-streaming kernel of tc_stream.cuh,
+// the weight gradient on tc_wgrad.cuh (both TMA-fed, weight-side operand in tensor memory), the
+// classifier layer's backward on the fp32 kernel of grad_mlp_narrow.cuh, and shapes TMA cannot
+// address (rows not 16-byte aligned) on the register-staged kernel of tc_gemm.cuh.  Otherwise - or
+// when asked - everything runs on the fp32 FMA kernel below (exact fp32 products, fp32 accumulation
+// in a fixed order).
 #include <algorithm>
 
 #include "ctx.h"
