@@ -141,6 +141,26 @@ DPSGD_API dpsgd_status dpsgd_mix_update(dpsgd_ctx* ctx);
 DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* ctx, int32_t update_then_mix);
 
 /*
+ * Algorithm 1 steps 3-5 in one pass for the MLP: with mode != 0, dpsgd_step() applies the gossip step
+ * X_next <- W X_cur - gamma dF(X_cur; xi) (Section 3) inside the kernels that form the weight
+ * gradients, tile by tile while the gradient is on chip.  Those blocks of the gradient are never
+ * written: per parameter the iteration moves 8 bytes through HBM (read X, write X_next) instead of 16
+ * (write G, then read X and G and write X_next).  After such a step the fused weight blocks of G hold
+ * old values; biases, and blocks whose product runs on another kernel, are still written to G and
+ * take the gossip step from there.  The result equals dpsgd_grad + dpsgd_mix_update up to fp32
+ * rounding order.
+ *   mode 0  off (default): two stages.
+ *   mode 1  fused for the weight blocks where it is faster on B200: rows of W with at most 3 entries
+ *           (a ring) and a stacked block of at least 512 MB (beyond L2); other blocks in two stages.
+ *   mode 2  fused for every block the kernel can take.
+ * The kernel applies when the model is the MLP on the tensor-core path (minibatch <= 64, layer input
+ * widths multiples of 4), the printed order of Algorithm 1 is in force, no momentum is set and no row
+ * of W has more than 8 entries; otherwise dpsgd_step() runs the two stages whatever the mode.
+ * dpsgd_grad, dpsgd_mix_update and the other entry points are not affected.
+ */
+DPSGD_API dpsgd_status dpsgd_set_fused_step(dpsgd_ctx* ctx, int32_t mode);
+
+/*
  * A local iteration without communication (Section 5.3, last paragraph: a node may run more than
  * one minibatch before it synchronises): samples xi_{k,i}, computes g_i at x_{k,i} and updates
  * x_i <- x_i - gamma g_i in place (the gossip step with W = I), momentum included when set.  Call it

@@ -42,6 +42,7 @@ SIGNATURES = {
     "dpsgd_local_step_nodes": [_vp, _u64, _vp],
     "dpsgd_set_node_batches": [_vp, _vp],
     "dpsgd_set_order": [_vp, _i32],
+    "dpsgd_set_fused_step": [_vp, _i32],
     "dpsgd_set_momentum": [_vp, _f32, _vp],
     "dpsgd_mix_update_consensus": [_vp, _vp],
     "dpsgd_step_consensus": [_vp, _u64, _vp],
@@ -213,6 +214,11 @@ class Dpsgd:
     def set_order(self, update_then_mix: bool):
         """Footnote c of Algorithm 1: apply the local gradient first, then average."""
         self._check(self._lib.dpsgd_set_order(self._h, 1 if update_then_mix else 0))
+
+    def set_fused_step(self, mode: int):
+        """MLP: let step() apply the gossip step inside the weight-gradient kernels (those blocks of G
+        are then not written).  0 off, 1 where it is faster, 2 wherever the kernel applies."""
+        self._check(self._lib.dpsgd_set_fused_step(self._h, int(mode)))
 
     def set_momentum(self, beta: float, V: Optional[torch.Tensor]):
         """Heavy-ball momentum (Section 5.3): V is an n x ld fp32 CUDA tensor, zero at the start; None = off."""

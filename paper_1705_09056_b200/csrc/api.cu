@@ -80,6 +80,9 @@ void classify_w(dpsgd_ctx* c) {
     int max_deg = 0;
     for (int i = 0; i < n; ++i) max_deg = std::max(max_deg, rp[i + 1] - rp[i]);
     c->W.max_deg = max_deg;
+    bool same_deg = true;
+    for (int i = 0; i < n; ++i) same_deg = same_deg && rp[i + 1] - rp[i] == max_deg;
+    c->W.uniform_deg = same_deg ? max_deg : 0;
 
     bool uniform = (int64_t)rp[n] == (int64_t)n * n;
     if (uniform)
@@ -487,10 +490,30 @@ DPSGD_API dpsgd_status dpsgd_step_consensus(dpsgd_ctx* c, uint64_t k, double* ou
     return mix_with_consensus(c, out_dev);
 }
 
+DPSGD_API dpsgd_status dpsgd_set_fused_step(dpsgd_ctx* c, int32_t on) {
+    if (!c) return DPSGD_ERR_ARG;
+    drop_graph(c);
+    if (on < 0 || on > 2) return fail(c, DPSGD_ERR_ARG, "mode must be 0, 1 or 2");
+    c->fuse_step = on;
+    return DPSGD_OK;
+}
+
 DPSGD_API dpsgd_status dpsgd_step(dpsgd_ctx* c, uint64_t k) {
     dpsgd_status s = need_bound(c);
     if (s != DPSGD_OK) return s;
     if ((s = need_model(c)) != DPSGD_OK) return s;
+    if (c->fuse_step && fused_step_supported(c)) {
+        // the weight-gradient kernels write their blocks of X_next themselves; the remaining columns
+        // (biases, blocks on other kernels, padding) take the gossip step from G afterwards
+        const float* X = c->X[c->cur];
+        float* Xn = c->X[c->cur ^ 1];
+        cudaError_t e = launch_grad_mlp(c, k, X, c->G, Xn);
+        if (e != cudaSuccess) return cuda_fail(c, e, "gradient kernels");
+        e = c->fused_blocks.empty() ? run_mix(c) : launch_mix_rest(c, X, c->G, Xn);
+        if (e != cudaSuccess) return cuda_fail(c, e, "mix_update kernel");
+        c->cur ^= 1;
+        return DPSGD_OK;
+    }
     cudaError_t e = run_grad(c, k);
     if (e != cudaSuccess) return cuda_fail(c, e, "gradient kernels");
     e = run_mix(c);

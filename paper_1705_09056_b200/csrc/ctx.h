@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "../../include/dpsgd.h"
@@ -12,12 +13,14 @@
 namespace dpsgd {
 
 constexpr int kMaxLayers = 8;
+constexpr int kFusedMaxDegree = 8;   // widest row of W the gradient kernel's gossip epilogue gathers
 
 // Mixing matrix W on the device, as the kernels consume it.
 struct MixW {
     int n = 0;
     int nnz = 0;
     int max_deg = 0;
+    int uniform_deg = 0;               // the common number of entries per row, 0 when rows differ
     const int32_t* row_ptr = nullptr;  // [n+1]
     const int32_t* col = nullptr;      // [nnz]
     const float* val = nullptr;        // [nnz]
@@ -102,6 +105,10 @@ struct dpsgd_ctx {
     int graph_cur = 0;                       // value of `cur` the graph was captured at
     int64_t graph_launches = 0;              // kernels in one replay
 
+    // gossip step fused into the MLP weight-gradient kernels (dpsgd_set_fused_step)
+    int fuse_step = 0;         // 0 off, 1 where it pays, 2 wherever the kernel applies
+    std::vector<std::pair<int64_t, int64_t>> fused_blocks;   // [begin, end) columns already written to X_next
+
     int64_t launches = 0;
     std::string err;
 };
@@ -132,7 +139,15 @@ cudaError_t launch_sample(dpsgd_ctx* c, uint64_t k, int32_t* idx);
 cudaError_t launch_set_k(dpsgd_ctx* c, uint64_t v);
 cudaError_t launch_advance_k(dpsgd_ctx* c);
 cudaError_t launch_grad_linear(dpsgd_ctx* c, uint64_t k, const float* X, float* G);
-cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G);
+// Xn != NULL: weight blocks whose product runs on the fused kernel are written to Xn after the gossip
+// step instead of to G, and listed in c->fused_blocks.
+cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G, float* Xn = nullptr);
+bool fused_step_supported(const dpsgd_ctx* c);
+bool fused_step_pays(const dpsgd_ctx* c, int din, int dout);
+cudaError_t run_tcw_fused(dpsgd_ctx* c, const float* h, int din, const float* delta, int dout, int dpitch,
+                          int64_t w_off, const float* X, float* Xn);
+// Gossip step on the columns of [0, ld) outside c->fused_blocks.
+cudaError_t launch_mix_rest(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
 size_t mlp_act_floats(const dpsgd_ctx* c);
 size_t mlp_delta_floats(const dpsgd_ctx* c);
 

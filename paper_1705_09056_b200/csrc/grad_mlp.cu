@@ -358,8 +358,9 @@ cudaError_t launch_tcw_inst(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtenso
     int chunks = (int)std::min<long long>(a.n_tiles, std::max<long long>(1, (12LL * sms + blocks - 1) / blocks));
     a.chunk = (a.n_tiles + chunks - 1) / chunks;
     a.chunks = (a.n_tiles + a.chunk - 1) / a.chunk;
-    a.total_items = (int)(blocks * a.chunks);
-    const int grid = std::min(a.total_items, sms);               // one persistent CTA per SM
+    a.nodes = c->n; a.splits = c->n; a.split_len = 1;            // node-major order
+    a.total_seqs = (int)(blocks * a.chunks);
+    const int grid = std::min(a.total_seqs, sms);                // one persistent CTA per SM
     kernel<<<grid, tcw::kThreads, smem, c->stream>>>(mapA, mapB, mapC, a);
     c->launches++;
     return cudaGetLastError();
@@ -419,8 +420,9 @@ size_t mlp_delta_floats(const dpsgd_ctx* c) {
     return a;
 }
 
-cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) {
+cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G, float* Xn) {
     const MlpPlan p = make_plan(c);
+    c->fused_blocks.clear();
     const MlpShape& s = c->mlp;
     const int n = c->n, B = c->batch, L = s.nlayers;
     const int32_t* y = static_cast<const int32_t*>(c->y);
@@ -496,7 +498,12 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G) 
                 a.B = delta; a.b_node = (int64_t)B * dp; a.b_pitch = dp; a.b_kcontig = 0;
                 a.C = g.C; a.c_node = c->ld; a.c_pitch = din;
                 a.M = din; a.N = dout; a.K = B; a.epi = tc::EPI_STORE;
-                cudaError_t e = run_tcw(c, g.Bm, din, delta, dout, dp, g.C);
+                cudaError_t e = cudaErrorNotSupported;
+                if (Xn && (c->fuse_step >= 2 || fused_step_pays(c, din, dout))) {   // gossip step applied in the product's epilogue: this block goes straight to X_next
+                    e = run_tcw_fused(c, g.Bm, din, delta, dout, dp, s.w_off[l - 1], X, Xn);
+                    if (e == cudaSuccess) c->fused_blocks.emplace_back(s.w_off[l - 1], s.w_off[l - 1] + (int64_t)dout * din);
+                }
+                if (e == cudaErrorNotSupported) e = run_tcw(c, g.Bm, din, delta, dout, dp, g.C);
                 if (e == cudaErrorNotSupported) e = run_tc(c, a, 64);
                 if (e != cudaSuccess) return e;
             } else run_gemm<false, false, EPI_STORE>(c, g);

@@ -7,6 +7,8 @@
 // and let it walk down the n rows; a warp therefore touches 512 contiguous bytes of one row
 // per access.  The stacked matrices are far larger than L2 on the bandwidth-bound shapes, so
 // once-only traffic uses streaming (evict-first) loads and stores.
+#include <algorithm>
+
 #include "ctx.h"
 
 namespace dpsgd {
@@ -182,7 +184,71 @@ mix_rowpar_kernel(const float4* __restrict__ X, const float4* __restrict__ G, fl
     Xn[(int64_t)i * ld4 + c] = a;
 }
 
+// Gossip step on a few column ranges of the stacked matrices (the columns a fused gradient kernel
+// has not already written): one thread per output group of 4 columns, as in the kernel above.
+struct ColRanges {
+    int count;
+    int64_t begin4[kMaxLayers + 1];   // first float4 column of each range
+    int64_t start4[kMaxLayers + 2];   // running total of the range lengths, start4[count] = all
+};
+
+__global__ void __launch_bounds__(128)
+mix_ranges_kernel(const float4* __restrict__ X, const float4* __restrict__ G, float4* __restrict__ Xn,
+                  const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col,
+                  const float* __restrict__ val, int64_t ld4, float ngamma, ColRanges rg) {
+    const int64_t t = (int64_t)blockIdx.x * 128 + threadIdx.x;
+    const int i = blockIdx.y;
+    if (t >= rg.start4[rg.count]) return;
+    int r = 0;
+    while (r + 1 < rg.count && t >= rg.start4[r + 1]) ++r;
+    const int64_t c = rg.begin4[r] + (t - rg.start4[r]);
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int pe = __ldg(row_ptr + i + 1);
+    for (int p = __ldg(row_ptr + i); p < pe; ++p) {
+        const float w = __ldg(val + p);
+        const float4 v = __ldg(X + (int64_t)__ldg(col + p) * ld4 + c);
+        a.x = fmaf(w, v.x, a.x); a.y = fmaf(w, v.y, a.y);
+        a.z = fmaf(w, v.z, a.z); a.w = fmaf(w, v.w, a.w);
+    }
+    const float4 g = __ldg(G + (int64_t)i * ld4 + c);
+    a.x = fmaf(ngamma, g.x, a.x); a.y = fmaf(ngamma, g.y, a.y);
+    a.z = fmaf(ngamma, g.z, a.z); a.w = fmaf(ngamma, g.w, a.w);
+    Xn[(int64_t)i * ld4 + c] = a;
+}
+
 }  // namespace
+
+cudaError_t launch_mix_rest(dpsgd_ctx* c, const float* X, const float* G, float* Xn) {
+    // complement of the fused blocks inside [0, ld); block bounds are multiples of 4 columns
+    std::vector<std::pair<int64_t, int64_t>> blocks = c->fused_blocks;
+    std::sort(blocks.begin(), blocks.end());
+    ColRanges rg{};
+    int64_t at = 0, total = 0;
+    auto add = [&](int64_t b, int64_t e) {
+        if (e <= b) return true;
+        if (rg.count >= kMaxLayers + 1) return false;
+        rg.begin4[rg.count] = b / 4;
+        rg.start4[rg.count] = total;
+        total += (e - b) / 4;
+        rg.count++;
+        return true;
+    };
+    for (const auto& b : blocks) {
+        if (b.first % 4 != 0 || b.second % 4 != 0 || b.first < at || b.second > c->ld) return cudaErrorInvalidValue;
+        if (!add(at, b.first)) return cudaErrorInvalidValue;
+        at = b.second;
+    }
+    if (!add(at, c->ld)) return cudaErrorInvalidValue;
+    rg.start4[rg.count] = total;
+    if (total == 0) return cudaSuccess;
+    if (c->n > 65535) return cudaErrorInvalidValue;
+    dim3 grid((unsigned)((total + 127) / 128), (unsigned)c->n);
+    mix_ranges_kernel<<<grid, 128, 0, c->stream>>>(
+        reinterpret_cast<const float4*>(X), reinterpret_cast<const float4*>(G), reinterpret_cast<float4*>(Xn),
+        c->W.row_ptr, c->W.col, c->W.val, c->ld / 4, -c->gamma, rg);
+    c->launches++;
+    return cudaGetLastError();
+}
 
 bool mix_is_small(const dpsgd_ctx* c) {
     return (int64_t)c->n * c->ld * (int64_t)sizeof(float) <= (int64_t(8) << 20) && c->n <= 65535 &&

@@ -19,6 +19,17 @@
 //                   which writes whole lines asynchronously and clips at the matrix edge; two
 //                   staging buffers, so the store of one tile overlaps the next.
 //
+// FUSE: the gossip step of Algorithm 1 (steps 4-5) is applied to the tile while it is on chip.  No
+// TMA store: sixteen more warps (the mixers; the gather is bound by the bytes they keep in flight)
+// take a staged tile, read the same tile of X from the node's neighbours in W and write
+//     X_next[node] = sum_j W_ij X[j] - gamma * gW
+// with 128-bit accesses along the input-unit index.  The neighbours' tiles are shared with the work
+// items of the neighbouring nodes; a CTA walks consecutive nodes at one tile position, so all but the
+// first read of an element come from L2, and the mixers prefetch the next node's tiles into L2 one
+// item ahead so that the first read does too.  This block of the gradient
+// never reaches HBM: 8 bytes per parameter (read X, write X_next) instead of 16 (write G; read X,
+// read G, write X_next).
+//
 // One persistent CTA per SM; a work item is (node, 128-row block of m, run of column tiles).  Every
 // mbarrier wait is bounded; a wait that runs out raises the status word, the TMA thread waits
 // (bounded) for its loads in flight, outstanding stores are drained, and the CTA frees its TMEM
@@ -38,17 +49,40 @@ using tcs::mbar_expect_tx;
 using tcs::tma_load_3d;
 
 constexpr int kThreads = 320;        // 4 epilogue warps, 4 converter warps, MMA warp, TMA warp
+constexpr int kMixWarps = 16;        // FUSE only: warps 10..25 apply the gossip step to staged tiles
+constexpr int kThreadsFused = kThreads + 32 * kMixWarps;
 constexpr int kTileM = 128;
 constexpr int kMaxK = 64;            // minibatch rows a raw tile holds
 constexpr int kStagesB = 3;
 constexpr uint32_t kAccStride = 64;  // TMEM columns per accumulator
 constexpr uint32_t kACols = 2 * kMaxK;   // heads, then remainders
 
+// What the fused gossip epilogue needs: the stacked X of this iteration, the buffer of the next one,
+// where this weight block starts inside a parameter row, W in CSR and -gamma.
+struct Mix {
+    const float* X;
+    float* Xn;
+    int64_t ld, w_off;
+    const int32_t* row_ptr;
+    const int32_t* col;
+    const float* val;
+    float ngamma;
+};
+
+// Work decomposition.  A work item is (node, 128-row block of m, run of `chunk` column tiles); the h
+// tile of the item is converted once and serves its column tiles.  Items are grouped into sequences of
+// `split_len` consecutive nodes at one (row block, run) position; a CTA takes whole sequences
+// (blockIdx.x, blockIdx.x + gridDim.x, ...), ordered run-fastest, then row block, then node range.
+// split_len = 1 gives plain node-major order.  The fused kernel walks longer node ranges so that the
+// neighbours' tiles of X it gathers for node i were fetched by the same CTA for nodes i-1 and i-2.
 struct Args {
     int M, N, K;                     // din, dout, minibatch
+    int nodes;
     int m_tiles, n_tiles, chunk, chunks;   // column tiles per item, items per (node, m block)
-    int total_items;
+    int splits, split_len;           // node ranges, nodes per range
+    int total_seqs;                  // m_tiles * chunks * splits
     int* status;
+    Mix mix;                         // FUSE only
 };
 
 __host__ __device__ constexpr uint32_t a_raw_bytes() { return kMaxK * kTileM * 4; }
@@ -67,17 +101,100 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
     asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
                  ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
 }
+__device__ __forceinline__ void prefetch_l2(const void* p) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
 __device__ __forceinline__ void sts32(uint32_t addr, float v) {
     asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
 
-struct Item { int node, m0, t0, t1; };
-__device__ __forceinline__ Item decode(const Args& g, int item) {
-    const int per_node = g.m_tiles * g.chunks;
-    Item w;
-    w.node = item / per_node;
-    const int rem = item - w.node * per_node;
+// Gossip step on ROWS rows (output units) of a staged gradient tile: warp `warp` of the kMixWarps
+// mixer warps takes rows warp, warp + kMixWarps, ...; its lanes cover the 128 input units of a row, four each.
+// `off` = offset of (first row of the tile, this lane's first column) inside a parameter row; rows at
+// or beyond `rows` and lanes with !col_ok lie outside the weight matrix.  DEG > 0: every row of W has
+// DEG entries (loads of four rows x DEG neighbours in flight); DEG == 0: any degree.
+template <int DEG, int ROWS>
+__device__ __forceinline__ void mix_rows(const Mix& mx, int node, uint32_t st, int64_t off, int din, int rows,
+                                         bool col_ok, int warp, int lane) {
+    constexpr int U = 4;
+    const int p0 = __ldg(mx.row_ptr + node);
+    const int deg = DEG > 0 ? DEG : __ldg(mx.row_ptr + node + 1) - p0;
+    float* out = mx.Xn + (int64_t)node * mx.ld + off;
+#pragma unroll 1
+    for (int r0 = warp; r0 < ROWS; r0 += kMixWarps * U) {
+        float4 acc[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (DEG > 0) {
+            float4 v[DEG > 0 ? DEG : 1][U];
+#pragma unroll
+            for (int p = 0; p < DEG; ++p) {
+                const float* xr = mx.X + (int64_t)__ldg(mx.col + p0 + p) * mx.ld + off;
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int r = r0 + kMixWarps * u;
+                    v[p][u] = (col_ok && r < rows) ? __ldcg(reinterpret_cast<const float4*>(xr + (int64_t)r * din))
+                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int p = 0; p < DEG; ++p) {
+                const float w = __ldg(mx.val + p0 + p);
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    acc[u].x = fmaf(w, v[p][u].x, acc[u].x); acc[u].y = fmaf(w, v[p][u].y, acc[u].y);
+                    acc[u].z = fmaf(w, v[p][u].z, acc[u].z); acc[u].w = fmaf(w, v[p][u].w, acc[u].w);
+                }
+            }
+        } else {
+#pragma unroll 1
+            for (int p = 0; p < deg; ++p) {
+                const float* xr = mx.X + (int64_t)__ldg(mx.col + p0 + p) * mx.ld + off;
+                const float w = __ldg(mx.val + p0 + p);
+                float4 v[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int r = r0 + kMixWarps * u;
+                    v[u] = (col_ok && r < rows) ? __ldcg(reinterpret_cast<const float4*>(xr + (int64_t)r * din))
+                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    acc[u].x = fmaf(w, v[u].x, acc[u].x); acc[u].y = fmaf(w, v[u].y, acc[u].y);
+                    acc[u].z = fmaf(w, v[u].z, acc[u].z); acc[u].w = fmaf(w, v[u].w, acc[u].w);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int r = r0 + kMixWarps * u;
+            if (col_ok && r < rows) {
+                const float4 g = tcs::lds128(st + (uint32_t)r * (kTileM * 4) + (uint32_t)lane * 16);
+                float4 o;
+                o.x = fmaf(mx.ngamma, g.x, acc[u].x); o.y = fmaf(mx.ngamma, g.y, acc[u].y);
+                o.z = fmaf(mx.ngamma, g.z, acc[u].z); o.w = fmaf(mx.ngamma, g.w, acc[u].w);
+                __stcs(reinterpret_cast<float4*>(out + (int64_t)r * din), o);
+            }
+        }
+    }
+}
+
+struct Item { int node, m0, t0, t1; };      // node < 0: past the end of a short last node range
+// Items this CTA walks (including the empty ones of a short last node range).
+__device__ __forceinline__ int cta_items(const Args& g) {
+    const int b = (int)blockIdx.x, grid = (int)gridDim.x;
+    return b < g.total_seqs ? ((g.total_seqs - b + grid - 1) / grid) * g.split_len : 0;
+}
+// The i-th item of this CTA.
+__device__ __forceinline__ Item cta_item(const Args& g, int i) {
+    const int round = i / g.split_len, j = i - round * g.split_len;
+    const int seq = (int)blockIdx.x + round * (int)gridDim.x;
+    const int per_split = g.m_tiles * g.chunks;
+    const int sp = seq / per_split, rem = seq - sp * per_split;
     const int mt = rem / g.chunks, ch = rem - mt * g.chunks;
+    Item w;
+    w.node = sp * g.split_len + j;
+    if (w.node >= g.nodes) w.node = -1;
     w.m0 = mt * kTileM;
     w.t0 = ch * g.chunk;
     w.t1 = min(g.n_tiles, w.t0 + g.chunk);
@@ -86,12 +203,13 @@ __device__ __forceinline__ Item decode(const Args& g, int item) {
 
 // NT = column tile / 16 (16, 32 or 64 output units per tile); PRECISE: three split MMAs per product.
 // mapA: h as (m, k, node), box 128 x 64.  mapB: delta as (n, k, node), box 16 NT x 64.  mapC: the
-// gradient block as (m, n, node), box 128 x 16 NT.
+// gradient block as (m, n, node), box 128 x 16 NT (not used with FUSE).
 //
 // Tensor memory columns: [0, 128) two accumulators, then two converted h tiles of 64 heads +
 // 64 remainders each.
-template <int NT, bool PRECISE>
-__global__ void __launch_bounds__(kThreads, 1)
+// FUSE: see the head of this file; DEG is the common row degree of W (0 = read it per node).
+template <int NT, bool PRECISE, bool FUSE = false, int DEG = 0>
+__global__ void __launch_bounds__(FUSE ? kThreadsFused : kThreads, 1)
 tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                 const __grid_constant__ CUtensorMap mapC, Args g) {
     constexpr int ROWS_B = 16 * NT;
@@ -133,7 +251,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             mbar_init(a_conv_full + b, 128); mbar_init(a_conv_empty + b, 1);
             mbar_init(b_conv_full + b, 128); mbar_init(b_conv_empty + b, 1);
             mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, 128);
-            mbar_init(stage_free + b, 1); mbar_init(stage_ready + b, 128);
+            mbar_init(stage_free + b, FUSE ? 32 * kMixWarps : 1); mbar_init(stage_ready + b, 128);
         }
         for (int s = 0; s < kStagesB; ++s) { mbar_init(b_raw_full + s, 1); mbar_init(b_raw_empty + s, 128); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -147,22 +265,25 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    const int my_items = cta_items(g);
     bool ok = true;
 
     if (warp < 4) {
         // ------------------------------ epilogue: TMEM -> shared memory -> TMA store ------------------------------
         const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
         uint32_t q = 0;
-        for (int item = blockIdx.x; item < g.total_items && ok; item += gridDim.x) {
-            const Item w = decode(g, item);
+        for (int i = 0; i < my_items && ok; ++i) {
+            const Item w = cta_item(g, i);
+            if (w.node < 0) continue;
             for (int t = w.t0; t < w.t1; ++t, ++q) {
                 const uint32_t ab = q & 1u, ph = (q >> 1) & 1u;
                 const uint32_t st = stage + ab * STAGE;
-                if (tid == 0) {     // the store issued two tiles ago has finished reading this staging buffer
+                if (!FUSE && tid == 0) {     // the store issued two tiles ago has finished reading this staging buffer
                     asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                     mbar_arrive(stage_free + ab);
                 }
-                const bool go = mbar_wait(acc_full + ab, ph) && mbar_wait(stage_free + ab, ph);
+                // FUSE: the mixers arrive once they have consumed the tile staged here two tiles ago
+                const bool go = mbar_wait(acc_full + ab, ph) && mbar_wait(stage_free + ab, FUSE ? ph ^ 1u : ph);
                 if (!__all_sync(0xffffffffu, go)) { ok = false; break; }     // tcgen05.ld needs the whole warp
                 tc::tc_fence_after();
 #pragma unroll 1
@@ -174,6 +295,10 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 }
                 tc::tc_fence_before();
                 mbar_arrive(acc_empty + ab);                                 // the accumulator may be overwritten
+                if (FUSE) {
+                    mbar_arrive(stage_ready + ab);                           // handed to the mixer warps
+                    continue;
+                }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_arrive(stage_ready + ab);
                 if (tid == 0) {
@@ -193,8 +318,9 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         const uint32_t ct = (uint32_t)tid - 128u, cw = (uint32_t)warp - 4u;
         const uint32_t lane_base = tmem_base + ((cw * 32u) << 16);
         uint32_t q = 0, it = 0;
-        for (int item = blockIdx.x; item < g.total_items && ok; item += gridDim.x, ++it) {
-            const Item w = decode(g, item);
+        for (int i = 0; i < my_items && ok; ++i) {
+            const Item w = cta_item(g, i);
+            if (w.node < 0) continue;
             const uint32_t abuf = it & 1u;
             {   // h tile -> tensor memory: row ct of A is column ct of the raw [k][m] tile
                 const bool go = mbar_wait(a_raw_full, it & 1u) && mbar_wait(a_conv_empty + abuf, ((it >> 1) & 1u) ^ 1u);
@@ -239,6 +365,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 mbar_arrive(b_conv_full + bb);
                 mbar_arrive(b_raw_empty + s);
             }
+            ++it;
         }
         if (!ok && lane == 0) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
     }
@@ -248,8 +375,9 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(ROWS_B >> 3) << 17) |
                                    ((uint32_t)(kTileM >> 4) << 24);
             uint32_t q = 0, it = 0;
-            for (int item = blockIdx.x; item < g.total_items && ok; item += gridDim.x, ++it) {
-                const Item w = decode(g, item);
+            for (int i = 0; i < my_items && ok; ++i) {
+                const Item w = cta_item(g, i);
+                if (w.node < 0) continue;
                 const uint32_t abuf = it & 1u;
                 if (!mbar_wait(a_conv_full + abuf, (it >> 1) & 1u)) { ok = false; break; }
                 const uint32_t a_hi = tmem_base + A_COL0 + abuf * kACols, a_lo = a_hi + kMaxK;
@@ -273,14 +401,16 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                     tc::mma_commit(acc_full + bb);
                 }
                 if (ok) tc::mma_commit(a_conv_empty + abuf);     // every MMA that reads this h tile has been issued
+                ++it;
             }
             if (!ok) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
         }
-    } else if (lane == 0) {
+    } else if (warp == 9 && lane == 0) {
         // ------------------------------ TMA loads ------------------------------
         uint32_t q = 0, it = 0;                  // delta tiles and h tiles issued so far
-        for (int item = blockIdx.x; item < g.total_items && ok; item += gridDim.x) {
-            const Item w = decode(g, item);
+        for (int i = 0; i < my_items && ok; ++i) {
+            const Item w = cta_item(g, i);
+            if (w.node < 0) continue;
             if (!mbar_wait(a_raw_empty, (it & 1u) ^ 1u)) { ok = false; break; }
             mbar_expect_tx(a_raw_full, A_RAW);
             tma_load_3d(a_raw, &mapA, w.m0, 0, w.node, a_raw_full);
@@ -299,6 +429,38 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             mbar_wait(b_raw_full + qq % kStagesB, (qq / kStagesB) & 1u);
         }
         if (!ok) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
+    }
+    if (FUSE && warp >= 10) {
+        // ------------------------------ mixers: gossip step on staged tiles ------------------------------
+        const int mw = warp - 10;
+        uint32_t q = 0;
+        for (int i = 0; i < my_items && ok; ++i) {
+            const Item w = cta_item(g, i);
+            if (w.node < 0) continue;
+            // the next item of this CTA, when it is the next node of the same range
+            const int next_node = ((i + 1) % g.split_len != 0 && w.node + 1 < g.nodes) ? w.node + 1 : -1;
+            for (int t = w.t0; t < w.t1; ++t, ++q) {
+                const uint32_t ab = q & 1u, ph = (q >> 1) & 1u;
+                if (!mbar_wait(stage_ready + ab, ph)) { ok = false; break; }
+                if (next_node >= 0) {
+                    // The same tile position of the next node's neighbours, one 128-byte line per thread and
+                    // neighbour: whatever is not in L2 yet (for a ring, one tile of three) is on its way
+                    // before the gather of the next item asks for it.
+                    const int line = mw * 32 + lane, row = line >> 2, seg = line & 3;
+                    if (row < min(ROWS_B, g.N - t * ROWS_B) && w.m0 + seg * 32 < g.M) {
+                        const int64_t o = g.mix.w_off + (int64_t)(t * ROWS_B + row) * g.M + w.m0 + seg * 32;
+                        const int pe = __ldg(g.mix.row_ptr + next_node + 1);
+                        for (int p = __ldg(g.mix.row_ptr + next_node); p < pe; ++p)
+                            prefetch_l2(g.mix.X + (int64_t)__ldg(g.mix.col + p) * g.mix.ld + o);
+                    }
+                }
+                const int64_t off = g.mix.w_off + (int64_t)(t * ROWS_B) * g.M + w.m0 + lane * 4;
+                mix_rows<DEG, ROWS_B>(g.mix, w.node, stage + ab * STAGE, off, g.M, g.N - t * ROWS_B,
+                                      w.m0 + lane * 4 < g.M, mw, lane);
+                mbar_arrive(stage_free + ab);
+            }
+        }
+        if (!ok && lane == 0) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
     }
     tc::tc_fence_before();
     __syncthreads();

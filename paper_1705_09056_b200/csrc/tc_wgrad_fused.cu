@@ -1,0 +1,115 @@
+// Weight-gradient product of the MLP with the gossip step of Algorithm 1 (steps 4-5) applied in its
+// epilogue: for one weight block of every node,
+//
+//     X_next[i][block] = sum_j W_ij X[j][block] - gamma * (delta_i^T h_i)
+//
+// so this block of the stochastic gradient dF(X_k; xi_k) (Section 3) is consumed on chip and never
+// written to HBM.  The kernel is tc_wgrad_kernel<..., FUSE = true> of tc_wgrad.cuh; this file holds
+// its host side only.
+#include <algorithm>
+
+#include "ctx.h"
+#include "tc_wgrad.cuh"
+#include "tma_host.h"
+
+namespace dpsgd {
+namespace {
+
+constexpr int kFusedChunk = 2;       // column tiles per item of the fused kernel
+
+template <int NT, bool PRECISE, int DEG>
+cudaError_t launch(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap& mapB, const CUtensorMap& mapC, tcw::Args a) {
+    auto kernel = tcw::tc_wgrad_kernel<NT, PRECISE, true, DEG>;
+    constexpr size_t smem = tcw::smem_bytes<NT, PRECISE>();
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int sms = 0, dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    // An item is (node, 128-row block, run of `chunk` column tiles); a CTA walks a range of consecutive
+    // nodes at one position, so that the tiles of X it gathers for node i (its neighbours in W) are the
+    // ones it fetched for nodes i-1 and i-2: they come from L2 as long as the data all CTAs touch during
+    // two node steps fits there.  Short runs keep that window small; the price is one h tile converted
+    // per node and run.  Node ranges are chosen to fill whole waves of CTAs; each range re-reads the
+    // tiles just outside its ends (weighted here as one node step).
+    a.nodes = c->n;
+    a.chunk = std::min(a.n_tiles, kFusedChunk);
+    a.chunks = (a.n_tiles + a.chunk - 1) / a.chunk;
+    const long long positions = (long long)a.m_tiles * a.chunks;
+    double best = 0.0;
+    a.splits = 1; a.split_len = c->n;
+    for (int s = 1; s <= std::min(c->n, 256); ++s) {
+        const int len = (c->n + s - 1) / s;
+        const int used = (c->n + len - 1) / len;                 // ranges that hold nodes
+        if (used != s) continue;
+        const long long waves = (positions * s + sms - 1) / sms;
+        const double cost = (double)waves * (len + 1.0);
+        if (s == 1 || cost < best) { best = cost; a.splits = s; a.split_len = len; }
+    }
+    a.total_seqs = (int)(positions * a.splits);
+    const int grid = std::min(a.total_seqs, sms);                // one persistent CTA per SM
+    kernel<<<grid, tcw::kThreadsFused, smem, c->stream>>>(mapA, mapB, mapC, a);
+    c->launches++;
+    return cudaGetLastError();
+}
+
+template <int NT, bool PRECISE>
+cudaError_t launch_deg(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap& mapB, const CUtensorMap& mapC,
+                       const tcw::Args& a, int deg) {
+    switch (deg) {            // common row degree of W: ring 3, ring with one more link 4, torus 5
+        case 3: return launch<NT, PRECISE, 3>(c, mapA, mapB, mapC, a);
+        case 5: return launch<NT, PRECISE, 5>(c, mapA, mapB, mapC, a);
+        default: return launch<NT, PRECISE, 0>(c, mapA, mapB, mapC, a);
+    }
+}
+
+}  // namespace
+
+bool fused_step_supported(const dpsgd_ctx* c) {
+    return c->model == DPSGD_MODEL_MLP && !c->swapped && c->V == nullptr && c->mlp_precision != 2 &&
+           c->batch <= tcw::kMaxK && c->W.max_deg >= 1 && c->W.max_deg <= kFusedMaxDegree;
+}
+
+// Where the fused kernel is faster than the two stages (measured on B200): the stacked weight block
+// does not fit L2, so the separate gossip pass would stream it from HBM, and rows of W are as short as
+// a ring's, so the gather stays cheap.  Smaller problems are L2-resident either way.
+bool fused_step_pays(const dpsgd_ctx* c, int din, int dout) {
+    const double block_bytes = (double)c->n * din * dout * sizeof(float);
+    return c->W.max_deg <= 3 && block_bytes >= 512.0 * 1024 * 1024;
+}
+
+// Returns cudaErrorNotSupported when the shapes or alignments rule the kernel out (the caller then
+// writes this block of G and leaves it to the mixing kernel).
+cudaError_t run_tcw_fused(dpsgd_ctx* c, const float* h, int din, const float* delta, int dout, int dpitch,
+                          int64_t w_off, const float* X, float* Xn) {
+    const int B = c->batch;
+    auto al = [](const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; };
+    if (B > tcw::kMaxK || din % 4 != 0 || dpitch % 4 != 0 || w_off % 4 != 0 || c->ld % 4 != 0 || !al(h) || !al(delta) ||
+        !al(X) || !al(Xn))
+        return cudaErrorNotSupported;
+    const int rows_b = dout <= 16 ? 16 : (dout <= 32 ? 32 : 64);
+    const uint64_t nodes = (uint64_t)c->n;
+    CUtensorMap mapA, mapB, mapC;
+    bool ok = make_map_3d(&mapA, h, (uint64_t)din, (uint64_t)B, nodes, (uint64_t)din * 4, (uint64_t)B * din * 4,
+                          tcw::kTileM, tcw::kMaxK, false);
+    ok = ok && make_map_3d(&mapB, delta, (uint64_t)dout, (uint64_t)B, nodes, (uint64_t)dpitch * 4,
+                           (uint64_t)B * dpitch * 4, (uint32_t)rows_b, tcw::kMaxK, false);
+    mapC = mapA;              // the fused kernel issues no TMA store; the parameter only keeps the signature
+    if (!ok) return cudaErrorNotSupported;
+    tcw::Args a{};
+    a.M = din; a.N = dout; a.K = B;
+    a.m_tiles = (din + tcw::kTileM - 1) / tcw::kTileM;
+    a.n_tiles = (dout + rows_b - 1) / rows_b;
+    a.status = &c->d_result->status;
+    a.mix.X = X; a.mix.Xn = Xn; a.mix.ld = c->ld; a.mix.w_off = w_off;
+    a.mix.row_ptr = c->W.row_ptr; a.mix.col = c->W.col; a.mix.val = c->W.val; a.mix.ngamma = -c->gamma;
+    const int deg = c->W.uniform_deg;
+    const bool precise = c->mlp_precision == 0;
+    switch (rows_b) {
+        case 16: return precise ? launch_deg<1, true>(c, mapA, mapB, mapC, a, deg) : launch_deg<1, false>(c, mapA, mapB, mapC, a, deg);
+        case 32: return precise ? launch_deg<2, true>(c, mapA, mapB, mapC, a, deg) : launch_deg<2, false>(c, mapA, mapB, mapC, a, deg);
+        default: return precise ? launch_deg<4, true>(c, mapA, mapB, mapC, a, deg) : launch_deg<4, false>(c, mapA, mapB, mapC, a, deg);
+    }
+}
+
+}  // namespace dpsgd

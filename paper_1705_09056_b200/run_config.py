@@ -27,6 +27,9 @@ def main():
     ap.add_argument("--fused-consensus", action="store_true",
                     help="log the consensus distance every step from inside the gossip kernel")
     ap.add_argument("--swapped", action="store_true", help="footnote c: update locally, then average")
+    ap.add_argument("--fused-step", type=int, default=0, nargs="?", const=1,
+                    help="MLP: gossip step inside the weight-gradient kernels (those blocks of G are never "
+                         "written): 1 where it is faster, 2 wherever the kernel applies")
     args = ap.parse_args()
 
     build.build()
@@ -56,11 +59,13 @@ def main():
         torch.cuda.synchronize()
         return a.elapsed_time(b) / reps
 
+    if args.swapped:
+        ctx.set_order(True)
+    if args.fused_step:
+        ctx.set_fused_step(args.fused_step)
     for k in range(args.warmup):
         ctx.step(k)
     l0 = ctx.launch_count()
-    if args.swapped:
-        ctx.set_order(True)
     log = torch.zeros(args.steps + args.warmup + 8, dtype=torch.float64, device=dev)
     if args.fused_consensus:
         def whole(k):
@@ -86,7 +91,7 @@ def main():
     ms_mix = timed(lambda k: ctx.mix_update(), max(3, args.steps // 5))
     print(json.dumps({
         "workload": w.name, "n": w.n, "N": w.N, "dims": list(w.dims), "batch": w.batch, "topology": w.topology,
-        "mix_kernel": binding.MIX_NAMES[ctx.mix_kind()], "ms_per_step": ms_step, "ms_per_step_one_call": ms_run,
+        "fused_step": args.fused_step, "mix_kernel": binding.MIX_NAMES[ctx.mix_kind()], "ms_per_step": ms_step, "ms_per_step_one_call": ms_run,
         "replica_steps_per_s": w.n / (ms_step * 1e-3), "ms_grad": ms_grad, "ms_mix_update": ms_mix,
         "launches_per_step": launches, "consensus": ctx.consensus_dist()}))
     ctx.close()
