@@ -493,7 +493,7 @@ DPSGD_API dpsgd_status dpsgd_step_consensus(dpsgd_ctx* c, uint64_t k, double* ou
 DPSGD_API dpsgd_status dpsgd_set_fused_step(dpsgd_ctx* c, int32_t on) {
     if (!c) return DPSGD_ERR_ARG;
     drop_graph(c);
-    if (on < 0 || on > 2) return fail(c, DPSGD_ERR_ARG, "mode must be 0, 1 or 2");
+    if (on < 0 || on > 3) return fail(c, DPSGD_ERR_ARG, "mode must be 0, 1, 2 or 3");
     c->fuse_step = on;
     return DPSGD_OK;
 }

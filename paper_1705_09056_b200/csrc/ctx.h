@@ -144,6 +144,8 @@ cudaError_t launch_grad_linear(dpsgd_ctx* c, uint64_t k, const float* X, float* 
 cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G, float* Xn = nullptr);
 bool fused_step_supported(const dpsgd_ctx* c);
 bool fused_step_pays(const dpsgd_ctx* c, int din, int dout);
+cudaError_t run_tcw_ring(dpsgd_ctx* c, const float* h, int din, const float* delta, int dout, int dpitch,
+                         int64_t w_off, const float* X, float* Xn);
 cudaError_t run_tcw_fused(dpsgd_ctx* c, const float* h, int din, const float* delta, int dout, int dpitch,
                           int64_t w_off, const float* X, float* Xn);
 // Gossip step on the columns of [0, ld) outside c->fused_blocks.

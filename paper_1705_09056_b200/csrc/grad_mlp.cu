@@ -500,7 +500,8 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G, 
                 a.M = din; a.N = dout; a.K = B; a.epi = tc::EPI_STORE;
                 cudaError_t e = cudaErrorNotSupported;
                 if (Xn && (c->fuse_step >= 2 || fused_step_pays(c, din, dout))) {   // gossip step applied in the product's epilogue: this block goes straight to X_next
-                    e = run_tcw_fused(c, g.Bm, din, delta, dout, dp, s.w_off[l - 1], X, Xn);
+                    if (c->fuse_step != 3) e = run_tcw_ring(c, g.Bm, din, delta, dout, dp, s.w_off[l - 1], X, Xn);
+                    if (e == cudaErrorNotSupported) e = run_tcw_fused(c, g.Bm, din, delta, dout, dp, s.w_off[l - 1], X, Xn);
                     if (e == cudaSuccess) c->fused_blocks.emplace_back(s.w_off[l - 1], s.w_off[l - 1] + (int64_t)dout * din);
                 }
                 if (e == cudaErrorNotSupported) e = run_tcw(c, g.Bm, din, delta, dout, dp, g.C);

@@ -51,11 +51,14 @@ using tcs::tma_load_3d;
 constexpr int kThreads = 320;        // 4 epilogue warps, 4 converter warps, MMA warp, TMA warp
 constexpr int kMixWarps = 16;        // FUSE only: warps 10..25 apply the gossip step to staged tiles
 constexpr int kThreadsFused = kThreads + 32 * kMixWarps;
+constexpr int kThreadsRing = 704;    // kRing: converters, MMA, TMA as above; warps 0-3 and 10-21 mix
+enum { kStore = 0, kGather = 1, kRing = 2 };
 constexpr int kTileM = 128;
 constexpr int kMaxK = 64;            // minibatch rows a raw tile holds
 constexpr int kStagesB = 3;
 constexpr uint32_t kAccStride = 64;  // TMEM columns per accumulator
 constexpr uint32_t kACols = 2 * kMaxK;   // heads, then remainders
+constexpr uint32_t A_COL0_ = 2 * kAccStride;   // first tensor-memory column of the converted h tiles
 
 // What the fused gossip epilogue needs: the stacked X of this iteration, the buffer of the next one,
 // where this weight block starts inside a parameter row, W in CSR and -gamma.
@@ -66,6 +69,7 @@ struct Mix {
     const int32_t* row_ptr;
     const int32_t* col;
     const float* val;
+    const float* band;               // kRing: [n][3] = (W_{i,i-1}, W_ii, W_{i,i+1})
     float ngamma;
 };
 
@@ -91,10 +95,12 @@ __host__ __device__ constexpr uint32_t b_lbo(int rows) { return (uint32_t)rows *
 __host__ __device__ constexpr uint32_t b_conv_bytes(int rows) { return (kMaxK / 4) * b_lbo(rows); }
 __host__ __device__ constexpr uint32_t stage_bytes(int rows) { return (uint32_t)rows * kTileM * 4; }
 
-template <int NT, bool PRECISE>
+// STAGED: two staging buffers for the output tile and one raw h tile; otherwise (kRing) no staging
+// and two raw h tiles.
+template <int NT, bool PRECISE, bool STAGED = true>
 constexpr size_t smem_bytes() {
-    return 1024 + a_raw_bytes() + kStagesB * b_raw_bytes(16 * NT) + 2 * (PRECISE ? 2 : 1) * b_conv_bytes(16 * NT) +
-           2 * stage_bytes(16 * NT) + 256;
+    return 1024 + (STAGED ? 1 : 2) * a_raw_bytes() + kStagesB * b_raw_bytes(16 * NT) + 2 * (PRECISE ? 2 : 1) * b_conv_bytes(16 * NT) +
+           (STAGED ? 2 * stage_bytes(16 * NT) : 0) + 256;
 }
 
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
@@ -207,9 +213,10 @@ __device__ __forceinline__ Item cta_item(const Args& g, int i) {
 //
 // Tensor memory columns: [0, 128) two accumulators, then two converted h tiles of 64 heads +
 // 64 remainders each.
-// FUSE: see the head of this file; DEG is the common row degree of W (0 = read it per node).
-template <int NT, bool PRECISE, bool FUSE = false, int DEG = 0>
-__global__ void __launch_bounds__(FUSE ? kThreadsFused : kThreads, 1)
+// MODE: kStore, kGather or kRing (see the head of this file); DEG is the common row degree of W for
+// kGather (0 = read it per node).
+template <int NT, bool PRECISE, int MODE = kStore, int DEG = 0>
+__global__ void __launch_bounds__(MODE == kGather ? kThreadsFused : (MODE == kRing ? kThreadsRing : kThreads), 1)
 tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                 const __grid_constant__ CUtensorMap mapC, Args g) {
     constexpr int ROWS_B = 16 * NT;
@@ -217,22 +224,25 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     constexpr uint32_t B_CONV = b_conv_bytes(ROWS_B), B_LBO = b_lbo(ROWS_B), SBO = 128;
     constexpr uint32_t NCOPY = PRECISE ? 2 : 1;
     constexpr uint32_t CONV_BUF = NCOPY * B_CONV;
-    constexpr uint32_t STAGE = stage_bytes(ROWS_B);
-    constexpr uint32_t A_COL0 = 2 * kAccStride;
+    constexpr bool FUSE = MODE == kGather;
+    constexpr uint32_t STAGE = MODE == kRing ? 0u : stage_bytes(ROWS_B);
+    constexpr uint32_t WIN_COL0 = A_COL0_ + 2 * kACols;      // kRing: two 64-column slots of the X window
+    constexpr uint32_t A_COL0 = A_COL0_;
     constexpr uint32_t TMEM_COLS = 512;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    constexpr uint32_t A_BUFS = MODE == kRing ? 2u : 1u;     // raw h tiles in flight (a new one every column tile in kRing)
     const uint32_t a_raw = base;
-    const uint32_t b_raw = a_raw + A_RAW;
+    const uint32_t b_raw = a_raw + A_BUFS * A_RAW;
     const uint32_t b_conv = b_raw + kStagesB * B_RAW;
     const uint32_t stage = b_conv + 2 * CONV_BUF;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + A_RAW + kStagesB * B_RAW + 2 * CONV_BUF + 2 * STAGE);
-    uint64_t* a_raw_full = bars;                 // 1
-    uint64_t* a_raw_empty = bars + 1;            // 1
-    uint64_t* a_conv_full = bars + 2;            // [2]
-    uint64_t* a_conv_empty = bars + 4;           // [2]
-    uint64_t* b_raw_full = bars + 6;             // [kStagesB]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + A_BUFS * A_RAW + kStagesB * B_RAW + 2 * CONV_BUF + 2 * STAGE);
+    uint64_t* a_raw_full = bars;                 // [A_BUFS]
+    uint64_t* a_raw_empty = bars + 2;            // [A_BUFS]
+    uint64_t* a_conv_full = bars + 4;            // [2]
+    uint64_t* a_conv_empty = bars + 6;           // [2]
+    uint64_t* b_raw_full = bars + 8;             // [kStagesB]
     uint64_t* b_raw_empty = b_raw_full + kStagesB;
     uint64_t* b_conv_full = b_raw_empty + kStagesB;   // [2]
     uint64_t* b_conv_empty = b_conv_full + 2;    // [2]
@@ -246,11 +256,11 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     const int KS = (g.K + 7) / 8;                // MMAs (k = 8) per product and column tile
 
     if (tid == 0) {
-        mbar_init(a_raw_full, 1); mbar_init(a_raw_empty, 128);
+        for (uint32_t b = 0; b < A_BUFS; ++b) { mbar_init(a_raw_full + b, 1); mbar_init(a_raw_empty + b, 128); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(a_conv_full + b, 128); mbar_init(a_conv_empty + b, 1);
             mbar_init(b_conv_full + b, 128); mbar_init(b_conv_empty + b, 1);
-            mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, 128);
+            mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, MODE == kRing ? 16 : 128);
             mbar_init(stage_free + b, FUSE ? 32 * kMixWarps : 1); mbar_init(stage_ready + b, 128);
         }
         for (int s = 0; s < kStagesB; ++s) { mbar_init(b_raw_full + s, 1); mbar_init(b_raw_empty + s, 128); }
@@ -268,7 +278,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     const int my_items = cta_items(g);
     bool ok = true;
 
-    if (warp < 4) {
+    if (MODE != kRing && warp < 4) {
         // ------------------------------ epilogue: TMEM -> shared memory -> TMA store ------------------------------
         const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
         uint32_t q = 0;
@@ -313,7 +323,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         }
         if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores complete before exit
         if (!ok && lane == 0) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
-    } else if (warp < 8) {
+    } else if (warp >= 4 && warp < 8) {
         // ------------------------------ converters ------------------------------
         const uint32_t ct = (uint32_t)tid - 128u, cw = (uint32_t)warp - 4u;
         const uint32_t lane_base = tmem_base + ((cw * 32u) << 16);
@@ -323,7 +333,9 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             if (w.node < 0) continue;
             const uint32_t abuf = it & 1u;
             {   // h tile -> tensor memory: row ct of A is column ct of the raw [k][m] tile
-                const bool go = mbar_wait(a_raw_full, it & 1u) && mbar_wait(a_conv_empty + abuf, ((it >> 1) & 1u) ^ 1u);
+                const uint32_t rbuf = it % A_BUFS, a_tile = a_raw + rbuf * A_RAW;
+                const bool go = mbar_wait(a_raw_full + rbuf, (it / A_BUFS) & 1u) &&
+                                mbar_wait(a_conv_empty + abuf, ((it >> 1) & 1u) ^ 1u);
                 if (!__all_sync(0xffffffffu, go)) { ok = false; break; }     // tcgen05.st needs the whole warp
                 tc::tc_fence_after();
                 const uint32_t a_cols = lane_base + A_COL0 + abuf * kACols;
@@ -332,7 +344,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                     uint32_t hi[16], lo[16];
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
-                        const float v = lds32(a_raw + (uint32_t)(k0 + k) * (kTileM * 4) + ct * 4);
+                        const float v = lds32(a_tile + (uint32_t)(k0 + k) * (kTileM * 4) + ct * 4);
                         if (PRECISE) tcs::split(v, hi[k], lo[k]);
                         else hi[k] = __float_as_uint(v);
                     }
@@ -342,7 +354,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc::tc_fence_before();
                 mbar_arrive(a_conv_full + abuf);
-                mbar_arrive(a_raw_empty);
+                mbar_arrive(a_raw_empty + rbuf);
             }
             for (int t = w.t0; t < w.t1; ++t, ++q) {
                 const uint32_t s = q % kStagesB, bb = q & 1u;
@@ -411,9 +423,10 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         for (int i = 0; i < my_items && ok; ++i) {
             const Item w = cta_item(g, i);
             if (w.node < 0) continue;
-            if (!mbar_wait(a_raw_empty, (it & 1u) ^ 1u)) { ok = false; break; }
-            mbar_expect_tx(a_raw_full, A_RAW);
-            tma_load_3d(a_raw, &mapA, w.m0, 0, w.node, a_raw_full);
+            const uint32_t rbuf = it % A_BUFS;
+            if (!mbar_wait(a_raw_empty + rbuf, ((it / A_BUFS) & 1u) ^ 1u)) { ok = false; break; }
+            mbar_expect_tx(a_raw_full + rbuf, A_RAW);
+            tma_load_3d(a_raw + rbuf * A_RAW, &mapA, w.m0, 0, w.node, a_raw_full + rbuf);
             ++it;
             for (int t = w.t0; t < w.t1; ++t, ++q) {
                 const uint32_t s = q % kStagesB;
@@ -423,12 +436,107 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             }
         }
         // loads still in flight (only when somebody gave up): let them land before the CTA leaves
-        if (it > 0) mbar_wait(a_raw_full, (it - 1) & 1u);
+        for (uint32_t j = 0; j < A_BUFS && j < it; ++j) {
+            const uint32_t ii = it - 1 - j;
+            mbar_wait(a_raw_full + ii % A_BUFS, (ii / A_BUFS) & 1u);
+        }
         for (uint32_t j = 0; j < (uint32_t)kStagesB && j < q; ++j) {
             const uint32_t qq = q - 1 - j;
             mbar_wait(b_raw_full + qq % kStagesB, (qq / kStagesB) & 1u);
         }
         if (!ok) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
+    }
+    if (MODE == kRing && (warp < 4 || warp >= 10)) {
+        // ------------------------------ ring mixers: X window in tensor memory ------------------------------
+        // Thread = (row m of the tile, 16 of its 64 columns): the accumulator's own layout, so a tile needs
+        // no staging.  The CTA walks consecutive nodes i at one tile position; the tiles of X_{i-1} and X_i
+        // are kept in two 64-column slots of tensor memory (each thread's own lane and columns: no
+        // synchronisation), so only X_{i+1} is read from memory - one read of X per element - and its
+        // loads for the next node are issued before this node is finished.
+        // sixteen warps: lane quarter warp % 4 (the lanes a warp may address), column group by warp:
+        // 0-3 -> 0, 12-15 -> 1, 16-19 -> 2, {20, 21, 10, 11} -> 3
+        const int quarter = warp & 3, cg = warp < 4 ? 0 : (warp < 12 || warp >= 20 ? 3 : ((warp - 12) >> 2) + 1);
+        const int m = quarter * 32 + lane;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const uint32_t win[2] = {lane_addr + WIN_COL0 + (uint32_t)cg * 16, lane_addr + WIN_COL0 + 64 + (uint32_t)cg * 16};
+        const int64_t cstride = g.M;                         // one output unit further = din elements further
+        auto load16 = [&](const float* p, int ncols, float (&v)[16]) {
+            if (ncols == 16) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = __ldcg(p + j * cstride);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = j < ncols ? __ldcg(p + j * cstride) : 0.f;
+            }
+        };
+        const int rounds = my_items / g.split_len;
+        const int per_split = g.m_tiles * g.chunks;
+        uint32_t q = 0;
+        for (int rd = 0; rd < rounds && ok; ++rd) {
+            // one node range at one tile position (decoded as in cta_item; chunk == 1: one column tile)
+            const int seq = (int)blockIdx.x + rd * (int)gridDim.x;
+            const int sp = seq / per_split, rem = seq - sp * per_split;
+            const int mt = rem / g.chunks, t = rem - mt * g.chunks;
+            const int n0 = sp * g.split_len, n1 = min(g.nodes, n0 + g.split_len);
+            const int m0 = mt * kTileM, c0 = t * ROWS_B + cg * 16;
+            const int ncols = m0 + m < g.M ? max(0, min(16, g.N - c0)) : 0;
+            const int64_t pos = g.mix.w_off + (int64_t)c0 * g.M + m0 + m;
+            const float* xpos = g.mix.X + pos;
+            float* opos = g.mix.Xn + pos;
+            float xr[16], xn[16];
+            for (int node = n0; node < n1; ++node, ++q) {
+                const bool cold = node == n0;                // first node of the range: nothing kept yet
+                const float wl = __ldg(g.mix.band + 3 * node), ws = __ldg(g.mix.band + 3 * node + 1),
+                            wr = __ldg(g.mix.band + 3 * node + 2);
+                // r starts as X_{i+1} (raw, it goes into the window first) and is accumulated in place
+                float tmp[16];
+                uint32_t bits[16];
+                const uint32_t jj = (uint32_t)(node - n0);
+                if (cold) {
+                    load16(xpos + (int64_t)(node + 1 == g.nodes ? 0 : node + 1) * g.mix.ld, ncols, xr);
+                    load16(xpos + (int64_t)(node == 0 ? g.nodes - 1 : node - 1) * g.mix.ld, ncols, tmp);
+                }
+                if (node + 1 < n1)        // the next node's X_{i+1}: in flight while this node is mixed
+                    load16(xpos + (int64_t)(node + 2 >= g.nodes ? node + 2 - g.nodes : node + 2) * g.mix.ld, ncols, xn);
+                if (!cold) tc::tmem_ld16(win[(jj - 1) & 1u], tmp);               // X_{i-1}
+#pragma unroll
+                for (int j = 0; j < 16; ++j) bits[j] = __float_as_uint(xr[j]);
+                tcs::tmem_st16(cold ? win[1] : win[(jj - 1) & 1u], bits);        // X_{i+1} takes its place
+#pragma unroll
+                for (int j = 0; j < 16; ++j) xr[j] = fmaf(wr, xr[j], wl * tmp[j]);
+                if (cold) {
+                    load16(xpos + (int64_t)node * g.mix.ld, ncols, tmp);         // X_i
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) bits[j] = __float_as_uint(tmp[j]);
+                    tcs::tmem_st16(win[0], bits);                                // the next node's left neighbour
+                } else {
+                    tc::tmem_ld16(win[jj & 1u], tmp);                            // X_i
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) xr[j] = fmaf(ws, tmp[j], xr[j]);
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                const uint32_t ab = q & 1u, ph = (q >> 1) & 1u;
+                const bool go = mbar_wait(acc_full + ab, ph);
+                if (!__all_sync(0xffffffffu, go)) { ok = false; break; }     // tcgen05.ld needs the whole warp
+                tc::tc_fence_after();
+                tc::tmem_ld16(lane_addr + ab * kAccStride + (uint32_t)cg * 16, tmp);
+                tc::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acc_empty + ab);                  // the accumulator may be overwritten
+                float* out = opos + (int64_t)node * g.mix.ld;
+                if (ncols == 16) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) __stcs(out + j * cstride, fmaf(g.mix.ngamma, tmp[j], xr[j]));
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (j < ncols) __stcs(out + j * cstride, fmaf(g.mix.ngamma, tmp[j], xr[j]));
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) xr[j] = xn[j];
+            }
+        }
+        if (!ok && lane == 0) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
     }
     if (FUSE && warp >= 10) {
         // ------------------------------ mixers: gossip step on staged tiles ------------------------------

@@ -17,9 +17,25 @@ namespace {
 
 constexpr int kFusedChunk = 2;       // column tiles per item of the fused kernel
 
+// Node ranges for the kernels that walk consecutive nodes at one tile position: whole waves of CTAs,
+// each range re-reading the tiles just outside its ends (weighted as one node step).
+void choose_ranges(tcw::Args& a, int n, int sms) {
+    const long long positions = (long long)a.m_tiles * a.chunks;
+    double best = 0.0;
+    a.splits = 1; a.split_len = n;
+    for (int s = 1; s <= std::min(n, 256); ++s) {
+        const int len = (n + s - 1) / s;
+        if ((n + len - 1) / len != s) continue;                  // ranges that would hold no node
+        const long long waves = (positions * s + sms - 1) / sms;
+        const double cost = (double)waves * (len + 1.0);
+        if (s == 1 || cost < best) { best = cost; a.splits = s; a.split_len = len; }
+    }
+    a.total_seqs = (int)(positions * a.splits);
+}
+
 template <int NT, bool PRECISE, int DEG>
 cudaError_t launch(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap& mapB, const CUtensorMap& mapC, tcw::Args a) {
-    auto kernel = tcw::tc_wgrad_kernel<NT, PRECISE, true, DEG>;
+    auto kernel = tcw::tc_wgrad_kernel<NT, PRECISE, tcw::kGather, DEG>;
     constexpr size_t smem = tcw::smem_bytes<NT, PRECISE>();
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -30,25 +46,32 @@ cudaError_t launch(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap& map
     // nodes at one position, so that the tiles of X it gathers for node i (its neighbours in W) are the
     // ones it fetched for nodes i-1 and i-2: they come from L2 as long as the data all CTAs touch during
     // two node steps fits there.  Short runs keep that window small; the price is one h tile converted
-    // per node and run.  Node ranges are chosen to fill whole waves of CTAs; each range re-reads the
-    // tiles just outside its ends (weighted here as one node step).
+    // per node and run.
     a.nodes = c->n;
     a.chunk = std::min(a.n_tiles, kFusedChunk);
     a.chunks = (a.n_tiles + a.chunk - 1) / a.chunk;
-    const long long positions = (long long)a.m_tiles * a.chunks;
-    double best = 0.0;
-    a.splits = 1; a.split_len = c->n;
-    for (int s = 1; s <= std::min(c->n, 256); ++s) {
-        const int len = (c->n + s - 1) / s;
-        const int used = (c->n + len - 1) / len;                 // ranges that hold nodes
-        if (used != s) continue;
-        const long long waves = (positions * s + sms - 1) / sms;
-        const double cost = (double)waves * (len + 1.0);
-        if (s == 1 || cost < best) { best = cost; a.splits = s; a.split_len = len; }
-    }
-    a.total_seqs = (int)(positions * a.splits);
+    choose_ranges(a, c->n, sms);
     const int grid = std::min(a.total_seqs, sms);                // one persistent CTA per SM
     kernel<<<grid, tcw::kThreadsFused, smem, c->stream>>>(mapA, mapB, mapC, a);
+    c->launches++;
+    return cudaGetLastError();
+}
+
+template <bool PRECISE>
+cudaError_t launch_ring(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap& mapB, tcw::Args a) {
+    auto kernel = tcw::tc_wgrad_kernel<4, PRECISE, tcw::kRing, 0>;
+    constexpr size_t smem = tcw::smem_bytes<4, PRECISE, false>();
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int sms = 0, dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    a.nodes = c->n;
+    a.chunk = 1;                                                 // the X window in tensor memory holds one tile position
+    a.chunks = a.n_tiles;
+    choose_ranges(a, c->n, sms);
+    const int grid = std::min(a.total_seqs, sms);                // one persistent CTA per SM
+    kernel<<<grid, tcw::kThreadsRing, smem, c->stream>>>(mapA, mapB, mapA, a);
     c->launches++;
     return cudaGetLastError();
 }
@@ -78,6 +101,32 @@ bool fused_step_pays(const dpsgd_ctx* c, int din, int dout) {
     return c->W.max_deg <= 3 && block_bytes >= 512.0 * 1024 * 1024;
 }
 
+// Ring W (Theorem 3's band): the kernel that keeps the X tiles of nodes i-1 and i in tensor memory
+// while it walks the nodes, so every element of X is read once.  Same contract as run_tcw_fused.
+cudaError_t run_tcw_ring(dpsgd_ctx* c, const float* h, int din, const float* delta, int dout, int dpitch,
+                         int64_t w_off, const float* X, float* Xn) {
+    const int B = c->batch;
+    auto al = [](const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; };
+    if (!c->can_ring || !c->W.band || c->n < 3 || B > tcw::kMaxK || din % 4 != 0 || dpitch % 4 != 0 || !al(h) || !al(delta))
+        return cudaErrorNotSupported;
+    const uint64_t nodes = (uint64_t)c->n;
+    CUtensorMap mapA, mapB;
+    bool ok = make_map_3d(&mapA, h, (uint64_t)din, (uint64_t)B, nodes, (uint64_t)din * 4, (uint64_t)B * din * 4,
+                          tcw::kTileM, tcw::kMaxK, false);
+    ok = ok && make_map_3d(&mapB, delta, (uint64_t)dout, (uint64_t)B, nodes, (uint64_t)dpitch * 4,
+                           (uint64_t)B * dpitch * 4, 64u, tcw::kMaxK, false);
+    if (!ok) return cudaErrorNotSupported;
+    tcw::Args a{};
+    a.M = din; a.N = dout; a.K = B;
+    a.m_tiles = (din + tcw::kTileM - 1) / tcw::kTileM;
+    a.n_tiles = (dout + 63) / 64;
+    a.status = &c->d_result->status;
+    a.mix.X = X; a.mix.Xn = Xn; a.mix.ld = c->ld; a.mix.w_off = w_off;
+    a.mix.row_ptr = c->W.row_ptr; a.mix.col = c->W.col; a.mix.val = c->W.val; a.mix.band = c->W.band;
+    a.mix.ngamma = -c->gamma;
+    return c->mlp_precision == 0 ? launch_ring<true>(c, mapA, mapB, a) : launch_ring<false>(c, mapA, mapB, a);
+}
+
 // Returns cudaErrorNotSupported when the shapes or alignments rule the kernel out (the caller then
 // writes this block of G and leaves it to the mixing kernel).
 cudaError_t run_tcw_fused(dpsgd_ctx* c, const float* h, int din, const float* delta, int dout, int dpitch,
@@ -102,7 +151,8 @@ cudaError_t run_tcw_fused(dpsgd_ctx* c, const float* h, int din, const float* de
     a.n_tiles = (dout + rows_b - 1) / rows_b;
     a.status = &c->d_result->status;
     a.mix.X = X; a.mix.Xn = Xn; a.mix.ld = c->ld; a.mix.w_off = w_off;
-    a.mix.row_ptr = c->W.row_ptr; a.mix.col = c->W.col; a.mix.val = c->W.val; a.mix.ngamma = -c->gamma;
+    a.mix.row_ptr = c->W.row_ptr; a.mix.col = c->W.col; a.mix.val = c->W.val; a.mix.band = c->W.band;
+    a.mix.ngamma = -c->gamma;
     const int deg = c->W.uniform_deg;
     const bool precise = c->mlp_precision == 0;
     switch (rows_b) {

@@ -29,6 +29,7 @@ def _perturbed(w, seed):
 
 
 FUSED_CASES = [
+    (7, "ring", (260, 200, 10), 40, 12),              # ranges of several nodes per CTA, ragged tiles both ways
     # n, topology, dims, m, B
     (5, "ring", (784, 1024, 10), 64, 32),             # the 784-1024-10 network
     (4, "ring", (132, 200, 70, 10), 50, 16),          # widths that are no multiples of the 128 x 64 tiles
@@ -42,8 +43,11 @@ FUSED_CASES = [
 ]
 
 
+@pytest.mark.parametrize("mode", [2, 3])      # 2: ring W on the kernel with the X window on chip; 3: the gathering kernel
 @pytest.mark.parametrize("n,topology,dims,m,B", FUSED_CASES)
-def test_fused_step_matches_oracle_and_two_stage_path(n, topology, dims, m, B):
+def test_fused_step_matches_oracle_and_two_stage_path(n, topology, dims, m, B, mode):
+    if mode == 3 and topology != "ring":
+        pytest.skip("same kernel as mode 2 for this W")
     w = wl.mlp_workload(n=n, dims=dims, m=m, batch=B, gamma=0.05, seed=21, topology=topology)
     X = _perturbed(w, 3)
     run, o = _setup(w, seed=5, X=X)
@@ -60,7 +64,7 @@ def test_fused_step_matches_oracle_and_two_stage_path(n, topology, dims, m, B):
         # the fused iteration from the same X, with G poisoned: weight blocks must not be read from it
         run.ctx.current()[:, :w.N] = torch.from_numpy(X).cuda()
         run.G.fill_(float("nan"))
-        run.ctx.set_fused_step(2)
+        run.ctx.set_fused_step(mode)
         run.ctx.step(k)
         got = run.x()
         assert np.isfinite(got).all()
@@ -109,7 +113,7 @@ def test_fused_mode_one_leaves_small_blocks_to_the_two_stage_path():
     assert np.array_equal(outs[0], outs[1])
     run, _ = _setup(w, seed=2, X=X)
     with pytest.raises(binding.DpsgdError) as e:
-        run.ctx.set_fused_step(3)
+        run.ctx.set_fused_step(4)
     assert e.value.status == binding.ERR_ARG
     run.close()
 
