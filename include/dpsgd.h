@@ -150,9 +150,13 @@ DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* ctx, int32_t update_then_mix);
  * take the gossip step from there.  The result equals dpsgd_grad + dpsgd_mix_update up to fp32
  * rounding order.
  *   mode 0  off (default): two stages.
- *   mode 1  fused for the weight blocks where it is faster on B200: rows of W with at most 3 entries
- *           (a ring) and a stacked block of at least 512 MB (beyond L2); other blocks in two stages.
- *   mode 2  fused for every block the kernel can take.
+ *   mode 1  fused for the weight blocks where it is faster on B200: a ring W (Theorem 3) and a stacked
+ *           block of at least 64 MB, or rows of W with at most 3 entries and a stacked block of at
+ *           least 512 MB (far beyond L2); other blocks in two stages.
+ *   mode 2  fused for every block a fused kernel can take.  A ring W takes the kernel that keeps the
+ *           tiles of X_{i-1} and X_i on chip while it walks the nodes (X is read once); any other W
+ *           the kernel that gathers the neighbours' tiles through L2.
+ *   mode 3  as mode 2, but the gathering kernel for a ring W too (for comparison).
  * The kernel applies when the model is the MLP on the tensor-core path (minibatch <= 64, layer input
  * widths multiples of 4), the printed order of Algorithm 1 is in force, no momentum is set and no row
  * of W has more than 8 entries; otherwise dpsgd_step() runs the two stages whatever the mode.

@@ -451,8 +451,8 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         // Thread = (row m of the tile, 16 of its 64 columns): the accumulator's own layout, so a tile needs
         // no staging.  The CTA walks consecutive nodes i at one tile position; the tiles of X_{i-1} and X_i
         // are kept in two 64-column slots of tensor memory (each thread's own lane and columns: no
-        // synchronisation), so only X_{i+1} is read from memory - one read of X per element - and its
-        // loads for the next node are issued before this node is finished.
+        // synchronisation), so only X_{i+1} is read from memory - one read of X per element - after an L2
+        // prefetch two nodes ahead.
         // sixteen warps: lane quarter warp % 4 (the lanes a warp may address), column group by warp:
         // 0-3 -> 0, 12-15 -> 1, 16-19 -> 2, {20, 21, 10, 11} -> 3
         const int quarter = warp & 3, cg = warp < 4 ? 0 : (warp < 12 || warp >= 20 ? 3 : ((warp - 12) >> 2) + 1);
@@ -483,27 +483,27 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             const int64_t pos = g.mix.w_off + (int64_t)c0 * g.M + m0 + m;
             const float* xpos = g.mix.X + pos;
             float* opos = g.mix.Xn + pos;
-            float xr[16], xn[16];
             for (int node = n0; node < n1; ++node, ++q) {
                 const bool cold = node == n0;                // first node of the range: nothing kept yet
                 const float wl = __ldg(g.mix.band + 3 * node), ws = __ldg(g.mix.band + 3 * node + 1),
                             wr = __ldg(g.mix.band + 3 * node + 2);
-                // r starts as X_{i+1} (raw, it goes into the window first) and is accumulated in place
-                float tmp[16];
+                float xr[16], tmp[16];
                 uint32_t bits[16];
                 const uint32_t jj = (uint32_t)(node - n0);
-                if (cold) {
-                    load16(xpos + (int64_t)(node + 1 == g.nodes ? 0 : node + 1) * g.mix.ld, ncols, xr);
-                    load16(xpos + (int64_t)(node == 0 ? g.nodes - 1 : node - 1) * g.mix.ld, ncols, tmp);
+                // X_{i+1}: the one tile read from memory; it was requested into L2 two nodes ago
+                load16(xpos + (int64_t)(node + 1 == g.nodes ? 0 : node + 1) * g.mix.ld, ncols, xr);
+                if (node + 2 < n1 && lane < ncols) {
+                    // lane j asks for the line that holds column j of the tile of X_{i+3} (this warp's 32 rows)
+                    const int ahead = node + 3 >= g.nodes ? node + 3 - g.nodes : node + 3;
+                    prefetch_l2(xpos - lane + (int64_t)ahead * g.mix.ld + lane * cstride);
                 }
-                if (node + 1 < n1)        // the next node's X_{i+1}: in flight while this node is mixed
-                    load16(xpos + (int64_t)(node + 2 >= g.nodes ? node + 2 - g.nodes : node + 2) * g.mix.ld, ncols, xn);
-                if (!cold) tc::tmem_ld16(win[(jj - 1) & 1u], tmp);               // X_{i-1}
+                if (cold) load16(xpos + (int64_t)(node == 0 ? g.nodes - 1 : node - 1) * g.mix.ld, ncols, tmp);
+                else tc::tmem_ld16(win[(jj - 1) & 1u], tmp);                     // X_{i-1}
 #pragma unroll
                 for (int j = 0; j < 16; ++j) bits[j] = __float_as_uint(xr[j]);
                 tcs::tmem_st16(cold ? win[1] : win[(jj - 1) & 1u], bits);        // X_{i+1} takes its place
 #pragma unroll
-                for (int j = 0; j < 16; ++j) xr[j] = fmaf(wr, xr[j], wl * tmp[j]);
+                for (int j = 0; j < 16; ++j) xr[j] = fmaf(wr, xr[j], wl * tmp[j]);   // accumulated in place
                 if (cold) {
                     load16(xpos + (int64_t)node * g.mix.ld, ncols, tmp);         // X_i
 #pragma unroll
@@ -532,8 +532,6 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                     for (int j = 0; j < 16; ++j)
                         if (j < ncols) __stcs(out + j * cstride, fmaf(g.mix.ngamma, tmp[j], xr[j]));
                 }
-#pragma unroll
-                for (int j = 0; j < 16; ++j) xr[j] = xn[j];
             }
         }
         if (!ok && lane == 0) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
