@@ -159,6 +159,45 @@ def time_steps(ctx, steps, warmup, torch):
     return a.elapsed_time(b) / steps    # ms per step == per launch (one kernel per step)
 
 
+def whole_iterations(torch, binding, wl, dev, steps=20, warmup=3):
+    """Whole D-PSGD iterations (sample + gradient + mix + update; consensus distance read once at the end)
+    on the two MLP configurations, two-stage and with the gossip step inside the gradient kernels.
+    Context for the headline line, which times the gossip step alone."""
+    out = {}
+    for name, idx in (("mlp_784-1024-10_n32_ring", 2), ("mlp_1024-2048-2048-10_n112_ring", 4)):
+        w = wl.config(idx, device=dev)
+        X0 = wl.stack_rows(w.x0, w.n, w.ld)
+        X1, G = torch.zeros_like(X0), torch.zeros_like(X0)
+        log = torch.zeros(steps + warmup, dtype=torch.float64, device=dev)
+        res = {"n": w.n, "N": w.N, "batch": w.batch}
+        for label, mode in (("two_stage", 0), ("fused", 1)):
+            X0.copy_(wl.stack_rows(w.x0, w.n, w.ld))
+            ctx = binding.Dpsgd(w.n, w.N, *w.csr(), gamma=w.gamma, seed=1)
+            ctx.bind(X0, X1, G)
+            ctx.set_model(w.model, w.dims, w.l2_lambda, w.batch, 0)
+            ctx.set_data(w.A, w.y)
+            ctx.set_fused_step(mode)
+            for k in range(warmup):
+                ctx.step(k)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            l0 = ctx.launch_count()
+            a.record()
+            for k in range(steps):
+                ctx.step(warmup + k)
+            b.record()
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / steps
+            res[label] = {"ms_per_step": ms, "replica_steps_per_s": w.n / (ms * 1e-3),
+                          "launches_per_step": (ctx.launch_count() - l0) / steps,
+                          "consensus_dist": ctx.consensus_dist()}
+            ctx.close()
+        out[name] = res
+        del X0, X1, G, w
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -276,6 +315,12 @@ def run_ours(args):
                "sample": f"one step on the first {cols} of {N} columns of all {n} rows "
                          "(separable per column), scaled linearly to a full step"}
 
+    iterations = None
+    if world == 1 and not args.no_iterations:
+        del X0, X1, G
+        torch.cuda.empty_cache()
+        iterations = whole_iterations(torch, binding, wl, dev)
+
     ring = results["ring"]
     line = {
         "metric": METRIC, "value": aggregate_throughput(n, world, ring["ms_per_step"]), "unit": "replica-steps/s",
@@ -287,7 +332,7 @@ def run_ours(args):
                      "peak_source": f"{peak_kind} HBM copy bandwidth (GB/s)", "unit": "GB/s",
                      "frac": ring["GBps"] / peak, "frac_of_nominal_8TBps": ring["GBps"] / NOMINAL_HBM_GBS,
                      "algorithmic_bytes_per_launch": bytes_per_launch, "traffic": TRAFFIC_BYTES_PER_LAUNCH},
-        "cpu_baseline": cpu, "topologies": results,
+        "cpu_baseline": cpu, "topologies": results, "iterations": iterations,
     }
     print(json.dumps(line))
     if world > 1:
@@ -310,6 +355,8 @@ def main():
     ap.add_argument("--ref-cols", type=int, default=1_000_000,
                     help="columns per step of the CPU reference arm (bounded sample)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-iterations", action="store_true",
+                    help="skip the whole-iteration timings of the MLP configurations")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
