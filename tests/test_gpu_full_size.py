@@ -132,3 +132,66 @@ def test_config5_full_size_sampled_nodes_and_columns():
     got = dctx.consensus_dist()
     assert abs(got - expect) <= 1e-3 * expect
     dctx.close()
+
+
+def test_config3_full_size_fused_steps():
+    """n = 32 ring, MLP 784-1024-10 at full size with the gossip step inside the weight-gradient
+    kernel: whole steps against the oracle (ReLU ties resolved against the two-stage gradient)."""
+    w = wl.config(2, device="cuda")
+    seed = 31
+    ctx, X0, X1, G = _context(w, seed)
+    A, y = w.A.cpu().numpy(), w.y.cpu().numpy()
+    o = orc.Oracle(w.n, w.N, *w.csr(), w.gamma, seed, w.model, w.dims, w.batch, 0.0, A, y)
+    o.set_x(np.tile(w.x0.cpu().numpy(), (w.n, 1)))
+    for k in range(2):
+        ctx.set_fused_step(0)
+        ctx.current()[:, :w.N] = torch.from_numpy(o.X).cuda()
+        ctx.grad(k)
+        G_ref, _ = mlp_oracle_grad_matching_gates(orc, o, k, G[:, :w.N].cpu().numpy())
+        G.fill_(float("nan"))
+        ctx.set_fused_step(2)
+        ctx.step(k)
+        X_ref = o.mix_update(G_ref)
+        assert row_rel_err(ctx.current()[:, :w.N].cpu().numpy(), X_ref) <= TOL_STEP
+    ctx.close()
+
+
+def test_config5_full_size_fused_step_on_column_slices():
+    """n = 112 ring, MLP 1024-2048-2048-10 at full size, the launch configuration of the timed runs
+    (node ranges of 28, several waves of CTAs): the fused iteration against the oracle's gossip step on
+    column slices of all rows (it is separable per column; the gradient columns come from the two-stage
+    path, which the test above pins to the oracle on sampled nodes), and against the two-stage result
+    everywhere."""
+    _need(16)
+    w = wl.config(4, device="cuda")
+    seed = 78
+    ctx, X0, X1, G = _context(w, seed)
+    rng = np.random.default_rng(4)
+    X0[:, :w.N] += 0.01 * torch.randn((w.n, w.N), device="cuda", generator=torch.Generator("cuda").manual_seed(6))
+    start = X0.clone()
+    k = 5
+    ctx.grad(k)
+    width = 20_000
+    layer2 = 2048 * 1024 + 2048                     # first column of the 2048 x 2048 block
+    starts = [0, w.N - width, layer2 - width // 2, layer2 + 2048 * 2048 - width // 2] + \
+             [int(s) for s in rng.integers(width, w.N - 2 * width, 3)]
+    Xh = {s: start[:, s:s + width].cpu().numpy() for s in starts}
+    Gh = {s: G[:, s:s + width].cpu().numpy() for s in starts}
+    ctx.mix_update()
+    two_stage = ctx.current().clone()
+    # the fused iteration from the same point; G poisoned so that nothing stale can be picked up
+    ctx.current().copy_(start)
+    G.fill_(float("nan"))
+    ctx.set_fused_step(1)
+    before = ctx.launch_count()
+    ctx.step(k)
+    assert ctx.launch_count() - before == 14
+    out = ctx.current()
+    assert bool(torch.isfinite(out).all())
+    for s in starts:
+        ref = orc.mix_update(Xh[s], Gh[s], *w.csr(), w.gamma)
+        assert row_rel_err(out[:, s:s + width].cpu().numpy(), ref) <= TOL_STEP, s
+    diff = (out.double() - two_stage.double()).norm(dim=1) / two_stage.double().norm(dim=1)
+    assert float(diff.max()) <= 2e-6
+    assert float(out[:, w.N:].abs().max()) == 0.0
+    ctx.close()
