@@ -52,7 +52,7 @@ glm_forward_kernel(const float* __restrict__ X, int64_t ld, const float* __restr
         for (; c + 3 * kFwdThreads < d4; c += 4 * kFwdThreads) {
             float4 a[4], v[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) { a[u] = __ldcs(r4 + c + u * kFwdThreads); v[u] = __ldg(x4 + c + u * kFwdThreads); }
+            for (int u = 0; u < 4; ++u) { a[u] = __ldg(r4 + c + u * kFwdThreads); v[u] = __ldg(x4 + c + u * kFwdThreads); }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 acc = fmaf(a[u].x, v[u].x, acc); acc = fmaf(a[u].y, v[u].y, acc);
@@ -60,7 +60,7 @@ glm_forward_kernel(const float* __restrict__ X, int64_t ld, const float* __restr
             }
         }
         for (; c < d4; c += kFwdThreads) {
-            const float4 a = __ldcs(r4 + c), v = __ldg(x4 + c);
+            const float4 a = __ldg(r4 + c), v = __ldg(x4 + c);
             acc = fmaf(a.x, v.x, acc); acc = fmaf(a.y, v.y, acc);
             acc = fmaf(a.z, v.z, acc); acc = fmaf(a.w, v.w, acc);
         }
