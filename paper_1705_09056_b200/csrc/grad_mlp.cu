@@ -441,7 +441,14 @@ cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G, 
         g.C = c->d_act + p.act_off[l]; g.c_node = (int64_t)B * dout; g.c_m = dout;
         g.aux = X + s.b_off[l - 1]; g.aux_node = c->ld; g.aux_m = 0;
         g.M = B; g.N = dout; g.K = din;
-        if (use_tc) {   // m = output unit, n = sample: h_l[b][o]
+        if (use_tc && l == L && dout <= narrow::kMaxOut && din % 4 == 0 && s.w_off[l - 1] % 4 == 0 &&
+            reinterpret_cast<uintptr_t>(X) % 16 == 0 && reinterpret_cast<uintptr_t>(g.A) % 16 == 0) {
+            // classifier layer: a CTA per (node, four samples) on the fp32 pipes
+            narrow::narrow_forward_kernel<<<dim3((B + narrow::kFwdSamples - 1) / narrow::kFwdSamples, n),
+                                            narrow::kFwdThreads, 0, c->stream>>>(
+                X, c->ld, s.w_off[l - 1], s.b_off[l - 1], g.A, g.C, B, din, dout);
+            c->launches++;
+        } else if (use_tc) {   // m = output unit, n = sample: h_l[b][o]
             tc::Args a{};
             a.A = g.Bm; a.a_node = g.b_node; a.a_pitch = din; a.a_kcontig = 1;
             a.B = g.A; a.b_node = g.a_node; a.b_pitch = din; a.b_kcontig = 1;

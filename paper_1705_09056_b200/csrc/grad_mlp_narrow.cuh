@@ -87,5 +87,67 @@ narrow_backward_kernel(const float* __restrict__ X, float* __restrict__ G, int64
     }
 }
 
+// Forward product of the same layer: out[b][o] = b_o + sum_k h[b][k] W[o][k] (logits: no ReLU).  On the
+// tensor-core kernel one CTA per node walks all of k alone (one 128-row tile, 90 % padding): latency,
+// not bandwidth.  Here a CTA owns four samples of a node: thread t takes the 16-byte columns t, t + 128, ...
+// of k, loads the up to 16 weight rows there once and uses them for the four samples (all loads of an
+// iteration in flight together), then the 64 partial sums are reduced by shuffles and across the four
+// warps in a fixed order.  Exact fp32 FMA products.
+constexpr int kFwdThreads = 128;
+constexpr int kFwdSamples = 4;
+
+// grid (ceil(B / 4), nodes), block 128.  din % 4 == 0, rows 16-byte aligned.
+__global__ void __launch_bounds__(kFwdThreads)
+narrow_forward_kernel(const float* __restrict__ X, int64_t ld, int64_t w_off, int64_t b_off,
+                      const float* __restrict__ h, float* __restrict__ out, int B, int din, int dout) {
+    __shared__ float part[kFwdThreads / 32][kFwdSamples * kMaxOut];
+    const int node = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b0 = blockIdx.x * kFwdSamples;
+    const int nb = min(kFwdSamples, B - b0);
+    const int d4 = din / 4;
+    const float4* W = reinterpret_cast<const float4*>(X + (int64_t)node * ld + w_off);
+    const float4* hv = reinterpret_cast<const float4*>(h + ((int64_t)node * B + b0) * din);
+    float acc[kFwdSamples][kMaxOut];
+#pragma unroll
+    for (int s = 0; s < kFwdSamples; ++s)
+#pragma unroll
+        for (int o = 0; o < kMaxOut; ++o) acc[s][o] = 0.f;
+    for (int c = tid; c < d4; c += kFwdThreads) {
+        float4 w[kMaxOut], x[kFwdSamples];
+#pragma unroll
+        for (int o = 0; o < kMaxOut; ++o)
+            w[o] = o < dout ? __ldg(W + (int64_t)o * d4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int s = 0; s < kFwdSamples; ++s)
+            x[s] = s < nb ? __ldg(hv + (int64_t)s * d4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int s = 0; s < kFwdSamples; ++s)
+#pragma unroll
+            for (int o = 0; o < kMaxOut; ++o) {
+                acc[s][o] = fmaf(x[s].x, w[o].x, acc[s][o]); acc[s][o] = fmaf(x[s].y, w[o].y, acc[s][o]);
+                acc[s][o] = fmaf(x[s].z, w[o].z, acc[s][o]); acc[s][o] = fmaf(x[s].w, w[o].w, acc[s][o]);
+            }
+    }
+#pragma unroll
+    for (int s = 0; s < kFwdSamples; ++s)
+#pragma unroll
+        for (int o = 0; o < kMaxOut; ++o) {
+            float v = acc[s][o];
+#pragma unroll
+            for (int sh = 16; sh > 0; sh >>= 1) v += __shfl_xor_sync(0xffffffffu, v, sh);
+            if (lane == 0) part[warp][s * kMaxOut + o] = v;
+        }
+    __syncthreads();
+    if (tid < kFwdSamples * kMaxOut) {
+        const int s = tid / kMaxOut, o = tid % kMaxOut;
+        if (s < nb && o < dout) {
+            float v = part[0][tid];
+#pragma unroll
+            for (int wv = 1; wv < kFwdThreads / 32; ++wv) v += part[wv][tid];
+            out[((int64_t)node * B + b0 + s) * dout + o] = v + __ldg(X + (int64_t)node * ld + b_off + o);
+        }
+    }
+}
+
 }  // namespace narrow
 }  // namespace dpsgd
