@@ -149,8 +149,9 @@ DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* ctx, int32_t update_then_mix);
  * old values; biases, and blocks whose product runs on another kernel, are still written to G and
  * take the gossip step from there.  The result equals dpsgd_grad + dpsgd_mix_update up to fp32
  * rounding order.
- *   mode 0  off (default): two stages.
- *   mode 1  fused for the weight blocks where it is faster on B200: a ring W (Theorem 3) and a stacked
+ *   mode 0  off: two stages.
+ *   mode 1  (default) fused for the weight blocks where it is faster on B200: a ring W (Theorem 3) and a
+ *           stacked
  *           block of at least 64 MB, or rows of W with at most 3 entries and a stacked block of at
  *           least 512 MB (far beyond L2); other blocks in two stages.
  *   mode 2  fused for every block a fused kernel can take.  A ring W takes the kernel that keeps the
@@ -213,7 +214,9 @@ DPSGD_API dpsgd_status dpsgd_mix_update_consensus(dpsgd_ctx* ctx, double* consen
  * distance (as the 112-node experiments of Section 5 would, per step). */
 DPSGD_API dpsgd_status dpsgd_step_consensus(dpsgd_ctx* ctx, uint64_t k, double* consensus_out_dev);
 
-/* One full iteration k of Algorithm 1: dpsgd_grad(k) followed by dpsgd_mix_update(). */
+/* One full iteration k of Algorithm 1: the result of dpsgd_grad(k) followed by dpsgd_mix_update().  For
+ * the MLP the two stages may run as one (see dpsgd_set_fused_step: mode 1 is the default); G then does
+ * not hold the whole gradient afterwards.  Call dpsgd_grad() when G itself is wanted. */
 DPSGD_API dpsgd_status dpsgd_step(dpsgd_ctx* ctx, uint64_t k);
 
 /* The loop of Algorithm 1: iterations k_first, k_first + 1, ... (dpsgd_step each), enqueued in one

@@ -106,7 +106,7 @@ struct dpsgd_ctx {
     int64_t graph_launches = 0;              // kernels in one replay
 
     // gossip step fused into the MLP weight-gradient kernels (dpsgd_set_fused_step)
-    int fuse_step = 0;         // 0 off, 1 where it pays, 2 wherever the kernel applies
+    int fuse_step = 1;         // 0 off, 1 where it pays (default), 2 wherever a fused kernel applies, 3 as 2 without the ring kernel
     std::vector<std::pair<int64_t, int64_t>> fused_blocks;   // [begin, end) columns already written to X_next
 
     int64_t launches = 0;
