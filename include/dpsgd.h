@@ -150,10 +150,9 @@ DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* ctx, int32_t update_then_mix);
  * take the gossip step from there.  The result equals dpsgd_grad + dpsgd_mix_update up to fp32
  * rounding order.
  *   mode 0  off: two stages.
- *   mode 1  (default) fused for the weight blocks where it is faster on B200: a ring W (Theorem 3) and a
- *           stacked
- *           block of at least 64 MB, or rows of W with at most 3 entries and a stacked block of at
- *           least 512 MB (far beyond L2); other blocks in two stages.
+ *   mode 1  (default) fused for the weight blocks where it is faster on B200: a ring W (Theorem 3)
+ *           and a stacked block of at least 64 MB, or rows of W with at most 3 entries and a stacked
+ *           block of at least 512 MB (far beyond L2); other blocks in two stages.
  *   mode 2  fused for every block a fused kernel can take.  A ring W takes the kernel that keeps the
  *           tiles of X_{i-1} and X_i on chip while it walks the nodes (X is read once); any other W
  *           the kernel that gathers the neighbours' tiles through L2.
