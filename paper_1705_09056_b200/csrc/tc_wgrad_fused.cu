@@ -110,7 +110,9 @@ cudaError_t run_tcw_ring(dpsgd_ctx* c, const float* h, int din, const float* del
                          int64_t w_off, const float* X, float* Xn) {
     const int B = c->batch;
     auto al = [](const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; };
-    if (!c->can_ring || !c->W.band || c->n < 3 || B > tcw::kMaxK || din % 4 != 0 || dpitch % 4 != 0 || !al(h) || !al(delta))
+    // w_off and din multiples of 4: the columns left to the mixing kernel are then whole groups of four
+    if (!c->can_ring || !c->W.band || c->n < 3 || B > tcw::kMaxK || din % 4 != 0 || dpitch % 4 != 0 || w_off % 4 != 0 ||
+        !al(h) || !al(delta))
         return cudaErrorNotSupported;
     const uint64_t nodes = (uint64_t)c->n;
     CUtensorMap mapA, mapB;
