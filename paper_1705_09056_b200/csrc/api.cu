@@ -485,6 +485,20 @@ DPSGD_API dpsgd_status dpsgd_step_consensus(dpsgd_ctx* c, uint64_t k, double* ou
     if ((s = need_model(c)) != DPSGD_OK) return s;
     if (!out_dev) return fail(c, DPSGD_ERR_ARG, "consensus_out_dev is NULL");
     if (!aligned(out_dev, 8)) return fail(c, DPSGD_ERR_ALIGN, "consensus_out_dev must be 8-byte aligned");
+    if (c->fuse_step && fused_step_supported(c)) {
+        // the iteration with the gossip step inside the gradient kernels, then one pass over the new X:
+        // cheaper than writing G for the mixing kernel that accumulates the distance on the way
+        const float* X = c->X[c->cur];
+        float* Xn = c->X[c->cur ^ 1];
+        cudaError_t e = launch_grad_mlp(c, k, X, c->G, Xn);
+        if (e != cudaSuccess) return cuda_fail(c, e, "gradient kernels");
+        if (c->fused_blocks.empty()) return mix_with_consensus(c, out_dev);
+        e = launch_mix_rest(c, X, c->G, Xn);
+        if (e == cudaSuccess) e = launch_consensus(c, Xn, out_dev);
+        if (e != cudaSuccess) return cuda_fail(c, e, "mix_update with consensus");
+        c->cur ^= 1;
+        return DPSGD_OK;
+    }
     cudaError_t e = run_grad(c, k);
     if (e != cudaSuccess) return cuda_fail(c, e, "gradient kernels");
     return mix_with_consensus(c, out_dev);

@@ -176,3 +176,26 @@ def test_fused_request_falls_back_where_it_does_not_apply(variant):
         outs.append(run.x().copy())
         run.close()
     assert np.array_equal(outs[0], outs[1])
+
+
+def test_step_consensus_with_the_fused_iteration():
+    """dpsgd_step_consensus in fused mode: the new X and its consensus distance (Theorem 4's
+    sum_i ||xbar - x_i||^2) equal the two-stage iteration's."""
+    w = wl.mlp_workload(n=6, dims=(128, 192, 10), m=60, batch=16, gamma=0.05, seed=31)
+    X = _perturbed(w, 8)
+    res = []
+    for mode in (0, 2):
+        run, o = _setup(w, seed=4, X=X)
+        run.ctx.set_fused_step(mode)
+        log = torch.zeros(3, dtype=torch.float64, device="cuda")
+        for k in range(3):
+            run.ctx.step_consensus(k, log[k:k + 1])
+            if mode == 0:
+                o.step(k)
+        torch.cuda.synchronize()
+        res.append((run.x().copy(), log.cpu().numpy()))
+        if mode == 0:
+            assert abs(res[0][1][2] - o.consensus_dist()) <= 1e-3 * o.consensus_dist()
+        run.close()
+    assert row_rel_err(res[1][0], res[0][0]) <= 1e-5
+    assert np.all(np.abs(res[1][1] - res[0][1]) <= 1e-4 * res[0][1])
