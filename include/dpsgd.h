@@ -158,8 +158,9 @@ DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* ctx, int32_t update_then_mix);
  *           the kernel that gathers the neighbours' tiles through L2.
  *   mode 3  as mode 2, but the gathering kernel for a ring W too (for comparison).
  * The kernel applies when the model is the MLP on the tensor-core path (minibatch <= 64, layer input
- * widths multiples of 4), the printed order of Algorithm 1 is in force, no momentum is set and no row
- * of W has more than 8 entries; otherwise dpsgd_step() runs the two stages whatever the mode.
+ * widths multiples of 4), the printed order of Algorithm 1 is in force, no momentum is set and either no
+ * row of W has more than 8 entries or W is the averaging matrix 1 1^T / n (its rows all mix to the column
+ * mean, formed once per iteration); otherwise dpsgd_step() runs the two stages whatever the mode.
  * dpsgd_grad, dpsgd_mix_update and the other entry points are not affected.
  */
 DPSGD_API dpsgd_status dpsgd_set_fused_step(dpsgd_ctx* ctx, int32_t mode);

@@ -129,6 +129,7 @@ void release(dpsgd_ctx* c) {
     if (c->capture_stream) cudaStreamDestroy(c->capture_stream);
     cudaFree(c->d_k);
     cudaFree(c->d_w_blob);
+    cudaFree(c->d_mean_blob);
     cudaFree(c->d_idx);
     cudaFree(c->d_coef);
     cudaFree(c->d_node_batch);
@@ -195,6 +196,10 @@ namespace dpsgd {
 // Lets entry points that take no context leave a message for dpsgd_last_error(NULL).
 void set_thread_error(const std::string& msg) { g_create_error = msg; }
 }  // namespace dpsgd
+
+namespace {
+cudaError_t prepare_fused_source(dpsgd_ctx* c, const float* X);   // defined beside dpsgd_set_fused_step
+}
 
 extern "C" {
 
@@ -490,10 +495,12 @@ DPSGD_API dpsgd_status dpsgd_step_consensus(dpsgd_ctx* c, uint64_t k, double* ou
         // cheaper than writing G for the mixing kernel that accumulates the distance on the way
         const float* X = c->X[c->cur];
         float* Xn = c->X[c->cur ^ 1];
-        cudaError_t e = launch_grad_mlp(c, k, X, c->G, Xn);
-        if (e != cudaSuccess) return cuda_fail(c, e, "gradient kernels");
-        if (c->fused_blocks.empty()) return mix_with_consensus(c, out_dev);
+        cudaError_t e = prepare_fused_source(c, X);
+        if (e == cudaSuccess) e = launch_grad_mlp(c, k, X, c->G, Xn);
+        if (e != cudaSuccess) { c->fsrc_X = nullptr; return cuda_fail(c, e, "gradient kernels"); }
+        if (c->fused_blocks.empty()) { c->fsrc_X = nullptr; return mix_with_consensus(c, out_dev); }
         e = launch_mix_rest(c, X, c->G, Xn);
+        c->fsrc_X = nullptr;
         if (e == cudaSuccess) e = launch_consensus(c, Xn, out_dev);
         if (e != cudaSuccess) return cuda_fail(c, e, "mix_update with consensus");
         c->cur ^= 1;
@@ -503,6 +510,46 @@ DPSGD_API dpsgd_status dpsgd_step_consensus(dpsgd_ctx* c, uint64_t k, double* ou
     if (e != cudaSuccess) return cuda_fail(c, e, "gradient kernels");
     return mix_with_consensus(c, out_dev);
 }
+
+}  // extern "C"
+
+namespace {
+// Fused iteration with W = w 1 1^T (more entries per row than the kernels gather): the column mean is
+// formed once (one pass over X) and the kernels gather from it as from a one-row matrix.  Sets or
+// clears the source the fused kernels read; allocates the small buffer on first use.
+cudaError_t prepare_fused_source(dpsgd_ctx* c, const float* X) {
+    c->fsrc_X = nullptr;
+    if (!(c->can_uniform && c->W.max_deg > kFusedMaxDegree)) return cudaSuccess;
+    const size_t mean_bytes = sizeof(float) * (size_t)c->ld;
+    if (!c->d_mean_blob || c->mean_ld != c->ld) {
+        cudaFree(c->d_mean_blob);
+        c->d_mean_blob = nullptr;
+        const size_t total = mean_bytes + sizeof(int32_t) * (2 * (size_t)c->n + 1) + sizeof(float) * (size_t)c->n;
+        cudaError_t e = cudaMalloc(&c->d_mean_blob, total);
+        if (e != cudaSuccess) return e;
+        std::vector<int32_t> rp((size_t)c->n + 1), col((size_t)c->n, 0);
+        std::vector<float> one((size_t)c->n, 1.f);
+        for (int i = 0; i <= c->n; ++i) rp[i] = i;
+        char* b = static_cast<char*>(c->d_mean_blob) + mean_bytes;
+        e = cudaMemcpy(b, rp.data(), sizeof(int32_t) * rp.size(), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(b + sizeof(int32_t) * rp.size(), col.data(), sizeof(int32_t) * col.size(), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(b + sizeof(int32_t) * (rp.size() + col.size()), one.data(), sizeof(float) * one.size(), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) { cudaFree(c->d_mean_blob); c->d_mean_blob = nullptr; return e; }
+        c->mean_ld = c->ld;
+    }
+    float* mean = static_cast<float*>(c->d_mean_blob);
+    cudaError_t e = launch_average(c, X, mean);
+    if (e != cudaSuccess) return e;
+    char* b = static_cast<char*>(c->d_mean_blob) + mean_bytes;
+    c->fsrc_X = mean; c->fsrc_ld = 0;
+    c->fsrc_row_ptr = reinterpret_cast<const int32_t*>(b);
+    c->fsrc_col = c->fsrc_row_ptr + c->n + 1;
+    c->fsrc_val = reinterpret_cast<const float*>(c->fsrc_col + c->n);
+    return cudaSuccess;
+}
+}  // namespace
+
+extern "C" {
 
 DPSGD_API dpsgd_status dpsgd_set_fused_step(dpsgd_ctx* c, int32_t on) {
     if (!c) return DPSGD_ERR_ARG;
@@ -521,9 +568,11 @@ DPSGD_API dpsgd_status dpsgd_step(dpsgd_ctx* c, uint64_t k) {
         // (biases, blocks on other kernels, padding) take the gossip step from G afterwards
         const float* X = c->X[c->cur];
         float* Xn = c->X[c->cur ^ 1];
-        cudaError_t e = launch_grad_mlp(c, k, X, c->G, Xn);
-        if (e != cudaSuccess) return cuda_fail(c, e, "gradient kernels");
+        cudaError_t e = prepare_fused_source(c, X);
+        if (e == cudaSuccess) e = launch_grad_mlp(c, k, X, c->G, Xn);
+        if (e != cudaSuccess) { c->fsrc_X = nullptr; return cuda_fail(c, e, "gradient kernels"); }
         e = c->fused_blocks.empty() ? run_mix(c) : launch_mix_rest(c, X, c->G, Xn);
+        c->fsrc_X = nullptr;
         if (e != cudaSuccess) return cuda_fail(c, e, "mix_update kernel");
         c->cur ^= 1;
         return DPSGD_OK;

@@ -106,6 +106,15 @@ struct dpsgd_ctx {
     int64_t graph_launches = 0;              // kernels in one replay
 
     // gossip step fused into the MLP weight-gradient kernels (dpsgd_set_fused_step)
+    // W = w 1 1^T in the fused iteration: every row mixes to the column mean, so the kernels gather from
+    // a one-row matrix (the mean, recomputed each iteration) through a CSR with one entry per row
+    void* d_mean_blob = nullptr;           // mean [ld] | row_ptr [n+1] | col [n] | val [n]
+    int64_t mean_ld = 0;
+    const float* fsrc_X = nullptr;         // what the fused kernels gather from during this iteration
+    int64_t fsrc_ld = 0;
+    const int32_t* fsrc_row_ptr = nullptr;
+    const int32_t* fsrc_col = nullptr;
+    const float* fsrc_val = nullptr;
     int fuse_step = 1;         // 0 off, 1 where it pays (default), 2 wherever a fused kernel applies, 3 as 2 without the ring kernel
     std::vector<std::pair<int64_t, int64_t>> fused_blocks;   // [begin, end) columns already written to X_next
 

@@ -195,7 +195,7 @@ struct ColRanges {
 __global__ void __launch_bounds__(128)
 mix_ranges_kernel(const float4* __restrict__ X, const float4* __restrict__ G, float4* __restrict__ Xn,
                   const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col,
-                  const float* __restrict__ val, int64_t ld4, float ngamma, ColRanges rg) {
+                  const float* __restrict__ val, int64_t src_ld4, int64_t ld4, float ngamma, ColRanges rg) {
     const int64_t t = (int64_t)blockIdx.x * 128 + threadIdx.x;
     const int i = blockIdx.y;
     if (t >= rg.start4[rg.count]) return;
@@ -206,7 +206,7 @@ mix_ranges_kernel(const float4* __restrict__ X, const float4* __restrict__ G, fl
     const int pe = __ldg(row_ptr + i + 1);
     for (int p = __ldg(row_ptr + i); p < pe; ++p) {
         const float w = __ldg(val + p);
-        const float4 v = __ldg(X + (int64_t)__ldg(col + p) * ld4 + c);
+        const float4 v = __ldg(X + (int64_t)__ldg(col + p) * src_ld4 + c);
         a.x = fmaf(w, v.x, a.x); a.y = fmaf(w, v.y, a.y);
         a.z = fmaf(w, v.z, a.z); a.w = fmaf(w, v.w, a.w);
     }
@@ -243,9 +243,11 @@ cudaError_t launch_mix_rest(dpsgd_ctx* c, const float* X, const float* G, float*
     if (total == 0) return cudaSuccess;
     if (c->n > 65535) return cudaErrorInvalidValue;
     dim3 grid((unsigned)((total + 127) / 128), (unsigned)c->n);
+    const bool mean = c->fsrc_X != nullptr;      // W = w 1 1^T: gather from the column mean (a one-row matrix)
     mix_ranges_kernel<<<grid, 128, 0, c->stream>>>(
-        reinterpret_cast<const float4*>(X), reinterpret_cast<const float4*>(G), reinterpret_cast<float4*>(Xn),
-        c->W.row_ptr, c->W.col, c->W.val, c->ld / 4, -c->gamma, rg);
+        reinterpret_cast<const float4*>(mean ? c->fsrc_X : X), reinterpret_cast<const float4*>(G),
+        reinterpret_cast<float4*>(Xn), mean ? c->fsrc_row_ptr : c->W.row_ptr, mean ? c->fsrc_col : c->W.col,
+        mean ? c->fsrc_val : c->W.val, mean ? c->fsrc_ld / 4 : c->ld / 4, c->ld / 4, -c->gamma, rg);
     c->launches++;
     return cudaGetLastError();
 }

@@ -65,7 +65,7 @@ constexpr uint32_t A_COL0_ = 2 * kAccStride;   // first tensor-memory column of 
 struct Mix {
     const float* X;
     float* Xn;
-    int64_t ld, w_off;
+    int64_t ld, ld_out, w_off;       // row strides of X (0 when every row gathers from one shared row) and of Xn
     const int32_t* row_ptr;
     const int32_t* col;
     const float* val;
@@ -125,7 +125,7 @@ __device__ __forceinline__ void mix_rows(const Mix& mx, int node, uint32_t st, i
     constexpr int U = 4;
     const int p0 = __ldg(mx.row_ptr + node);
     const int deg = DEG > 0 ? DEG : __ldg(mx.row_ptr + node + 1) - p0;
-    float* out = mx.Xn + (int64_t)node * mx.ld + off;
+    float* out = mx.Xn + (int64_t)node * mx.ld_out + off;
 #pragma unroll 1
     for (int r0 = warp; r0 < ROWS; r0 += kMixWarps * U) {
         float4 acc[U];

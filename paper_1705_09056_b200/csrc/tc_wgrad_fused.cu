@@ -79,7 +79,8 @@ cudaError_t launch_ring(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap
 template <int NT, bool PRECISE>
 cudaError_t launch_deg(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap& mapB, const CUtensorMap& mapC,
                        const tcw::Args& a, int deg) {
-    switch (deg) {            // common row degree of W: ring 3, ring with one more link 4, torus 5
+    switch (deg) {            // common row degree: the column mean 1, ring 3, torus 5
+        case 1: return launch<NT, PRECISE, 1>(c, mapA, mapB, mapC, a);
         case 3: return launch<NT, PRECISE, 3>(c, mapA, mapB, mapC, a);
         case 5: return launch<NT, PRECISE, 5>(c, mapA, mapB, mapC, a);
         default: return launch<NT, PRECISE, 0>(c, mapA, mapB, mapC, a);
@@ -90,7 +91,7 @@ cudaError_t launch_deg(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap&
 
 bool fused_step_supported(const dpsgd_ctx* c) {
     return c->model == DPSGD_MODEL_MLP && !c->swapped && c->V == nullptr && c->mlp_precision != 2 &&
-           c->batch <= tcw::kMaxK && c->W.max_deg >= 1 && c->W.max_deg <= kFusedMaxDegree;
+           c->batch <= tcw::kMaxK && c->W.max_deg >= 1 && (c->W.max_deg <= kFusedMaxDegree || c->can_uniform);
 }
 
 // Where a fused kernel is faster than the two stages (measured on B200).  Ring W: the kernel with the
@@ -101,7 +102,8 @@ bool fused_step_supported(const dpsgd_ctx* c) {
 bool fused_step_pays(const dpsgd_ctx* c, int din, int dout) {
     const double block_bytes = (double)c->n * din * dout * sizeof(float);
     if (c->can_ring && c->n >= 3) return block_bytes >= 64.0 * 1024 * 1024;
-    return c->W.max_deg <= 3 && block_bytes >= 512.0 * 1024 * 1024;
+    const bool short_rows = c->W.max_deg <= 3 || (c->can_uniform && c->W.max_deg > kFusedMaxDegree);   // the mean counts as one row
+    return short_rows && block_bytes >= 512.0 * 1024 * 1024;
 }
 
 // Ring W (Theorem 3's band): the kernel that keeps the X tiles of nodes i-1 and i in tensor memory
@@ -126,7 +128,7 @@ cudaError_t run_tcw_ring(dpsgd_ctx* c, const float* h, int din, const float* del
     a.m_tiles = (din + tcw::kTileM - 1) / tcw::kTileM;
     a.n_tiles = (dout + 63) / 64;
     a.status = &c->d_result->status;
-    a.mix.X = X; a.mix.Xn = Xn; a.mix.ld = c->ld; a.mix.w_off = w_off;
+    a.mix.X = X; a.mix.Xn = Xn; a.mix.ld = c->ld; a.mix.ld_out = c->ld; a.mix.w_off = w_off;
     a.mix.row_ptr = c->W.row_ptr; a.mix.col = c->W.col; a.mix.val = c->W.val; a.mix.band = c->W.band;
     a.mix.ngamma = -c->gamma;
     return c->mlp_precision == 0 ? launch_ring<true>(c, mapA, mapB, a) : launch_ring<false>(c, mapA, mapB, a);
@@ -155,10 +157,12 @@ cudaError_t run_tcw_fused(dpsgd_ctx* c, const float* h, int din, const float* de
     a.m_tiles = (din + tcw::kTileM - 1) / tcw::kTileM;
     a.n_tiles = (dout + rows_b - 1) / rows_b;
     a.status = &c->d_result->status;
-    a.mix.X = X; a.mix.Xn = Xn; a.mix.ld = c->ld; a.mix.w_off = w_off;
-    a.mix.row_ptr = c->W.row_ptr; a.mix.col = c->W.col; a.mix.val = c->W.val; a.mix.band = c->W.band;
+    // gathered from X through W, or (W = w 1 1^T) from the column mean through a one-entry-per-row matrix
+    a.mix.X = c->fsrc_X ? c->fsrc_X : X; a.mix.Xn = Xn; a.mix.ld = c->fsrc_X ? c->fsrc_ld : c->ld; a.mix.ld_out = c->ld; a.mix.w_off = w_off;
+    a.mix.row_ptr = c->fsrc_X ? c->fsrc_row_ptr : c->W.row_ptr; a.mix.col = c->fsrc_X ? c->fsrc_col : c->W.col;
+    a.mix.val = c->fsrc_X ? c->fsrc_val : c->W.val; a.mix.band = c->W.band;
     a.mix.ngamma = -c->gamma;
-    const int deg = c->W.uniform_deg;
+    const int deg = c->fsrc_X ? 1 : c->W.uniform_deg;
     const bool precise = c->mlp_precision == 0;
     switch (rows_b) {
         case 16: return precise ? launch_deg<1, true>(c, mapA, mapB, mapC, a, deg) : launch_deg<1, false>(c, mapA, mapB, mapC, a, deg);

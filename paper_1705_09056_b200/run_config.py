@@ -27,9 +27,10 @@ def main():
     ap.add_argument("--fused-consensus", action="store_true",
                     help="log the consensus distance every step from inside the gossip kernel")
     ap.add_argument("--swapped", action="store_true", help="footnote c: update locally, then average")
-    ap.add_argument("--fused-step", type=int, default=0, nargs="?", const=1,
+    ap.add_argument("--fused-step", type=int, default=None, nargs="?", const=1,
                     help="MLP: gossip step inside the weight-gradient kernels (those blocks of G are never "
-                         "written): 1 where it is faster, 2 wherever the kernel applies")
+                         "written): 0 two stages, 1 where it is faster (the library's default), 2 wherever a "
+                         "fused kernel applies, 3 as 2 without the ring kernel")
     args = ap.parse_args()
 
     build.build()
@@ -61,7 +62,7 @@ def main():
 
     if args.swapped:
         ctx.set_order(True)
-    if args.fused_step:
+    if args.fused_step is not None:
         ctx.set_fused_step(args.fused_step)
     for k in range(args.warmup):
         ctx.step(k)

@@ -41,6 +41,7 @@ FUSED_CASES = [
     (4, "ring", (18, 33, 7), 40, 5),                  # rows of 18 floats: the fused kernel cannot take them, plain path
     (2, "ring", (64, 48, 12), 30, 4),                 # two nodes: coinciding neighbours summed in W
     (5, "ring", (64, 33, 36, 24, 10), 40, 8),         # third block starts at an odd column: left to the two stages
+    (12, "dense", (128, 96, 10), 40, 8),              # W = 11^T/n with more entries per row than the kernels gather: column mean
 ]
 
 
