@@ -161,11 +161,13 @@ def time_steps(ctx, steps, warmup, torch):
 
 def whole_iterations(torch, binding, wl, dev, steps=20, warmup=3):
     """Whole D-PSGD iterations (sample + gradient + mix + update; consensus distance read once at the end)
-    on the two MLP configurations, two-stage and with the gossip step inside the gradient kernels.
+    on the two MLP configurations (the larger one also with the dense averaging matrix, its C-PSGD
+    baseline), two-stage and with the gossip step inside the gradient kernels.
     Context for the headline line, which times the gossip step alone."""
     out = {}
-    for name, idx in (("mlp_784-1024-10_n32_ring", 2), ("mlp_1024-2048-2048-10_n112_ring", 4)):
-        w = wl.config(idx, device=dev)
+    for name, idx, topo in (("mlp_784-1024-10_n32_ring", 2, "ring"), ("mlp_1024-2048-2048-10_n112_ring", 4, "ring"),
+                            ("mlp_1024-2048-2048-10_n112_dense_cpsgd_averaging", 4, "dense")):
+        w = wl.config(idx, device=dev, topology=topo)
         X0 = wl.stack_rows(w.x0, w.n, w.ld)
         X1, G = torch.zeros_like(X0), torch.zeros_like(X0)
         log = torch.zeros(steps + warmup, dtype=torch.float64, device=dev)
