@@ -19,16 +19,22 @@
 //                   which writes whole lines asynchronously and clips at the matrix edge; two
 //                   staging buffers, so the store of one tile overlaps the next.
 //
-// FUSE: the gossip step of Algorithm 1 (steps 4-5) is applied to the tile while it is on chip.  No
-// TMA store: sixteen more warps (the mixers; the gather is bound by the bytes they keep in flight)
-// take a staged tile, read the same tile of X from the node's neighbours in W and write
+// That is MODE kStore.  In the two other modes the gossip step of Algorithm 1 (steps 4-5) is applied to
+// the tile while it is on chip and the kernel writes
 //     X_next[node] = sum_j W_ij X[j] - gamma * gW
-// with 128-bit accesses along the input-unit index.  The neighbours' tiles are shared with the work
-// items of the neighbouring nodes; a CTA walks consecutive nodes at one tile position, so all but the
-// first read of an element come from L2, and the mixers prefetch the next node's tiles into L2 one
-// item ahead so that the first read does too.  This block of the gradient
-// never reaches HBM: 8 bytes per parameter (read X, write X_next) instead of 16 (write G; read X,
-// read G, write X_next).
+// so that this block of the gradient never reaches HBM: 8 bytes per parameter (read X, write X_next)
+// instead of 16 (write G; read X, read G, write X_next).  A CTA then walks a range of consecutive nodes
+// at one tile position, so that the neighbours' tiles of X it needs for node i are the ones it touched
+// for nodes i-1 and i-2.
+//
+//   kGather (any W with few entries per row, or the column mean as a one-row matrix): no TMA store;
+//           sixteen more warps (the mixers; a gather is bound by the bytes its threads keep in flight)
+//           take a staged tile, read the same tile of X from the node's neighbours with 128-bit loads
+//           (all but the first read of an element come from L2; the next node's tiles are prefetched
+//           into L2 one item ahead) and write X_next.  Two column tiles per item.
+//   kRing   (Theorem 3's ring): no epilogue warps and no staging; sixteen mixer warps read the
+//           accumulator in its own layout and keep the tiles of X_{i-1} and X_i in tensor memory, so
+//           X is read from memory once.  One column tile per item (the window holds one position).
 //
 // One persistent CTA per SM; a work item is (node, 128-row block of m, run of column tiles).  Every
 // mbarrier wait is bounded; a wait that runs out raises the status word, the TMA thread waits
@@ -49,7 +55,7 @@ using tcs::mbar_expect_tx;
 using tcs::tma_load_3d;
 
 constexpr int kThreads = 320;        // 4 epilogue warps, 4 converter warps, MMA warp, TMA warp
-constexpr int kMixWarps = 16;        // FUSE only: warps 10..25 apply the gossip step to staged tiles
+constexpr int kMixWarps = 16;        // kGather: warps 10..25 apply the gossip step to staged tiles
 constexpr int kThreadsFused = kThreads + 32 * kMixWarps;
 constexpr int kThreadsRing = 704;    // kRing: converters, MMA, TMA as above; warps 0-3 and 10-21 mix
 enum { kStore = 0, kGather = 1, kRing = 2 };
@@ -86,7 +92,7 @@ struct Args {
     int splits, split_len;           // node ranges, nodes per range
     int total_seqs;                  // m_tiles * chunks * splits
     int* status;
-    Mix mix;                         // FUSE only
+    Mix mix;                         // kGather, kRing
 };
 
 __host__ __device__ constexpr uint32_t a_raw_bytes() { return kMaxK * kTileM * 4; }
@@ -209,7 +215,7 @@ __device__ __forceinline__ Item cta_item(const Args& g, int i) {
 
 // NT = column tile / 16 (16, 32 or 64 output units per tile); PRECISE: three split MMAs per product.
 // mapA: h as (m, k, node), box 128 x 64.  mapB: delta as (n, k, node), box 16 NT x 64.  mapC: the
-// gradient block as (m, n, node), box 128 x 16 NT (not used with FUSE).
+// gradient block as (m, n, node), box 128 x 16 NT (kStore only).
 //
 // Tensor memory columns: [0, 128) two accumulators, then two converted h tiles of 64 heads +
 // 64 remainders each.
@@ -224,7 +230,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     constexpr uint32_t B_CONV = b_conv_bytes(ROWS_B), B_LBO = b_lbo(ROWS_B), SBO = 128;
     constexpr uint32_t NCOPY = PRECISE ? 2 : 1;
     constexpr uint32_t CONV_BUF = NCOPY * B_CONV;
-    constexpr bool FUSE = MODE == kGather;
+    constexpr bool FUSE = MODE == kGather;            // staged tiles go to the mixer warps instead of a TMA store
     constexpr uint32_t STAGE = MODE == kRing ? 0u : stage_bytes(ROWS_B);
     constexpr uint32_t WIN_COL0 = A_COL0_ + 2 * kACols;      // kRing: two 64-column slots of the X window
     constexpr uint32_t A_COL0 = A_COL0_;

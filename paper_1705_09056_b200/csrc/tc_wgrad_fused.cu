@@ -4,8 +4,8 @@
 //     X_next[i][block] = sum_j W_ij X[j][block] - gamma * (delta_i^T h_i)
 //
 // so this block of the stochastic gradient dF(X_k; xi_k) (Section 3) is consumed on chip and never
-// written to HBM.  The kernel is tc_wgrad_kernel<..., FUSE = true> of tc_wgrad.cuh; this file holds
-// its host side only.
+// written to HBM.  The kernels are tc_wgrad_kernel<..., kGather> and <..., kRing> of tc_wgrad.cuh; this
+// file holds their host side: shape checks, tensor maps, the division of the work into node ranges.
 #include <algorithm>
 
 #include "ctx.h"
