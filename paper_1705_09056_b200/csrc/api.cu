@@ -132,6 +132,7 @@ void release(dpsgd_ctx* c) {
     cudaFree(c->d_mean_blob);
     cudaFree(c->d_idx);
     cudaFree(c->d_coef);
+    cudaFree(c->d_glm_part);
     cudaFree(c->d_node_batch);
     cudaFree(c->d_active);
     cudaFree(c->d_act);

@@ -86,6 +86,8 @@ struct dpsgd_ctx {
     // scratch (library-owned)
     int32_t* d_idx = nullptr;    // [n][B]
     float* d_coef = nullptr;     // [n][B] per-sample backward coefficients (linear models)
+    float* d_glm_part = nullptr; // [n][ceil(B / 4)][ld] shares of the gradient, one per group of four draws
+    size_t glm_part_floats = 0;
     int32_t* d_node_batch = nullptr;  // [n] per-node minibatch sizes B_i <= B; NULL: every node uses B
     int32_t* d_active = nullptr;      // [n] nodes that take part in a masked local step
     float* d_act = nullptr;      // MLP activations h_0..h_L  (see grad_mlp.cu for the layout)

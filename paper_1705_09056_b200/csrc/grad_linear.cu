@@ -147,13 +147,153 @@ glm_backward_kernel(const float* __restrict__ X, float* __restrict__ G, int64_t 
     }
 }
 
+// ---- rows kept in registers: forward and backward from ONE read of the sampled rows ----
+//
+// A CTA owns kRowsS consecutive draws of a node.  Thread t holds the 16-byte columns t, t + 256, ... of
+// each of their data rows (d <= 4096: at most four per row), so the dot products (shuffles, then a
+// fixed-order sum over the warps), the coefficients and the CTA's share sum_s coef_s a_s of the gradient
+// all come from that one read.  The shares go to a scratch [node][group][ld] and a second, small kernel
+// adds them in group order (bit-reproducible), applies the L2 term and writes the padding.
+constexpr int kRowsS = 4;
+constexpr int kRowsThreads = 256;
+constexpr int kRowsMaxR = 4;             // 16-byte columns per thread and row: d <= 4 * 4 * 256
+
+__global__ void __launch_bounds__(kRowsThreads)
+glm_rows_kernel(const float* __restrict__ X, int64_t ld, const float* __restrict__ A, const float* __restrict__ y,
+                int64_t m, int d, int B, uint64_t seed, uint64_t k, const uint64_t* __restrict__ k_ptr, int model,
+                int32_t* __restrict__ idx, float* __restrict__ part, int groups,
+                const int32_t* __restrict__ node_batch) {
+    __shared__ float red[kRowsThreads / 32][kRowsS];
+    __shared__ float coef[kRowsS];
+    const int node = blockIdx.y, grp = blockIdx.x, tid = threadIdx.x;
+    if (k_ptr) k = *k_ptr;        // iteration counter kept on the device (graph replay)
+    const int Bi = node_batch ? __ldg(node_batch + node) : B;
+    const int d4 = d / 4;
+    const float4* x4 = reinterpret_cast<const float4*>(X + (int64_t)node * ld);
+    float4 row[kRowsS][kRowsMaxR], xv[kRowsMaxR];
+    int32_t jdx[kRowsS];
+#pragma unroll
+    for (int s = 0; s < kRowsS; ++s) {
+        const int b = grp * kRowsS + s;
+        jdx[s] = b < B ? sample_index(seed, k, (uint32_t)node, (uint32_t)b, (uint32_t)m) : 0;
+        if (tid == 0 && b < B) idx[node * B + b] = jdx[s];
+        const float4* r4 = reinterpret_cast<const float4*>(A + ((int64_t)node * m + jdx[s]) * d);
+#pragma unroll
+        for (int r = 0; r < kRowsMaxR; ++r) {
+            const int c = tid + r * kRowsThreads;
+            row[s][r] = (b < Bi && c < d4) ? __ldg(r4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < kRowsMaxR; ++r) {
+        const int c = tid + r * kRowsThreads;
+        xv[r] = c < d4 ? __ldg(x4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int s = 0; s < kRowsS; ++s) {
+        float acc = 0.f;
+#pragma unroll
+        for (int r = 0; r < kRowsMaxR; ++r) {
+            acc = fmaf(row[s][r].x, xv[r].x, acc); acc = fmaf(row[s][r].y, xv[r].y, acc);
+            acc = fmaf(row[s][r].z, xv[r].z, acc); acc = fmaf(row[s][r].w, xv[r].w, acc);
+        }
+        acc = warp_allsum(acc);
+        if ((tid & 31) == 0) red[tid >> 5][s] = acc;
+    }
+    __syncthreads();
+    if (tid < kRowsS) {
+        const int b = grp * kRowsS + tid;
+        float cf = 0.f;
+        if (b < Bi) {
+            float dot = 0.f;
+#pragma unroll
+            for (int t = 0; t < kRowsThreads / 32; ++t) dot += red[t][tid];
+            const float yv = __ldg(y + (int64_t)node * m + jdx[tid]);
+            if (model == DPSGD_MODEL_LSQ) {
+                cf = (dot - yv) / (float)Bi;
+            } else {
+                const float z = dot + __ldg(X + (int64_t)node * ld + d);
+                cf = -yv * (1.f / (1.f + expf(yv * z))) / (float)Bi;
+            }
+        }
+        coef[tid] = cf;
+    }
+    __syncthreads();
+    float* out = part + ((int64_t)node * groups + grp) * ld;
+#pragma unroll
+    for (int r = 0; r < kRowsMaxR; ++r) {
+        const int c = tid + r * kRowsThreads;
+        if (c < d4) {
+            float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int s = 0; s < kRowsS; ++s) {
+                const float w = coef[s];
+                a.x = fmaf(w, row[s][r].x, a.x); a.y = fmaf(w, row[s][r].y, a.y);
+                a.z = fmaf(w, row[s][r].z, a.z); a.w = fmaf(w, row[s][r].w, a.w);
+            }
+            reinterpret_cast<float4*>(out)[c] = a;
+        }
+    }
+    if (tid == 0 && model == DPSGD_MODEL_LOGISTIC) {   // the bias column's share: sum of the coefficients
+        float sb = 0.f;
+#pragma unroll
+        for (int s = 0; s < kRowsS; ++s) sb += coef[s];
+        out[d] = sb;
+    }
+}
+
+// G[node][c] = sum over the groups, in order; + l2 x for the logistic weights; zero beyond the parameters.
+__global__ void __launch_bounds__(128)
+glm_rows_reduce_kernel(const float* __restrict__ X, float* __restrict__ G, int64_t ld, const float* __restrict__ part,
+                       int groups, int d, int model, float l2) {
+    const int node = blockIdx.y;
+    const int64_t c = (int64_t)blockIdx.x * 128 + threadIdx.x;
+    if (c >= ld) return;
+    const int last = model == DPSGD_MODEL_LOGISTIC ? d : d - 1;      // last parameter column
+    float s = 0.f;
+    if (c <= last) {
+        const float* p = part + (int64_t)node * groups * ld + c;
+        int g = 0;
+        for (; g + 8 <= groups; g += 8) {          // eight loads in flight, added in group order
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = __ldg(p + (int64_t)(g + u) * ld);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) s += v[u];
+        }
+        for (; g < groups; ++g) s += __ldg(p + (int64_t)g * ld);
+        if (model == DPSGD_MODEL_LOGISTIC && c < d) s = fmaf(l2, __ldg(X + (int64_t)node * ld + c), s);
+    }
+    G[(int64_t)node * ld + c] = s;
+}
+
 }  // namespace
 
 cudaError_t launch_grad_linear(dpsgd_ctx* c, uint64_t k, const float* X, float* G) {
     const int n = c->n, B = c->batch, d = c->d;
     const float* y = static_cast<const float*>(c->y);
-    const int fwd_grid = n * B;
     const bool vec = (d % 4 == 0);
+    if (vec && d >= 1024 && d <= 16 * kRowsThreads * kRowsMaxR / 4 && n <= 65535) {
+        // one read of the sampled rows: they stay in registers between the forward and the backward part
+        // (rows of a few hundred bytes leave most of such a CTA idle: they keep the two kernels below)
+        const int groups = (B + kRowsS - 1) / kRowsS;
+        const size_t need = (size_t)n * groups * c->ld;
+        if (c->glm_part_floats < need) {
+            cudaFree(c->d_glm_part);
+            c->d_glm_part = nullptr; c->glm_part_floats = 0;
+            cudaError_t e = cudaMalloc(&c->d_glm_part, need * sizeof(float));
+            if (e != cudaSuccess) return e;
+            c->glm_part_floats = need;
+        }
+        glm_rows_kernel<<<dim3(groups, n), kRowsThreads, 0, c->stream>>>(
+            X, c->ld, c->A, y, c->m, d, B, c->seed, k, c->k_dev_active, c->model, c->d_idx, c->d_glm_part, groups,
+            c->d_node_batch);
+        glm_rows_reduce_kernel<<<dim3((unsigned)((c->ld + 127) / 128), n), 128, 0, c->stream>>>(
+            X, G, c->ld, c->d_glm_part, groups, d, c->model, c->l2);
+        c->launches += 2;
+        return cudaGetLastError();
+    }
+    const int fwd_grid = n * B;
     if (vec)
         glm_forward_kernel<4><<<fwd_grid, kFwdThreads, 0, c->stream>>>(
             X, c->ld, c->A, y, c->m, d, B, n, c->seed, k, c->k_dev_active, c->model, c->d_idx, c->d_coef,

@@ -57,6 +57,10 @@ LIN_CASES = [
     (binding.MODEL_LOGISTIC, 4, 130, 64, 7),       # ragged d
     (binding.MODEL_LOGISTIC, 6, 260, 300, 128),
     (binding.MODEL_LOGISTIC, 1, 8, 10, 1),
+    # rows of 4 KB and more stay in registers between the forward and the backward part
+    (binding.MODEL_LSQ, 3, 1024, 40, 6),           # N == ld: no column beyond the parameters
+    (binding.MODEL_LOGISTIC, 3, 2052, 50, 9),      # ragged against the 256 x 16-byte columns and the groups of four draws
+    (binding.MODEL_LSQ, 2, 4096, 20, 1),
 ]
 
 

@@ -24,9 +24,10 @@ def _ragged_reference(w, X, idx, sizes):
                          [idx[i, :sizes[i]] for i in range(w.n)], w.l2_lambda)
 
 
+@pytest.mark.parametrize("d", [52, 1028])     # narrow rows: two kernels; wide rows: the kernel that keeps them in registers
 @pytest.mark.parametrize("model", [binding.MODEL_LSQ, binding.MODEL_LOGISTIC])
-def test_per_node_minibatch_sizes_linear(model):
-    n, d, m, B = 6, 52, 96, 16
+def test_per_node_minibatch_sizes_linear(model, d):
+    n, m, B = 6, 96, 16
     sizes = [1, 16, 7, 8, 9, 3]
     w = (wl.lsq_workload(n=n, d=d, m=m, batch=B, seed=4) if model == binding.MODEL_LSQ
          else wl.logistic_workload(n=n, d=d, m=m, batch=B, l2_lambda=1e-3, seed=4))
