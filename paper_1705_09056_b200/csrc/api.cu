@@ -578,6 +578,14 @@ DPSGD_API dpsgd_status dpsgd_step(dpsgd_ctx* c, uint64_t k) {
         c->cur ^= 1;
         return DPSGD_OK;
     }
+    if (c->fuse_step && linear_step_fuses(c)) {
+        // linear model with wide rows on a small matrix: the reduction of the gradient shares and the
+        // gossip step in one launch (G is written as well)
+        cudaError_t e = launch_linear_step(c, k, c->X[c->cur], c->G, c->X[c->cur ^ 1]);
+        if (e != cudaSuccess) return cuda_fail(c, e, "gradient and mix_update kernels");
+        c->cur ^= 1;
+        return DPSGD_OK;
+    }
     cudaError_t e = run_grad(c, k);
     if (e != cudaSuccess) return cuda_fail(c, e, "gradient kernels");
     e = run_mix(c);

@@ -150,6 +150,8 @@ cudaError_t launch_sample(dpsgd_ctx* c, uint64_t k, int32_t* idx);
 cudaError_t launch_set_k(dpsgd_ctx* c, uint64_t v);
 cudaError_t launch_advance_k(dpsgd_ctx* c);
 cudaError_t launch_grad_linear(dpsgd_ctx* c, uint64_t k, const float* X, float* G);
+bool linear_step_fuses(const dpsgd_ctx* c);
+cudaError_t launch_linear_step(dpsgd_ctx* c, uint64_t k, const float* X, float* G, float* Xn);
 // Xn != NULL: weight blocks whose product runs on the fused kernel are written to Xn after the gossip
 // step instead of to G, and listed in c->fused_blocks.
 cudaError_t launch_grad_mlp(dpsgd_ctx* c, uint64_t k, const float* X, float* G, float* Xn = nullptr);

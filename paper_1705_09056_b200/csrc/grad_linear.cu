@@ -267,30 +267,119 @@ glm_rows_reduce_kernel(const float* __restrict__ X, float* __restrict__ G, int64
     G[(int64_t)node * ld + c] = s;
 }
 
+// The same reduction followed at once by the gossip step of Algorithm 1 (steps 4-5) for its four columns:
+// G = sum of the shares (+ l2 x), X_next = sum_j W_ij X_j - gamma G.  For matrices small enough to sit in
+// L2, where a separate mixing launch costs more than its work.
+__global__ void __launch_bounds__(128)
+glm_rows_reduce_mix_kernel(const float4* __restrict__ X, float4* __restrict__ G, float4* __restrict__ Xn, int64_t ld4,
+                           const float4* __restrict__ part, int groups, int d, int model, float l2,
+                           const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col,
+                           const float* __restrict__ val, float ngamma) {
+    const int node = blockIdx.y;
+    const int64_t c = (int64_t)blockIdx.x * 128 + threadIdx.x;
+    if (c >= ld4) return;
+    const int last = model == DPSGD_MODEL_LOGISTIC ? d : d - 1;      // last parameter column
+    const float4 x = __ldg(X + (int64_t)node * ld4 + c);
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (4 * c <= last) {
+        const float4* p = part + (int64_t)node * groups * ld4 + c;
+        int g = 0;
+        for (; g + 8 <= groups; g += 8) {          // eight loads in flight, added in group order
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = __ldg(p + (int64_t)(g + u) * ld4);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
+        }
+        for (; g < groups; ++g) {
+            const float4 v = __ldg(p + (int64_t)g * ld4);
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        }
+        const int64_t c0 = 4 * c;
+        if (model == DPSGD_MODEL_LOGISTIC) {
+            if (c0 < d) s.x = fmaf(l2, x.x, s.x);
+            if (c0 + 1 < d) s.y = fmaf(l2, x.y, s.y);
+            if (c0 + 2 < d) s.z = fmaf(l2, x.z, s.z);
+            if (c0 + 3 < d) s.w = fmaf(l2, x.w, s.w);
+        }
+        // shares never written beyond the parameters hold stale scratch: zero them
+        if (c0 + 1 > last) s.y = 0.f;
+        if (c0 + 2 > last) s.z = 0.f;
+        if (c0 + 3 > last) s.w = 0.f;
+    }
+    G[(int64_t)node * ld4 + c] = s;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int pe = __ldg(row_ptr + node + 1);
+    for (int p = __ldg(row_ptr + node); p < pe; ++p) {
+        const float w = __ldg(val + p);
+        const float4 v = __ldg(X + (int64_t)__ldg(col + p) * ld4 + c);
+        a.x = fmaf(w, v.x, a.x); a.y = fmaf(w, v.y, a.y);
+        a.z = fmaf(w, v.z, a.z); a.w = fmaf(w, v.w, a.w);
+    }
+    a.x = fmaf(ngamma, s.x, a.x); a.y = fmaf(ngamma, s.y, a.y);
+    a.z = fmaf(ngamma, s.z, a.z); a.w = fmaf(ngamma, s.w, a.w);
+    Xn[(int64_t)node * ld4 + c] = a;
+}
+
+bool rows_path(const dpsgd_ctx* c) {
+    return c->d % 4 == 0 && c->d >= 1024 && c->d <= 16 * kRowsThreads * kRowsMaxR / 4 && c->n <= 65535;
+}
+
+// First half of the rows-in-registers gradient: the shares of every group of four draws.
+cudaError_t launch_rows(dpsgd_ctx* c, uint64_t k, const float* X, int* groups_out) {
+    const int n = c->n, B = c->batch;
+    const int groups = (B + kRowsS - 1) / kRowsS;
+    const size_t need = (size_t)n * groups * c->ld;
+    if (c->glm_part_floats < need) {
+        cudaFree(c->d_glm_part);
+        c->d_glm_part = nullptr; c->glm_part_floats = 0;
+        cudaError_t e = cudaMalloc(&c->d_glm_part, need * sizeof(float));
+        if (e != cudaSuccess) return e;
+        c->glm_part_floats = need;
+    }
+    glm_rows_kernel<<<dim3(groups, n), kRowsThreads, 0, c->stream>>>(
+        X, c->ld, c->A, static_cast<const float*>(c->y), c->m, c->d, B, c->seed, k, c->k_dev_active, c->model,
+        c->d_idx, c->d_glm_part, groups, c->d_node_batch);
+    c->launches++;
+    *groups_out = groups;
+    return cudaGetLastError();
+}
+
 }  // namespace
+
+// Whole iteration of a linear model in two launches: shares of the gradient, then their reduction and the
+// gossip step together.  False when the shapes or the options call for the separate stages.
+bool linear_step_fuses(const dpsgd_ctx* c) {
+    return c->model != DPSGD_MODEL_MLP && rows_path(c) && !c->kind_forced && mix_is_small(c) && !c->swapped &&
+           c->V == nullptr;
+}
+
+cudaError_t launch_linear_step(dpsgd_ctx* c, uint64_t k, const float* X, float* G, float* Xn) {
+    int groups = 0;
+    cudaError_t e = launch_rows(c, k, X, &groups);
+    if (e != cudaSuccess) return e;
+    const int64_t ld4 = c->ld / 4;
+    glm_rows_reduce_mix_kernel<<<dim3((unsigned)((ld4 + 127) / 128), c->n), 128, 0, c->stream>>>(
+        reinterpret_cast<const float4*>(X), reinterpret_cast<float4*>(G), reinterpret_cast<float4*>(Xn), ld4,
+        reinterpret_cast<const float4*>(c->d_glm_part), groups, c->d, c->model, c->l2, c->W.row_ptr, c->W.col,
+        c->W.val, -c->gamma);
+    c->launches++;
+    return cudaGetLastError();
+}
 
 cudaError_t launch_grad_linear(dpsgd_ctx* c, uint64_t k, const float* X, float* G) {
     const int n = c->n, B = c->batch, d = c->d;
     const float* y = static_cast<const float*>(c->y);
     const bool vec = (d % 4 == 0);
-    if (vec && d >= 1024 && d <= 16 * kRowsThreads * kRowsMaxR / 4 && n <= 65535) {
+    if (rows_path(c)) {
         // one read of the sampled rows: they stay in registers between the forward and the backward part
         // (rows of a few hundred bytes leave most of such a CTA idle: they keep the two kernels below)
-        const int groups = (B + kRowsS - 1) / kRowsS;
-        const size_t need = (size_t)n * groups * c->ld;
-        if (c->glm_part_floats < need) {
-            cudaFree(c->d_glm_part);
-            c->d_glm_part = nullptr; c->glm_part_floats = 0;
-            cudaError_t e = cudaMalloc(&c->d_glm_part, need * sizeof(float));
-            if (e != cudaSuccess) return e;
-            c->glm_part_floats = need;
-        }
-        glm_rows_kernel<<<dim3(groups, n), kRowsThreads, 0, c->stream>>>(
-            X, c->ld, c->A, y, c->m, d, B, c->seed, k, c->k_dev_active, c->model, c->d_idx, c->d_glm_part, groups,
-            c->d_node_batch);
+        int groups = 0;
+        cudaError_t e = launch_rows(c, k, X, &groups);
+        if (e != cudaSuccess) return e;
         glm_rows_reduce_kernel<<<dim3((unsigned)((c->ld + 127) / 128), n), 128, 0, c->stream>>>(
             X, G, c->ld, c->d_glm_part, groups, d, c->model, c->l2);
-        c->launches += 2;
+        c->launches++;
         return cudaGetLastError();
     }
     const int fwd_grid = n * B;
