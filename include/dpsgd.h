@@ -162,6 +162,9 @@ DPSGD_API dpsgd_status dpsgd_set_order(dpsgd_ctx* ctx, int32_t update_then_mix);
  * row of W has more than 8 entries or W is the averaging matrix 1 1^T / n (its rows all mix to the column
  * mean, formed once per iteration); otherwise dpsgd_step() runs the two stages whatever the mode.
  * dpsgd_grad, dpsgd_mix_update and the other entry points are not affected.
+ * The linear models have a small counterpart under any mode but 0: with data rows of 4 to 16 KB and
+ * a stacked matrix of at most 8 MB, dpsgd_step() adds up the gradient's per-group shares and applies
+ * the gossip step in one launch (G is still written in full there).
  */
 DPSGD_API dpsgd_status dpsgd_set_fused_step(dpsgd_ctx* ctx, int32_t mode);
 
