@@ -33,7 +33,7 @@ BYTES_PER_REPLICA_PARAM = 12          # read X, read G, write X_next (fp32 each)
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 METRIC = "replica-steps/s at n nodes; fused mix+update HBM GB/s vs B200 peak"
-ORACLE_SAMPLE_COLS = 10_000_000
+ORACLE_SAMPLE_COLS = 5_000_000          # columns per oracle step in BOTH CPU legs (vectors beyond any host cache)
 
 
 def measured_peak():
@@ -91,33 +91,48 @@ class ClockSampler:
                 "power_w_max": max(float(r[2]) for r in rows), "samples": len(rows), "reasons": reasons}
 
 
+def oracle_gossip_sample(cols, steps, warmup):
+    """Times the oracle's gossip step, as it stands (one numpy thread), on the first `cols` columns of
+    all 64 rows.  Returns seconds per call."""
+    import numpy as np
+    from oracle import dpsgd_oracle as orc
+    from paper_1705_09056_b200 import workloads as wl
+    rng = np.random.default_rng(1)
+    X = rng.standard_normal((N_NODES, cols), dtype=np.float32)
+    G = rng.standard_normal((N_NODES, cols), dtype=np.float32)
+    csr = wl.topology("ring", N_NODES)
+    for _ in range(warmup):
+        orc.mix_update(X[:, :cols // 16], G[:, :cols // 16], *csr, GAMMA)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        X = orc.mix_update(X, G, *csr, GAMMA)
+    return (time.perf_counter() - t0) / steps
+
+
+def oracle_sample_text(cols):
+    return (f"first {cols} of {N_PARAMS} columns of all {N_NODES} rows per step (the step acts on every column "
+            "alone); value = replica-steps/s of a full step extrapolated linearly in the columns")
+
+
 def run_reference(args):
     """The CPU oracle, as it stands, on the host cores: a bounded column sample per step."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import numpy as np
-    from oracle import dpsgd_oracle as orc
-    from paper_1705_09056_b200 import workloads as wl
     cols = min(N_PARAMS, max(1, args.ref_cols))
-    rng = np.random.default_rng(1)
-    X = rng.standard_normal((N_NODES, cols), dtype=np.float32)
-    G = rng.standard_normal((N_NODES, cols), dtype=np.float32)
-    csr = wl.topology("ring", N_NODES)
-    for _ in range(args.warmup):
-        orc.mix_update(X[:, :cols // 16], G[:, :cols // 16], *csr, GAMMA)
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        X = orc.mix_update(X, G, *csr, GAMMA)
-    dt = (time.perf_counter() - t0) / args.steps
-    value = N_NODES * (cols / N_PARAMS) / dt
-    sample = f"first {cols} of {N_PARAMS} columns of all {N_NODES} rows per step (the step is separable per column), scaled linearly"
+    dt = oracle_gossip_sample(cols, args.steps, args.warmup)
+    scale = N_PARAMS / cols
+    value = N_NODES / (dt * scale)
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": "replica-steps/s",
-        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3 * N_PARAMS / cols,
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt * 1e3,                      # measured: one call on the sample
+        "sample_to_full_step_scale": scale,           # a full step = scale x the sample
+        "ms_per_full_step_extrapolated": dt * 1e3 * scale,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic", "config": workload_config("ring"),
-        "cpu_baseline": {"value": value, "unit": "replica-steps/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "replica-steps/s", "cores": 1, "kind": "oracle",
+                         "host_cores_available": os.cpu_count(), "sample": oracle_sample_text(cols)},
         "e2e": {"value": value, "unit": "replica-steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
@@ -159,19 +174,139 @@ def time_steps(ctx, steps, warmup, torch):
     return a.elapsed_time(b) / steps    # ms per step == per launch (one kernel per step)
 
 
-def whole_iterations(torch, binding, wl, dev, steps=20, warmup=3):
-    """Whole D-PSGD iterations (sample + gradient + mix + update; consensus distance read once at the end)
-    on the two MLP configurations (the larger one also with the dense averaging matrix, its C-PSGD
-    baseline), two-stage and with the gossip step inside the gradient kernels.
-    Context for the headline line, which times the gossip step alone."""
+# dpsgd_step_consensus after a fused MLP iteration: False while the distance is a pass of its own over the
+# new X; the two-stage ring / uniform gossip kernels always accumulate it on the way.
+FUSED_STEP_CONSENSUS_IN_PASS = False
+
+
+def _event_ms(torch, fn, reps):
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    fn(reps)
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+def _entry(n, ms, launches, bytes_per_step, peak, l2_resident=False):
+    """One timed variant: rate, launches, algorithmic HBM bytes of an iteration and what bounds it."""
+    gbs = bytes_per_step / (ms * 1e-3) / 1e9
+    e = {"ms_per_step": ms, "replica_steps_per_s": n / (ms * 1e-3), "launches_per_step": launches,
+         "algorithmic_bytes_per_step": bytes_per_step, "GBps": gbs}
+    if l2_resident:
+        e["bound"] = f"latency: {launches:g} dependent launches of {ms * 1e3 / max(launches, 1):.1f} us each"
+    else:
+        e["bound"] = "hbm"
+        e["frac_of_measured_peak"] = gbs / peak
+    return e
+
+
+def mlp_bytes(n, dims, fused, consensus_pass):
+    """Algorithmic HBM bytes of one MLP iteration, per replica-parameter of each weight block (fp32):
+    forward reads the weights (4); the input gradient re-reads the hidden layers' weights (4, not layer 1);
+    two stages: the gradient is written (4) and the gossip step reads X and G and writes X' (12);
+    fused: the weight-gradient kernel reads X and writes X' (8); a separate consensus pass reads X' (4)."""
+    P = sum(dims[l + 1] * dims[l] + dims[l + 1] for l in range(len(dims) - 1))
+    hidden = sum(dims[l + 1] * dims[l] for l in range(1, len(dims) - 1))
+    per = 4 * P + 4 * hidden + (8 * P if fused else 16 * P) + (4 * P if consensus_pass else 0)
+    return n * per
+
+
+def oracle_mlp_baseline(orc, w, nodes, cols):
+    """Oracle, one numpy thread: gradients of `nodes` of the n nodes and the gossip step on the first `cols`
+    columns of all rows, each scaled linearly to the whole iteration."""
+    import numpy as np
+    A, y, x0 = w.A[:nodes].cpu().numpy(), w.y[:nodes].cpu().numpy(), w.x0.cpu().numpy()
+    idx = orc.sample_indices(1, 0, w.n, w.batch, w.m_per_node)
+    t0 = time.perf_counter()
+    for i in range(nodes):
+        orc.grad_mlp(x0, w.dims, A[i], y[i], idx[i])
+    t_grad = (time.perf_counter() - t0) * w.n / nodes
+    cols = min(cols, w.N)
+    X = np.tile(x0[:cols], (w.n, 1))
+    t0 = time.perf_counter()
+    orc.mix_update(X, X, *w.csr(), w.gamma)
+    t_mix = (time.perf_counter() - t0) * w.N / cols
+    return {"value": w.n / (t_grad + t_mix), "unit": "replica-steps/s", "cores": 1, "kind": "oracle",
+            "host_cores_available": os.cpu_count(),
+            "sample": f"gradients of {nodes} of {w.n} nodes and the gossip step on the first {cols} of {w.N} columns, "
+                      f"each scaled linearly to one whole iteration ({t_grad:.2f} s + {t_mix:.2f} s)"}
+
+
+def linear_iterations(torch, binding, wl, dev, peak, cpu_legs, steps=200, warmup=10):
+    """Configurations 1 and 2 (least squares n=8; logistic regression n=16 with 65536 x 4096 samples per node):
+    whole iterations per dpsgd_step call and enqueued by one dpsgd_run call."""
+    import numpy as np
     out = {}
-    for name, idx, topo in (("mlp_784-1024-10_n32_ring", 2, "ring"), ("mlp_1024-2048-2048-10_n112_ring", 4, "ring"),
-                            ("mlp_1024-2048-2048-10_n112_dense_cpsgd_averaging", 4, "dense")):
+    for name, idx in (("lsq_64_n8_ring", 0), ("logistic_4096_n16_ring_65536_samples_per_node", 1)):
+        free, _ = torch.cuda.mem_get_info()
+        if idx == 1 and free < 24 * 2 ** 30:
+            out[name] = {"skipped": "needs 24 GiB of free device memory for the 17.2 GB dataset"}
+            continue
+        w = wl.config(idx, device=dev)
+        X0 = wl.stack_rows(w.x0, w.n, w.ld)
+        X1, G = torch.zeros_like(X0), torch.zeros_like(X0)
+        ctx = binding.Dpsgd(w.n, w.N, *w.csr(), gamma=w.gamma, seed=1)
+        ctx.bind(X0, X1, G)
+        ctx.set_model(w.model, w.dims, w.l2_lambda, w.batch, 0)
+        ctx.set_data(w.A, w.y)
+        for k in range(warmup):
+            ctx.step(k)
+        ctx.run(warmup, 16)                 # first use of the replay path (captures its graph where it applies)
+        # sampled rows are read once (second use from the chip), then the 12 B/unit gossip step
+        bytes_step = 4 * w.n * w.batch * (w.dims[0] + 1) + 12 * w.n * w.N
+        l0 = ctx.launch_count()
+        ms_step = _event_ms(torch, lambda r: [ctx.step(100 + k) for k in range(r)], steps)
+        launches = (ctx.launch_count() - l0) / steps
+        l0 = ctx.launch_count()
+        ms_run = _event_ms(torch, lambda r: ctx.run(1000, r), steps)
+        launches_run = (ctx.launch_count() - l0) / steps
+        res = {"n": w.n, "N": w.N, "batch": w.batch, "iterations_of_the_configuration": w.iterations,
+               "per_dpsgd_step_call": _entry(w.n, ms_step, launches, bytes_step, peak, l2_resident=True),
+               "one_dpsgd_run_call": _entry(w.n, ms_run, launches_run, bytes_step, peak, l2_resident=True)}
+        ctx.sync()
+        if cpu_legs:
+            from oracle import dpsgd_oracle as orc
+            reps = 20 if idx == 0 else 3
+            ids = orc.sample_indices(1, 0, w.n, w.batch, w.m_per_node)
+            it = torch.from_numpy(ids.astype(np.int64)).to(dev)
+            node = torch.arange(w.n, device=dev)[:, None]
+            A_s, y_s = w.A[node, it].cpu().numpy(), w.y[node, it].cpu().numpy()     # the sampled rows only
+            local = np.tile(np.arange(w.batch, dtype=np.int32), (w.n, 1))
+            X = np.zeros((w.n, w.N), dtype=np.float32)
+            t0 = time.perf_counter()
+            for _ in range(reps):
+                Gr = orc.gradients(X, w.model, w.dims, A_s, y_s, local, w.l2_lambda)
+                X = orc.mix_update(X, Gr, *w.csr(), w.gamma)
+            dt = (time.perf_counter() - t0) / reps
+            res["cpu_baseline"] = {"value": w.n / dt, "unit": "replica-steps/s", "cores": 1, "kind": "oracle",
+                                   "host_cores_available": os.cpu_count(),
+                                   "sample": f"{reps} whole iterations (gradients of all {w.n} nodes + gossip step) on the "
+                                             "rows one minibatch draws, gathered outside the timed region"}
+        ctx.close()
+        out[name] = res
+        del X0, X1, G, w
+        torch.cuda.empty_cache()
+    return out
+
+
+def mlp_iterations(torch, binding, wl, dev, peak, cpu_legs, steps=20, warmup=3):
+    """Configurations 3 and 5: whole iterations, two-stage and with the gossip step inside the gradient
+    kernels.  Configuration 5 (n = 112, ring beside the averaging matrix of C-PSGD) is defined as reporting
+    the consensus distance in every iteration, so dpsgd_step_consensus is the timed call there; the same
+    iterations without the distance are given beside it."""
+    out = {}
+    for name, idx, topo, per_step_consensus in (
+            ("mlp_784-1024-10_n32_ring", 2, "ring", False),
+            ("mlp_1024-2048-2048-10_n112_ring", 4, "ring", True),
+            ("mlp_1024-2048-2048-10_n112_dense_cpsgd_averaging", 4, "dense", True)):
         w = wl.config(idx, device=dev, topology=topo)
         X0 = wl.stack_rows(w.x0, w.n, w.ld)
         X1, G = torch.zeros_like(X0), torch.zeros_like(X0)
         log = torch.zeros(steps + warmup, dtype=torch.float64, device=dev)
-        res = {"n": w.n, "N": w.N, "batch": w.batch}
+        res = {"n": w.n, "N": w.N, "batch": w.batch, "iterations_of_the_configuration": w.iterations}
+        l2_resident = 3 * w.n * w.ld * 4 < 126e6 * 3          # configuration 3: X (104 MB) stays in L2
         for label, mode in (("two_stage", 0), ("fused", 1)):
             X0.copy_(wl.stack_rows(w.x0, w.n, w.ld))
             ctx = binding.Dpsgd(w.n, w.N, *w.csr(), gamma=w.gamma, seed=1)
@@ -179,24 +314,38 @@ def whole_iterations(torch, binding, wl, dev, steps=20, warmup=3):
             ctx.set_model(w.model, w.dims, w.l2_lambda, w.batch, 0)
             ctx.set_data(w.A, w.y)
             ctx.set_fused_step(mode)
-            for k in range(warmup):
-                ctx.step(k)
-            torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            l0 = ctx.launch_count()
-            a.record()
-            for k in range(steps):
-                ctx.step(warmup + k)
-            b.record()
-            torch.cuda.synchronize()
-            ms = a.elapsed_time(b) / steps
-            res[label] = {"ms_per_step": ms, "replica_steps_per_s": w.n / (ms * 1e-3),
-                          "launches_per_step": (ctx.launch_count() - l0) / steps,
-                          "consensus_dist": ctx.consensus_dist()}
+            variants = [("", lambda k: ctx.step(k), False)]
+            if per_step_consensus:
+                variants = [("_consensus_every_step", lambda k: ctx.step_consensus(k, log[k:k + 1]), True)] + variants
+            for suffix, call, with_c in variants:
+                for k in range(warmup):
+                    call(k)
+                l0 = ctx.launch_count()
+                ms = _event_ms(torch, lambda r: [call(warmup + k) for k in range(r)], steps)
+                launches = (ctx.launch_count() - l0) / steps
+                # the distance costs a pass of its own unless the gossip kernel accumulates it on the way
+                own_pass = with_c and mode == 1 and not FUSED_STEP_CONSENSUS_IN_PASS
+                e = _entry(w.n, ms, launches, mlp_bytes(w.n, w.dims, mode == 1, own_pass), peak, l2_resident)
+                if with_c:
+                    e["consensus_dist_last_step"] = float(log[warmup + steps - 1])
+                    e["consensus_pass"] = "separate pass over the new X" if own_pass else "inside the gossip kernels"
+                res[label + suffix] = e
+            res[label]["consensus_dist"] = ctx.consensus_dist()
             ctx.close()
+        if cpu_legs:
+            from oracle import dpsgd_oracle as orc
+            res["cpu_baseline"] = oracle_mlp_baseline(orc, w, nodes=4, cols=500_000)
         out[name] = res
         del X0, X1, G, w
         torch.cuda.empty_cache()
+    return out
+
+
+def whole_iterations(torch, binding, wl, dev, peak, cpu_legs=True):
+    """Whole D-PSGD iterations (sample + gradient + mix + update) of the four model configurations.
+    Context for the headline line, which times the gossip step alone on configuration 4."""
+    out = linear_iterations(torch, binding, wl, dev, peak, cpu_legs)
+    out.update(mlp_iterations(torch, binding, wl, dev, peak, cpu_legs))
     return out
 
 
@@ -302,26 +451,17 @@ def run_ours(args):
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        import numpy as np
-        from oracle import dpsgd_oracle as orc
         cols = ORACLE_SAMPLE_COLS
-        rng = np.random.default_rng(1)
-        Xs = rng.standard_normal((n, cols), dtype=np.float32)
-        Gs = rng.standard_normal((n, cols), dtype=np.float32)
-        csr = wl.topology("ring", n)
-        t0 = time.perf_counter()
-        orc.mix_update(Xs, Gs, *csr, GAMMA)
-        dt = time.perf_counter() - t0
-        cpu = {"value": n * (cols / N) / dt, "unit": "replica-steps/s", "cores": 1, "kind": "oracle",
-               "host_cores_available": os.cpu_count(), "seconds": dt,
-               "sample": f"one step on the first {cols} of {N} columns of all {n} rows "
-                         "(separable per column), scaled linearly to a full step"}
+        dt = oracle_gossip_sample(cols, 2, 1)
+        cpu = {"value": n / (dt * N / cols), "unit": "replica-steps/s", "cores": 1, "kind": "oracle",
+               "host_cores_available": os.cpu_count(), "seconds_per_sample_step": dt,
+               "sample": oracle_sample_text(cols)}
 
     iterations = None
     if world == 1 and not args.no_iterations:
         del X0, X1, G
         torch.cuda.empty_cache()
-        iterations = whole_iterations(torch, binding, wl, dev)
+        iterations = whole_iterations(torch, binding, wl, dev, peak, cpu_legs=not args.no_cpu_baseline)
 
     ring = results["ring"]
     line = {
@@ -333,7 +473,7 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "kernel": "mix_ring_kernel", "achieved": ring["GBps"], "peak": peak,
                      "peak_source": f"{peak_kind} HBM copy bandwidth (GB/s)", "unit": "GB/s",
                      "frac": ring["GBps"] / peak, "frac_of_nominal_8TBps": ring["GBps"] / NOMINAL_HBM_GBS,
-                     "algorithmic_bytes_per_launch": bytes_per_launch, "traffic": TRAFFIC_BYTES_PER_LAUNCH},
+                     "algorithmic_bytes_per_launch": bytes_per_launch, "traffic": traffic_bytes_per_launch()},
         "cpu_baseline": cpu, "topologies": results, "iterations": iterations,
     }
     print(json.dumps(line))
@@ -343,8 +483,20 @@ def run_ours(args):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one mix_ring_kernel launch.  Captured with ncu on
 # n = 64 x N = 2,000,000 (1.499 GB against 1.536 GB algorithmic) and scaled by 25,000,000 / 2,000,000:
-# traffic grows in proportion to N.  Set to None whenever mix_ring_kernel changes.
-TRAFFIC_BYTES_PER_LAUNCH = 18.74e9
+# traffic grows in proportion to N.  The figure belongs to the kernel source it was captured from: when
+# the file's hash differs, the line reports null until the counters are taken again.
+TRAFFIC_CAPTURE = {"bytes_per_launch": 18.74e9, "source": "paper_1705_09056_b200/csrc/mix_update.cu",
+                   "sha256_16": "e24eac603b395f6a"}
+
+
+def traffic_bytes_per_launch():
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, TRAFFIC_CAPTURE["source"]), "rb") as f:
+            same = hashlib.sha256(f.read()).hexdigest()[:16] == TRAFFIC_CAPTURE["sha256_16"]
+    except OSError:
+        same = False
+    return TRAFFIC_CAPTURE["bytes_per_launch"] if same else None
 
 
 def main():
@@ -354,7 +506,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--ref-cols", type=int, default=1_000_000,
+    ap.add_argument("--ref-cols", type=int, default=ORACLE_SAMPLE_COLS,
                     help="columns per step of the CPU reference arm (bounded sample)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-iterations", action="store_true",

@@ -23,6 +23,13 @@
  *    unless stated otherwise.  Calls on one context must not overlap in time.
  *  - There is no CPU fallback: without a CUDA device every compute call fails with
  *    DPSGD_ERR_CUDA.
+ *  - Device code never traps.  The kernels that wait for tile copies (the tiled gossip kernel, the
+ *    tensor-core gradient kernels) bound every wait; a wait that runs out raises a status word in
+ *    device memory, the CTA skips its tile and returns, and the NEXT call that waits for the
+ *    stream reports DPSGD_ERR_TIMEOUT once and clears the word: dpsgd_sync, dpsgd_consensus_dist,
+ *    dpsgd_mix_update_host, dpsgd_set_model, dpsgd_set_node_batches, dpsgd_destroy.  X is not
+ *    valid after such a report.  The asynchronous calls (dpsgd_step, dpsgd_mix_update, ...)
+ *    cannot see it; end a run with dpsgd_sync before trusting X.
  *
  * Stacked layout: row i of X / G starts at element i*ld; ld >= N, ld a multiple of 32 floats
  * (128 bytes), base pointers 128-byte aligned.  Padding columns [N, ld) must be zero in X and
@@ -67,7 +74,7 @@ enum {
 };
 
 /*
- * Inputs of Algorithm 1 ("Require: step length gamma, weight matrix W"): creates a context
+ * Inputs of Algorithm 1 (its step length gamma and weight matrix W): creates a context
  * for n nodes with N parameters each.  W comes as host CSR (row_ptr[n+1], col_idx[nnz],
  * val[nnz]); it is validated against Section 3's definition and copied:
  *   square; column indices in range, strictly increasing inside a row; 0 <= W_ij <= 1;
@@ -234,6 +241,24 @@ DPSGD_API dpsgd_status dpsgd_run(dpsgd_ctx* ctx, uint64_t k_first, int64_t itera
  * of Eq. 13), accumulated in fp64.  Waits for the stream and writes one double to host memory.
  */
 DPSGD_API dpsgd_status dpsgd_consensus_dist(dpsgd_ctx* ctx, double* out_host);
+
+/*
+ * Waits for everything enqueued on the bound stream and reports what the device recorded meanwhile:
+ * DPSGD_ERR_TIMEOUT if a kernel's bounded wait ran out since the last synchronising call (the word is
+ * cleared, so the next report concerns later work), DPSGD_ERR_CUDA if the stream failed, else
+ * DPSGD_OK.  The barrier of Algorithm 1 between iterations needs no such call: kernel boundaries on
+ * the stream are that barrier.  Call it before reading X on another stream or trusting a run.
+ */
+DPSGD_API dpsgd_status dpsgd_sync(dpsgd_ctx* ctx);
+
+/*
+ * Self-test of the give-up path (no counterpart in the paper): enqueues one small CTA that waits on a
+ * barrier at which nothing ever arrives, with the kernels' bounded wait cut to max_polls polls
+ * (1 .. 2^20; a poll takes well under a microsecond).  The CTA then raises the status word and
+ * returns; it faults nothing and holds nothing.  The next synchronising call returns
+ * DPSGD_ERR_TIMEOUT, and the context stays usable.  X, G and the iteration state are not touched.
+ */
+DPSGD_API dpsgd_status dpsgd_selftest_wait(dpsgd_ctx* ctx, uint32_t max_polls);
 
 /* Output of Algorithm 1: xbar = (1/n) sum_i x_i into xbar_dev (fp32 [ld], 16-byte aligned). */
 DPSGD_API dpsgd_status dpsgd_average(dpsgd_ctx* ctx, float* xbar_dev);

@@ -33,7 +33,7 @@ MODEL_LOGISTIC = 1
 MODEL_MLP = 2
 
 # ------------------------------------------------------------------------------------------
-# Algorithm 1, step "randomly sample xi_{k,i} from local data of node i".
+# Algorithm 1 step 2: every node draws xi_{k,i} from its own local data.
 # The paper fixes no generator; this implementation uses the counter-based Philox4x32-10 of Salmon,
 # Moraes, Dror and Shaw (SC'11), keyed by the run seed, with the counter holding
 # (draw block, node, iteration).
@@ -86,7 +86,7 @@ def sample_indices(seed: int, k: int, n: int, B: int, m: int) -> np.ndarray:
 
 
 # ------------------------------------------------------------------------------------------
-# Algorithm 1, step "compute a local stochastic gradient at x_{k,i}" (minibatch mean,
+# Algorithm 1 step 3: the local stochastic gradient at the node's own x_{k,i} (minibatch mean,
 # footnote a).  One node at a time; x is that node's fp32 parameter row.
 # ------------------------------------------------------------------------------------------
 

@@ -47,6 +47,8 @@ SIGNATURES = {
     "dpsgd_mix_update_consensus": [_vp, _vp],
     "dpsgd_step_consensus": [_vp, _u64, _vp],
     "dpsgd_consensus_dist": [_vp, ctypes.POINTER(ctypes.c_double)],
+    "dpsgd_sync": [_vp],
+    "dpsgd_selftest_wait": [_vp, ctypes.c_uint32],
     "dpsgd_average": [_vp, _vp],
     "dpsgd_mix_update_host": [_vp, _vp, _i64, ctypes.POINTER(ctypes.c_double)],
     "dpsgd_consensus_dist_noalloc": [_vp, _i32, _i64, _i64, _vp, _vp],
@@ -244,6 +246,14 @@ class Dpsgd:
         out = ctypes.c_double()
         self._check(self._lib.dpsgd_consensus_dist(self._h, ctypes.byref(out)))
         return out.value
+
+    def sync(self):
+        """Waits for the bound stream; raises ERR_TIMEOUT if a kernel's bounded wait ran out meanwhile."""
+        self._check(self._lib.dpsgd_sync(self._h))
+
+    def selftest_wait(self, max_polls: int = 4096):
+        """Enqueues the self-test CTA whose wait runs out (see dpsgd_selftest_wait)."""
+        self._check(self._lib.dpsgd_selftest_wait(self._h, max_polls))
 
     def average(self, xbar: Optional[torch.Tensor] = None) -> torch.Tensor:
         if xbar is None:

@@ -143,6 +143,24 @@ void release(dpsgd_ctx* c) {
     delete c;
 }
 
+// Copies the device status word back, waits for the stream and clears the word when a kernel set it.
+// DPSGD_ERR_TIMEOUT when a bounded device-side wait ran out since the last check.
+dpsgd_status collect_device_status(dpsgd_ctx* c) {
+    if (!c->d_result || !c->h_result) return DPSGD_OK;
+    cudaError_t e = cudaMemcpyAsync(&c->h_result->status, &c->d_result->status, sizeof(int), cudaMemcpyDeviceToHost,
+                                    c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "stream synchronisation");
+    if (c->h_result->status != 0) {
+        c->h_result->status = 0;
+        e = cudaMemsetAsync(&c->d_result->status, 0, sizeof(int), c->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+        return fail(c, DPSGD_ERR_TIMEOUT,
+                    "a kernel gave up waiting for a tile copy since the last synchronising call; X is not valid");
+    }
+    return DPSGD_OK;
+}
+
 dpsgd_status need_bound(dpsgd_ctx* c) {
     if (!c) return DPSGD_ERR_ARG;
     if (!c->bound) return fail(c, DPSGD_ERR_STATE, "no buffers bound: call dpsgd_bind first");
@@ -263,9 +281,9 @@ DPSGD_API dpsgd_status dpsgd_create(dpsgd_ctx** out, int32_t n, int64_t N, const
 
 DPSGD_API dpsgd_status dpsgd_destroy(dpsgd_ctx* c) {
     if (!c) return DPSGD_ERR_ARG;
-    if (c->bound) cudaStreamSynchronize(c->stream);
+    const dpsgd_status s = c->bound ? collect_device_status(c) : DPSGD_OK;
     release(c);
-    return DPSGD_OK;
+    return s == DPSGD_ERR_TIMEOUT ? s : DPSGD_OK;
 }
 
 DPSGD_API dpsgd_status dpsgd_bind(dpsgd_ctx* c, float* X0, float* X1, float* G, int64_t ld, void* stream) {
@@ -323,7 +341,8 @@ DPSGD_API dpsgd_status dpsgd_set_model(dpsgd_ctx* c, int32_t kind, const int32_t
                  (long long)want, (long long)c->N);
         return fail(c, DPSGD_ERR_ARG, buf);
     }
-    if (c->bound) cudaStreamSynchronize(c->stream);
+    const dpsgd_status pending = c->bound ? collect_device_status(c) : DPSGD_OK;
+    if (pending != DPSGD_OK) return pending;
     drop_graph(c);
     cudaFree(c->d_idx); cudaFree(c->d_coef); cudaFree(c->d_act); cudaFree(c->d_delta);
     cudaFree(c->d_node_batch);
@@ -441,8 +460,9 @@ DPSGD_API dpsgd_status dpsgd_set_node_batches(dpsgd_ctx* c, const int32_t* batch
     if (!c) return DPSGD_ERR_ARG;
     if (c->model < 0) return fail(c, DPSGD_ERR_STATE, "call dpsgd_set_model before dpsgd_set_node_batches");
     drop_graph(c);
-    cudaError_t e = cudaStreamSynchronize(c->stream);   // kernels in flight may still read the old sizes
-    if (e != cudaSuccess) return cuda_fail(c, e, "dpsgd_set_node_batches");
+    cudaError_t e = cudaSuccess;
+    const dpsgd_status pending = collect_device_status(c);   // waits: kernels in flight may still read the old sizes
+    if (pending != DPSGD_OK) return pending;
     if (!batch_host) {
         cudaFree(c->d_node_batch);
         c->d_node_batch = nullptr;
@@ -678,10 +698,24 @@ DPSGD_API dpsgd_status dpsgd_consensus_dist(dpsgd_ctx* c, double* out) {
     if (e != cudaSuccess) return cuda_fail(c, e, "consensus distance");
     *out = c->h_result->value;
     if (c->h_result->status != 0) {
+        c->h_result->status = 0;
         cudaMemsetAsync(&c->d_result->status, 0, sizeof(int), c->stream);
-        return fail(c, DPSGD_ERR_TIMEOUT, "a kernel gave up waiting for a tile copy; X is not valid");
+        return fail(c, DPSGD_ERR_TIMEOUT,
+                    "a kernel gave up waiting for a tile copy since the last synchronising call; X is not valid");
     }
     return DPSGD_OK;
+}
+
+DPSGD_API dpsgd_status dpsgd_sync(dpsgd_ctx* c) {
+    if (!c) return DPSGD_ERR_ARG;
+    return collect_device_status(c);
+}
+
+DPSGD_API dpsgd_status dpsgd_selftest_wait(dpsgd_ctx* c, uint32_t max_polls) {
+    if (!c) return DPSGD_ERR_ARG;
+    if (max_polls < 1 || max_polls > (1u << 20)) return fail(c, DPSGD_ERR_ARG, "max_polls must be in [1, 2^20]");
+    cudaError_t e = launch_wait_probe(c, max_polls);
+    return e == cudaSuccess ? DPSGD_OK : cuda_fail(c, e, "wait probe kernel");
 }
 
 DPSGD_API dpsgd_status dpsgd_average(dpsgd_ctx* c, float* xbar) {

@@ -209,9 +209,28 @@ extern "C" DPSGD_API dpsgd_status dpsgd_consensus_dist_noalloc(const float* X_de
                  "use a context and dpsgd_consensus_dist instead", (long long)ld, (long long)kNoAllocMaxLd);
         return noalloc_fail(DPSGD_ERR_UNSUPPORTED, buf);
     }
+    // Both pointers must be memory of the CURRENT device: the scratch address below belongs to it, and
+    // a kernel handed another GPU's pointer would fault.  The query allocates nothing.
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return noalloc_fail(DPSGD_ERR_CUDA, std::string("cudaGetDevice: ") + cudaGetErrorString(e));
+    const void* ptrs[2] = {X_dev, out_dev};
+    for (const void* p : ptrs) {
+        cudaPointerAttributes attr;
+        e = cudaPointerGetAttributes(&attr, p);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return noalloc_fail(DPSGD_ERR_ARG, std::string("X_dev / out_dev is not a CUDA pointer: ") + cudaGetErrorString(e));
+        }
+        if (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged)
+            return noalloc_fail(DPSGD_ERR_ARG, "X_dev and out_dev must be device memory");
+        if (attr.type == cudaMemoryTypeDevice && attr.device != dev)
+            return noalloc_fail(DPSGD_ERR_ARG, "X_dev and out_dev must belong to the current device");
+    }
     double* partials = nullptr;
-    cudaError_t e = noalloc_scratch(&partials);
+    e = noalloc_scratch(&partials);
     if (e != cudaSuccess) return noalloc_fail(DPSGD_ERR_CUDA, std::string("scratch set-up: ") + cudaGetErrorString(e));
+    cudaGetLastError();   // an error left by an earlier launch on this thread is not this call's
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int64_t ld4 = ld / 4;
     const int grid = (int)((ld4 + kThreads - 1) / kThreads);

@@ -134,6 +134,8 @@ cudaError_t launch_mix_rowpar(dpsgd_ctx* c, const float* X, const float* G, floa
 bool mix_is_small(const dpsgd_ctx* c);
 cudaError_t launch_mix_tiled(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
 bool mix_tiled_supported(const dpsgd_ctx* c);
+// One CTA that waits, with the kernels' bounded wait cut to max_polls polls, on an mbarrier nothing arrives at.
+cudaError_t launch_wait_probe(dpsgd_ctx* c, uint32_t max_polls);
 void mix_tiled_release(dpsgd_ctx* c);
 
 cudaError_t launch_consensus(dpsgd_ctx* c, const float* X, double* result_dev);

@@ -203,10 +203,28 @@ mix_tiled_kernel(const __grid_constant__ CUtensorMap mapX, const float4* __restr
                 __stcs(out + (int64_t)i * ld4, a);
             }
         }
+        // the swapped order rewrote the X tile with ordinary stores; order them before the bulk copy that
+        // refills the stage (generic-proxy writes against the async proxy)
+        if (SWAPPED) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncthreads();                       // everyone is done reading stage s
         if (it + S < my_tiles) issue(it + S, s);
         if (++s == S) { s = 0; parity ^= 1u; }
     }
+}
+
+// The give-up path of the bounded waits, on its own: one mbarrier that expects an arrival nobody makes.
+// After max_polls unsuccessful polls the CTA raises the status word, exactly as mix_tiled_kernel does, and
+// returns; it holds nothing else (no copy in flight, no tensor memory).
+__global__ void wait_probe_kernel(uint32_t max_polls, int* __restrict__ status) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    bool done = false;
+    for (uint32_t spin = 0; spin < max_polls && !done; ++spin) done = mbar_try_wait(&bar, 0);
+    if (!done && threadIdx.x == 0) atomicExch(status, (int)DPSGD_ERR_TIMEOUT);
 }
 
 bool make_map(CUtensorMap* map, const float* base, int n, int64_t ld, int T) {
@@ -289,6 +307,12 @@ void mix_tiled_release(dpsgd_ctx* c) {
     cudaFree(st->d_nz);
     delete st;
     c->tma_state = nullptr;
+}
+
+cudaError_t launch_wait_probe(dpsgd_ctx* c, uint32_t max_polls) {
+    wait_probe_kernel<<<1, 32, 0, c->stream>>>(max_polls, &c->d_result->status);
+    c->launches++;
+    return cudaGetLastError();
 }
 
 cudaError_t launch_mix_tiled(dpsgd_ctx* c, const float* X, const float* G, float* Xn) {

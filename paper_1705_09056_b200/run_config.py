@@ -1,8 +1,12 @@
-"""Runs whole D-PSGD iterations (sample + gradient + mix + update) of one model configuration
-and prints CUDA-event timings: replica-steps/s and the split between gradient and gossip step.
+"""The measurement command of the package: runs one configuration a few times and prints CUDA-event
+timings as one JSON line.  Also the command to put under a profiler for a single kernel.
 
   python -m paper_1705_09056_b200.run_config --config 2 --steps 50
-  (0 least squares, 1 logistic, 2 MLP 784-1024-10, 4 MLP 1024-2048-2048-10)
+      whole D-PSGD iterations (sample + gradient + mix + update): replica-steps/s and the split
+      between gradient and gossip step (0 least squares, 1 logistic, 2 MLP 784-1024-10,
+      4 MLP 1024-2048-2048-10)
+  python -m paper_1705_09056_b200.run_config --config 3 --n 64 --N 2000000 --topology ring --steps 3
+      the gossip step alone on supplied N(0,1) gradients (the bandwidth configuration, any shape)
 """
 from __future__ import annotations
 
@@ -14,12 +18,55 @@ import torch
 from . import binding, build, workloads as wl
 
 
+def gossip_step_alone(args, dev):
+    """dpsgd_mix_update (or dpsgd_mix_update_consensus) on an n x N matrix with supplied gradients."""
+    n, N = args.n or 64, args.N or 25_000_000
+    topology = args.topology or "ring"
+    ld = wl.padded_ld(N)
+    X0 = wl.stress_matrix(n, ld, N, 1, dev)
+    X1 = torch.zeros_like(X0)
+    G = wl.stress_matrix(n, ld, N, 2, dev)
+    ctx = binding.Dpsgd(n, N, *wl.topology(topology, n), gamma=0.01)
+    ctx.bind(X0, X1, G)
+    if args.kind >= 0:
+        ctx.mix_kind(args.kind)
+    if args.swapped:
+        ctx.set_order(True)
+    if args.momentum > 0.0:
+        V = torch.zeros_like(X0)
+        ctx.set_momentum(args.momentum, V)
+    out = torch.zeros(1, dtype=torch.float64, device=dev)
+    step = (lambda: ctx.mix_update_consensus(out)) if args.fused_consensus else ctx.mix_update
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        step()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / max(1, args.steps)
+    res = {"workload": "stress", "n": n, "N": N, "topology": topology,
+           "kernel": binding.MIX_NAMES[ctx.mix_kind()], "ms_per_step": ms,
+           "GBps": (20.0 if args.momentum > 0.0 else 12.0) * n * N / (ms * 1e-3) / 1e9}
+    if args.consensus:
+        res["consensus"] = ctx.consensus_dist()
+    ctx.sync()
+    print(json.dumps(res))
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--config", type=int, default=2, choices=[0, 1, 2, 4])
+    ap.add_argument("--config", type=int, default=2, choices=[0, 1, 2, 3, 4])
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--n", type=int, default=0, help="override the node count")
+    ap.add_argument("--N", type=int, default=0, help="config 3: parameters per replica (default 25,000,000)")
+    ap.add_argument("--kind", type=int, default=-1, help="config 3: force a DPSGD_MIX_* kernel")
+    ap.add_argument("--momentum", type=float, default=0.0,
+                    help="config 3: momentum of the Section 5.3 runs (one more matrix)")
     ap.add_argument("--m", type=int, default=0, help="override the local dataset size")
     ap.add_argument("--topology", default="")
     ap.add_argument("--precision", type=int, default=0, help="MLP: 0 fp32-faithful, 1 single TF32 pass")
@@ -35,6 +82,8 @@ def main():
 
     build.build()
     dev = torch.device("cuda", 0)
+    if args.config == 3:
+        return gossip_step_alone(args, dev)
     over = {}
     if args.n:
         over["n"] = args.n

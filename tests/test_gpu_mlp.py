@@ -9,7 +9,9 @@ from gpu_util import GpuRun, row_rel_err, mlp_oracle_grad_matching_gates, TOL_ST
 
 pytestmark = pytest.mark.gpu
 
-TOL_G = 5e-5      # row-wise relative error of the gradient against the fp64 oracle (3 x TF32 products: ~2^-20 each)
+# row-wise relative error of the gradient against the fp64 oracle, by arithmetic of the products:
+# tensor cores (three TF32 MMAs on split operands, ~2^-20 per product) and exact fp32 FMA
+TOL_G = {0: 5e-5, 2: 2e-5}
 
 
 def _setup(w, seed, precision=0, X=None):
@@ -52,7 +54,7 @@ def test_mlp_gradient_and_step_match_oracle(n, dims, m, B, precision):
         assert np.array_equal(run.ctx.sample(k).cpu().numpy(), o.sample(k))
         run.ctx.grad(k)
         G_ref, _ = mlp_oracle_grad_matching_gates(orc, o, k, run.g())
-        assert row_rel_err(run.g(), G_ref) <= TOL_G
+        assert row_rel_err(run.g(), G_ref) <= TOL_G[precision]
         if run.ld > w.N:
             assert float(run.G[:, w.N:].abs().max()) == 0.0
         # per-layer check so that a wrong block cannot hide behind a large one
@@ -61,7 +63,7 @@ def test_mlp_gradient_and_step_match_oracle(n, dims, m, B, precision):
             for size in (dims[l + 1] * dims[l], dims[l + 1]):
                 blk_ref, blk = G_ref[:, off:off + size], run.g()[:, off:off + size]
                 scale = np.linalg.norm(blk_ref.astype(np.float64), axis=1).max()
-                assert np.abs(blk.astype(np.float64) - blk_ref).max() <= 5e-5 * max(scale, 1e-12), (l, size)
+                assert np.abs(blk.astype(np.float64) - blk_ref).max() <= TOL_G[precision] * max(scale, 1e-12), (l, size)
                 off += size
         X_ref = o.mix_update(G_ref)
         run.ctx.mix_update()
@@ -125,5 +127,5 @@ def test_mlp_large_batch_uses_fma_kernel():
     run, o = _setup(w, seed=5)
     run.ctx.grad(0)
     G_ref, _ = mlp_oracle_grad_matching_gates(orc, o, 0, run.g())
-    assert row_rel_err(run.g(), G_ref) <= TOL_G
+    assert row_rel_err(run.g(), G_ref) <= TOL_G[2]
     run.close()

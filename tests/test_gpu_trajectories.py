@@ -1,0 +1,303 @@
+"""Free-running trajectories at the configurations' own lengths: the library and the oracle both run
+Algorithm 1 for T iterations from the same start WITHOUT being resynchronised, and are compared on
+what the target fixes: sampled indices bit for bit every iteration, rows of X_T within 1e-3
+(max_i ||x_i - x_i^oracle|| / ||x_i^oracle||), node average within 1e-4.
+
+The oracle's functions are called as they stand; the tests only spread its independent pieces (one
+node's gradient, one block of columns of the gossip step) over host threads.
+
+When DPSGD_TRAJ_LOG names a file, every test appends its per-checkpoint errors to it as JSON lines.
+"""
+import json
+import os
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import dpsgd_oracle as orc
+from paper_1705_09056_b200 import binding, workloads as wl
+from gpu_util import row_rel_err, TOL_TRAJ, TOL_AVG, GATE_REL
+
+pytestmark = pytest.mark.gpu
+
+POOL = ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1))
+
+
+def _need(gib):
+    free, _ = torch.cuda.mem_get_info()
+    if free < gib * 2 ** 30:
+        pytest.skip(f"needs {gib} GiB of device memory")
+
+
+def _log(record):
+    path = os.environ.get("DPSGD_TRAJ_LOG")
+    if path:
+        with open(path, "a") as f:
+            f.write(json.dumps(record) + "\n")
+
+
+def avg_rel_err(got, ref):
+    a_ref = orc.node_average(ref)
+    a = got.astype(np.float64).mean(axis=0)
+    return float(np.linalg.norm(a - a_ref) / max(np.linalg.norm(a_ref), 1e-30))
+
+
+def oracle_mix_update_blocks(o, G, block=65536):
+    """o.mix_update(G), one block of columns per thread (the gossip step acts on every column alone)."""
+    f = orc.mix_update_swapped if o.swapped else orc.mix_update
+    cuts = list(range(0, o.N, block)) + [o.N]
+    parts = list(POOL.map(lambda c: f(o.X[:, c[0]:c[1]], G[:, c[0]:c[1]], o.row_ptr, o.col, o.val, o.gamma),
+                          zip(cuts[:-1], cuts[1:])))
+    o.X = np.concatenate(parts, axis=1)
+    return o.X
+
+
+def oracle_mlp_step(o, k):
+    """One oracle iteration of an MLP run: the n nodes' gradients (one per thread), then the gossip step."""
+    idx = o.sample(k)
+    rows = list(POOL.map(lambda i: orc.grad_mlp(o.X[i], o.dims, o.A[i], o.y[i], idx[i]).astype(np.float32),
+                         range(o.n)))
+    return oracle_mix_update_blocks(o, np.stack(rows))
+
+
+def _context(w, seed, mode=None):
+    X0 = wl.stack_rows(w.x0, w.n, w.ld)
+    X1, G = torch.zeros_like(X0), torch.zeros_like(X0)
+    ctx = binding.Dpsgd(w.n, w.N, *w.csr(), gamma=w.gamma, seed=seed)
+    ctx.bind(X0, X1, G)
+    ctx.set_model(w.model, w.dims, w.l2_lambda, w.batch, 0)
+    ctx.set_data(w.A, w.y)
+    if mode is not None:
+        ctx.set_fused_step(mode)
+    ctx._bufs = (X0, X1, G)
+    return ctx
+
+
+def test_config2_logistic_1000_iterations_full_data():
+    """n = 16 ring, 65536 x 4096 samples per node on the device (17.2 GB), minibatch 128, gamma 0.1,
+    T = 1000.  The oracle is handed the rows its own indices select; the library's indices must
+    equal them in every iteration."""
+    _need(24)
+    w = wl.config(1, device="cuda")
+    seed, T = 20251, w.iterations
+    assert T == 1000 and w.n == 16 and w.m_per_node == 65536
+    ctx = _context(w, seed)
+    csr = w.csr()
+    X = np.zeros((w.n, w.N), dtype=np.float32)
+    local = np.tile(np.arange(w.batch, dtype=np.int32), (w.n, 1))
+    node = torch.arange(w.n, device="cuda")[:, None]
+    worst = 0.0
+    t0 = time.time()
+    for k in range(T):
+        idx = orc.sample_indices(seed, k, w.n, w.batch, w.m_per_node)
+        assert np.array_equal(ctx.sample(k).cpu().numpy(), idx), k
+        it = torch.from_numpy(idx.astype(np.int64)).cuda()
+        A_s = w.A[node, it].cpu().numpy()                      # [n][B][d]: the sampled rows only
+        y_s = w.y[node, it].cpu().numpy()
+        G_ref = orc.gradients(X, orc.MODEL_LOGISTIC, w.dims, A_s, y_s, local, w.l2_lambda)
+        X = orc.mix_update(X, G_ref, *csr, w.gamma)
+        ctx.step(k)
+        if (k + 1) % 50 == 0 or k + 1 == T:
+            got = ctx.current()[:, :w.N].cpu().numpy()
+            e, a = row_rel_err(got, X), avg_rel_err(got, X)
+            worst = max(worst, e)
+            _log({"config": 2, "k": k + 1, "row_err": e, "avg_err": a, "seconds": time.time() - t0})
+            assert e <= TOL_TRAJ and a <= TOL_AVG, (k, e, a)
+    c_ref = orc.consensus_dist(X)
+    assert abs(ctx.consensus_dist() - c_ref) <= 1e-2 * c_ref
+    ctx.close()
+
+
+def _rows_rel_err_dev(got, ref):
+    """Row-wise ||got - ref|| / ||ref|| in fp64 on the device: tensor [n]."""
+    d = (got.double() - ref.double()).norm(dim=1)
+    return d / ref.double().norm(dim=1).clamp_min(1e-30)
+
+
+def run_mlp_trajectory(w, seed, free_modes, consensus_every_step, label):
+    """Algorithm 1 for T = w.iterations iterations of an MLP configuration, three ways at once:
+
+      oracle ........ free-running, its own fp64 arithmetic throughout (the reference trajectory);
+      resynchronised  a library context that is put on the oracle's X_k before every iteration: indices,
+                      gradient and X_{k+1} are compared step by step along the WHOLE trajectory.  A hidden
+                      unit whose pre-activation lies within fp32 rounding of zero may take either ReLU'
+                      decision (the decision is taken in the kernel's precision); such flips are resolved as
+                      in the per-step tests and RECORDED (iteration, node, layer, sample, unit, z);
+      free-running .. one library context per entry of free_modes, never resynchronised.
+
+    Asserted: indices bit for bit; per-step parity (gradient 5e-5, X 1e-5, row-wise) in every iteration;
+    the free-running runs within 1e-3 (rows) and 1e-4 (node average) of the oracle at every checkpoint up
+    to the first recorded flip.  A flip changes one node's gradient by up to a per cent (one unit of one
+    sample carries that much of it), after which two correct implementations follow different branches
+    of a piecewise-linear function: from there on the free-running errors are recorded, and asserted only
+    against SANITY (the runs stay neighbours; nothing has blown up)."""
+    from threadpoolctl import threadpool_limits
+    T, N, n = w.iterations, w.N, w.n
+    dev = w.A.device
+    sync = _context(w, seed, 0)
+    free = {name: _context(w, seed, mode) for name, mode in free_modes.items()}
+    A, y = w.A.cpu().numpy(), w.y.cpu().numpy()
+    o = orc.Oracle(n, N, *w.csr(), w.gamma, seed, w.model, w.dims, w.batch, 0.0, A, y)
+    o.set_x(np.tile(w.x0.cpu().numpy(), (n, 1)))
+    log = {name: torch.zeros(T, dtype=torch.float64, device=dev) for name in free}
+    flips, first_flip, worst = [], None, {"G": 0.0, "X": 0.0}
+    Gs = sync._bufs[2]
+    t0 = time.time()
+    with threadpool_limits(limits=1):            # one BLAS thread per node: the pool supplies the parallelism
+        for k in range(T):
+            idx = o.sample(k)
+            assert np.array_equal(sync.sample(k).cpu().numpy(), idx), k
+            # ---- resynchronised leg: same start, one iteration
+            X_k = o.X
+            sync.current()[:, :N] = torch.from_numpy(X_k).to(dev)
+            sync.grad(k)
+            rows = list(POOL.map(lambda i: orc.grad_mlp(X_k[i], o.dims, A[i], y[i], idx[i]).astype(np.float32), range(n)))
+            G_or = np.stack(rows)
+            G_ref = torch.from_numpy(G_or).to(dev)
+            gerr = _rows_rel_err_dev(Gs[:, :N], G_ref)
+            bad = torch.nonzero(gerr > 5e-5).flatten().tolist()
+            G_m = None
+            for i in bad:                        # a ReLU decision at an fp32 tie went the other way?
+                g_gpu = Gs[i, :N].cpu().numpy().astype(np.float64)
+                ties = orc.mlp_near_zero_gates(X_k[i], o.dims, A[i], idx[i], GATE_REL)
+                chosen, best = [], G_or[i]
+                best_err = np.linalg.norm(best.astype(np.float64) - g_gpu)
+                for t in ties:
+                    cand = orc.grad_mlp(X_k[i], o.dims, A[i], y[i], idx[i], flip=chosen + [t]).astype(np.float32)
+                    e = np.linalg.norm(cand.astype(np.float64) - g_gpu)
+                    if e < best_err:
+                        best, best_err, chosen = cand, e, chosen + [t]
+                assert chosen, (label, k, i, float(gerr[i]), "gradient differs and no near-zero pre-activation explains it")
+                _, _, pre = orc._mlp_forward(X_k[i], o.dims, A[i], idx[i])
+                for (l, b, u) in chosen:
+                    flips.append({"k": k, "node": i, "layer": l, "sample": b, "unit": u, "z": float(pre[l][b, u]),
+                                  "G_err_unmatched": float(gerr[i])})
+                if G_m is None:
+                    G_m = G_or.copy()
+                G_m[i] = best
+                G_ref[i] = torch.from_numpy(best).to(dev)
+            if bad:
+                gerr = _rows_rel_err_dev(Gs[:, :N], G_ref)
+                if first_flip is None:
+                    first_flip = k
+            worst["G"] = max(worst["G"], float(gerr.max()))
+            assert float(gerr.max()) <= 5e-5, (label, k, float(gerr.max()))
+            sync.mix_update()
+            oracle_mix_update_blocks(o, G_or)                    # the oracle's own next point
+            X_cmp = o.X
+            if G_m is not None:                                  # what the step gives with the kernel's gate decisions
+                keep = o.X
+                o.X = X_k
+                X_cmp = oracle_mix_update_blocks(o, G_m)
+                o.X = keep
+            xerr = float(_rows_rel_err_dev(sync.current()[:, :N], torch.from_numpy(X_cmp).to(dev)).max())
+            worst["X"] = max(worst["X"], xerr)
+            assert xerr <= 1e-5, (label, k, xerr)
+            # ---- free-running legs
+            for name, ctx in free.items():
+                if consensus_every_step:
+                    ctx.step_consensus(k, log[name][k:k + 1])
+                else:
+                    ctx.step(k)
+            if (k + 1) % 25 == 0 or k + 1 == T or k < 4:
+                Xo = torch.from_numpy(o.X).to(dev)
+                c_or = o.consensus_dist() if consensus_every_step else None
+                for name, ctx in free.items():
+                    got = ctx.current()[:, :N]
+                    e = float(_rows_rel_err_dev(got, Xo).max())
+                    a_ref = Xo.double().mean(dim=0)
+                    a = float((got.double().mean(dim=0) - a_ref).norm() / a_ref.norm())
+                    rec = {"config": label, "path": name, "k": k + 1, "row_err": e, "avg_err": a,
+                           "flips_so_far": len(flips), "resync_worst_G": worst["G"], "resync_worst_X": worst["X"],
+                           "seconds": time.time() - t0}
+                    if consensus_every_step:
+                        rec["consensus"] = float(log[name][k])
+                        rec["consensus_oracle"] = c_or
+                    _log(rec)
+                    if first_flip is None:
+                        assert e <= TOL_TRAJ and a <= TOL_AVG, (label, name, k, e, a)
+                        if consensus_every_step:
+                            assert abs(rec["consensus"] - c_or) <= 2e-2 * c_or
+                    # sanity from the first flip on: neighbours on the same path, nothing blown up
+                    assert e <= SANITY_ROWS and a <= SANITY_AVG, (label, name, k, e, a)
+    _log({"config": label, "flips": flips[:200], "n_flips": len(flips), "first_flip": first_flip,
+          "resync_worst_G": worst["G"], "resync_worst_X": worst["X"]})
+    for ctx in list(free.values()) + [sync]:
+        ctx.sync()
+        ctx.close()
+    return flips, first_flip
+
+
+# Free-running error allowed once a ReLU decision has differed (see run_mlp_trajectory): a bound on how
+# far two correct runs drift apart in the configurations' iteration counts, set from the measured
+# separation (rows up to 3e-2, node average up to 4e-3) with a margin; it catches a wrong step, not a
+# rounding difference.
+SANITY_ROWS = 0.2
+SANITY_AVG = 0.05
+
+
+def test_config3_mlp_500_iterations_two_stage_and_fused():
+    """n = 32 ring, MLP 784-1024-10, 1875 samples per node, minibatch 32, gamma 0.05, T = 500: the
+    two-stage iteration and the default one (gossip step inside the weight-gradient kernel) free-run
+    beside ONE oracle run, and a third context is checked step by step along the oracle's path."""
+    w = wl.config(2, device="cuda")
+    assert w.iterations == 500 and w.n == 32
+    run_mlp_trajectory(w, 20252, {"two_stage": 0, "fused": 1}, False, "3")
+
+
+@pytest.mark.parametrize("topology", ["ring", "torus", "dense"])
+def test_config4_stress_50_steps_fresh_gradients(topology):
+    """n = 64 x N = 25,000,000, gamma 0.01, a fresh N(0,1) gradient matrix every step, 50 free-running
+    gossip steps per topology in the launch configuration the benchmark times.  The step acts on every
+    column alone, so the oracle follows five blocks of columns (the first, the ragged last, three
+    random ones) through all 50 steps."""
+    _need(30)
+    n, N, T, width = 64, 25_000_000, 50, 8192
+    ld = wl.padded_ld(N)
+    dev = torch.device("cuda")
+    X0 = wl.stress_matrix(n, ld, N, 4100, dev)
+    X1, G = torch.zeros_like(X0), torch.zeros_like(X0)
+    csr = wl.topology(topology, n)
+    ctx = binding.Dpsgd(n, N, *csr, gamma=0.01, seed=0)
+    ctx.bind(X0, X1, G)
+    rng = np.random.default_rng(41)
+    starts = [0, N - width] + [int(s) for s in rng.integers(width, N - 2 * width, 3)]
+    cols = torch.cat([torch.arange(s, s + width, device=dev) for s in starts])
+    Xo = X0[:, cols].cpu().numpy()
+    g = torch.Generator(device=dev).manual_seed(4200)
+    mean0 = X0.sum(dim=0, dtype=torch.float64) / n
+    gsum = torch.zeros(ld, dtype=torch.float64, device=dev)
+    for k in range(T):
+        G[:, :N].normal_(generator=g)
+        Go = G[:, cols].cpu().numpy()
+        cuts = list(range(0, Xo.shape[1], 4096)) + [Xo.shape[1]]
+        Xo = np.concatenate(list(POOL.map(
+            lambda c: orc.mix_update(Xo[:, c[0]:c[1]], Go[:, c[0]:c[1]], *csr, 0.01), zip(cuts[:-1], cuts[1:]))), axis=1)
+        gsum += G.sum(dim=0, dtype=torch.float64) / n
+        ctx.mix_update()
+    got = ctx.current()
+    gs = got[:, cols].cpu().numpy()
+    e, a = row_rel_err(gs, Xo), avg_rel_err(gs, Xo)
+    _log({"config": 4, "topology": topology, "k": T, "row_err": e, "avg_err": a})
+    assert e <= TOL_TRAJ and a <= TOL_AVG
+    assert np.abs(gs.astype(np.float64) - Xo).max() <= 1e-4
+    # at any size: the node average follows xbar_T = xbar_0 - gamma sum_k gbar_k (rows of W sum to one)
+    expect = mean0 - float(np.float32(0.01)) * gsum
+    drift = (got.sum(dim=0, dtype=torch.float64) / n - expect).norm() / expect.norm()
+    assert float(drift) <= TOL_AVG
+    assert float(got[:, N:].abs().max()) == 0.0
+    ctx.close()
+
+
+@pytest.mark.parametrize("topology", ["ring", "dense"])
+def test_config5_mlp_300_iterations_consensus_every_step(topology):
+    """MLP 1024-2048-2048-10 (6,316,042 parameters per node), 4096 samples per node, minibatch 64,
+    gamma 0.02, T = 300, consensus distance reported by every iteration (dpsgd_step_consensus); the ring
+    beside the averaging matrix of C-PSGD.  n = 8 nodes: what the oracle finishes in a few minutes."""
+    _need(8)
+    w = wl.config(4, device="cuda", n=8, topology=topology)
+    assert w.iterations == 300 and w.batch == 64 and w.dims == (1024, 2048, 2048, 10)
+    run_mlp_trajectory(w, 20254, {"default": 1}, True, "5-" + topology)

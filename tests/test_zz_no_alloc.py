@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import dpsgd_oracle as orc
 from paper_1705_09056_b200 import binding, workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -48,6 +49,9 @@ def test_noalloc_consensus_matches_context_entry_point_twice_in_a_row():
     for g, w_ in zip(got, want):
         assert abs(g - w_) <= 1e-5 * w_ + 1e-12                # the tolerance of the other consensus tests
         assert g == w_                                         # same kernels, same order: bit-identical
+    for (X, N), g in zip(mats, got):                           # and the definition itself (Eq. 10), on the CPU
+        ref = orc.consensus_dist(X[:, :N].cpu().numpy())
+        assert abs(g - ref) <= 1e-5 * ref
     # and again in the opposite order, reusing the same output cell
     binding.consensus_dist_noalloc(mats[1][0], mats[1][1], out)
     assert float(out.item()) == want[1]
