@@ -260,6 +260,24 @@ DPSGD_API dpsgd_status dpsgd_sync(dpsgd_ctx* ctx);
  */
 DPSGD_API dpsgd_status dpsgd_selftest_wait(dpsgd_ctx* ctx, uint32_t max_polls);
 
+/*
+ * A layer of the paper's image workloads (Section 5.1: ResNet-20 on CIFAR-10; Section 5.3: a 32-layer
+ * residual network): 3x3 convolution, zero padding 1, stride 1 or 2, for all nodes at once, each node with
+ * the filters of its OWN current parameter row x_{k,i} (forward half of Algorithm 1 step 3 for such a model):
+ *   out[i][b][o][p][q] = act( bias_i[o] + sum_{c,kh,kw} w_i[o][c][kh][kw] * in[i][b][c][stride p + kh - 1][stride q + kw - 1] )
+ * with the input read as zero outside the image, act = ReLU when relu != 0, else the identity.
+ *   in_dev   device, fp32 [n][batch][c_in][h][w] (NCHW per node), 16-byte aligned, caller-owned
+ *   out_dev  device, fp32 [n][batch][c_out][h'][w'], h' = (h - 1) / stride + 1, w' likewise, 16-byte aligned
+ *   w_off    column of the first filter weight inside a parameter row; the c_out x c_in x 3 x 3 block is
+ *            row-major in (o, c, kh, kw); b_off: column of the c_out biases.  Both blocks inside [0, N).
+ * Products are fp32-faithful on the tensor cores (three TF32 MMAs on split operands).  Asynchronous on the
+ * bound stream.  Shapes taken: w and w' powers of two, 4 <= w <= 256, w' <= 128, h' * w' a multiple or a
+ * divisor of 128, c_out a multiple of 16, c_in <= 256; otherwise DPSGD_ERR_UNSUPPORTED.
+ */
+DPSGD_API dpsgd_status dpsgd_conv3x3_forward(dpsgd_ctx* ctx, const float* in_dev, int32_t batch, int32_t c_in, int32_t h,
+                                             int32_t w, int32_t c_out, int32_t stride, int64_t w_off, int64_t b_off,
+                                             int32_t relu, float* out_dev);
+
 /* Output of Algorithm 1: xbar = (1/n) sum_i x_i into xbar_dev (fp32 [ld], 16-byte aligned). */
 DPSGD_API dpsgd_status dpsgd_average(dpsgd_ctx* ctx, float* xbar_dev);
 

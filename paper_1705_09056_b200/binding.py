@@ -50,6 +50,7 @@ SIGNATURES = {
     "dpsgd_sync": [_vp],
     "dpsgd_selftest_wait": [_vp, ctypes.c_uint32],
     "dpsgd_average": [_vp, _vp],
+    "dpsgd_conv3x3_forward": [_vp, _vp, _i32, _i32, _i32, _i32, _i32, _i32, _i64, _i64, _i32, _vp],
     "dpsgd_mix_update_host": [_vp, _vp, _i64, ctypes.POINTER(ctypes.c_double)],
     "dpsgd_consensus_dist_noalloc": [_vp, _i32, _i64, _i64, _vp, _vp],
     "dpsgd_current": [_vp, ctypes.POINTER(_vp)],
@@ -254,6 +255,20 @@ class Dpsgd:
     def selftest_wait(self, max_polls: int = 4096):
         """Enqueues the self-test CTA whose wait runs out (see dpsgd_selftest_wait)."""
         self._check(self._lib.dpsgd_selftest_wait(self._h, max_polls))
+
+    def conv3x3_forward(self, x: torch.Tensor, c_out: int, stride: int, w_off: int, b_off: int, relu: bool = True,
+                        out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """3x3 convolution (padding 1) of x [n][B][C][H][W] with every node's own filters, read from the
+        current X at columns w_off (filters) and b_off (biases)."""
+        assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous() and x.dim() == 5 and x.shape[0] == self.n
+        _, B, C, H, W = x.shape
+        ho, wo = (H - 1) // stride + 1, (W - 1) // stride + 1
+        if out is None:
+            out = torch.empty((self.n, B, c_out, ho, wo), dtype=torch.float32, device=x.device)
+        assert out.is_cuda and out.is_contiguous() and tuple(out.shape) == (self.n, B, c_out, ho, wo)
+        self._check(self._lib.dpsgd_conv3x3_forward(self._h, _ptr(x), B, C, H, W, c_out, stride, w_off, b_off,
+                                                    1 if relu else 0, _ptr(out)))
+        return out
 
     def average(self, xbar: Optional[torch.Tensor] = None) -> torch.Tensor:
         if xbar is None:

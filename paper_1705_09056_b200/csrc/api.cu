@@ -404,9 +404,15 @@ dpsgd_status mix_with_consensus(dpsgd_ctx* c, double* out_dev) {
     const float* X = c->X[c->cur];
     float* Xn = c->X[c->cur ^ 1];
     const bool fused = c->mix_kind == DPSGD_MIX_RING || c->mix_kind == DPSGD_MIX_UNIFORM_DENSE;
+    const bool small = !c->kind_forced && mix_is_small(c);
     cudaError_t e;
     if (fused) {
         e = launch_mix_variant(c, X, c->G, Xn, c->swapped, out_dev, c->V);   // V, when set, updated in the pass
+    } else if (c->mix_kind == DPSGD_MIX_TILED_CSR && !small) {
+        // any sparse W on the tile-staging kernel: the statistics come from the rows it has in registers
+        const float* D = nullptr;
+        e = step_direction(c, &D);
+        if (e == cudaSuccess) e = launch_mix_tiled(c, X, D, Xn, out_dev);
     } else {                                // no fused kernel for this W: mix, then one pass over the new X
         e = run_mix(c);
         if (e == cudaSuccess) e = launch_consensus(c, Xn, out_dev);
@@ -618,7 +624,7 @@ DPSGD_API dpsgd_status dpsgd_step(dpsgd_ctx* c, uint64_t k) {
 // memory and advance it, so that one graph can be replayed for any k.
 dpsgd_status capture_pair(dpsgd_ctx* c) {
     cudaError_t e = cudaSuccess;
-    if (!c->d_k) e = cudaMalloc(&c->d_k, sizeof(uint64_t));
+    if (!c->d_k) e = cudaMalloc(&c->d_k, 2 * sizeof(uint64_t));
     if (e != cudaSuccess) return cuda_fail(c, e, "iteration counter");
     // record on a private stream (the bound one may be the legacy default stream, which cannot
     // capture); the instantiated graph is launched on the bound stream
@@ -630,13 +636,19 @@ dpsgd_status capture_pair(dpsgd_ctx* c) {
     e = cudaStreamBeginCapture(c->capture_stream, cudaStreamCaptureModeThreadLocal);
     if (e != cudaSuccess) return cuda_fail(c, e, "begin capture");
     c->stream = c->capture_stream;
-    c->k_dev_active = c->d_k;
+    // The one-launch step kernel reads the iteration number from one slot and leaves the next number in the
+    // other, so the two captured iterations alternate slots (the replay starts from slot 0) and need no
+    // counter kernel; every other path reads slot 0 and a one-thread kernel advances it.
+    const bool self = c->fuse_step && linear_node_step_fuses(c);
     dpsgd_status s = DPSGD_OK;
     for (int t = 0; t < 2 && s == DPSGD_OK; ++t) {
+        c->k_dev_active = c->d_k + (self ? t : 0);
+        c->k_dev_next = self ? c->d_k + (t ^ 1) : nullptr;
         s = dpsgd_step(c, 0);
-        if (s == DPSGD_OK && launch_advance_k(c) != cudaSuccess) s = DPSGD_ERR_CUDA;
+        if (!self && s == DPSGD_OK && launch_advance_k(c) != cudaSuccess) s = DPSGD_ERR_CUDA;
     }
     c->k_dev_active = nullptr;
+    c->k_dev_next = nullptr;
     c->stream = bound_stream;
     cudaGraph_t graph = nullptr;
     e = cudaStreamEndCapture(c->capture_stream, &graph);
@@ -716,6 +728,23 @@ DPSGD_API dpsgd_status dpsgd_selftest_wait(dpsgd_ctx* c, uint32_t max_polls) {
     if (max_polls < 1 || max_polls > (1u << 20)) return fail(c, DPSGD_ERR_ARG, "max_polls must be in [1, 2^20]");
     cudaError_t e = launch_wait_probe(c, max_polls);
     return e == cudaSuccess ? DPSGD_OK : cuda_fail(c, e, "wait probe kernel");
+}
+
+DPSGD_API dpsgd_status dpsgd_conv3x3_forward(dpsgd_ctx* c, const float* in_dev, int32_t batch, int32_t c_in, int32_t h,
+                                             int32_t w, int32_t c_out, int32_t stride, int64_t w_off, int64_t b_off,
+                                             int32_t relu, float* out_dev) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    if (!in_dev || !out_dev) return fail(c, DPSGD_ERR_ARG, "in_dev or out_dev is NULL");
+    if (!aligned(in_dev, 16) || !aligned(out_dev, 16)) return fail(c, DPSGD_ERR_ALIGN, "in_dev and out_dev must be 16-byte aligned");
+    if (const char* why = conv3x3_forward_unsupported(batch, c_in, h, w, c_out, stride)) return fail(c, DPSGD_ERR_UNSUPPORTED, why);
+    const int64_t wsz = (int64_t)c_out * c_in * 9;
+    if (w_off < 0 || b_off < 0 || w_off + wsz > c->N || b_off + c_out > c->N)
+        return fail(c, DPSGD_ERR_ARG, "filter or bias block lies outside the parameter row");
+    const char* why = nullptr;
+    cudaError_t e = launch_conv3x3_forward(c, in_dev, batch, c_in, h, w, c_out, stride, w_off, b_off, relu, out_dev, &why);
+    if (e == cudaErrorNotSupported && why) return fail(c, DPSGD_ERR_UNSUPPORTED, why);
+    return e == cudaSuccess ? DPSGD_OK : cuda_fail(c, e, "convolution kernel");
 }
 
 DPSGD_API dpsgd_status dpsgd_average(dpsgd_ctx* c, float* xbar) {

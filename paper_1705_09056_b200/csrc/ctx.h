@@ -100,8 +100,9 @@ struct dpsgd_ctx {
     void* tma_state = nullptr;     // tensor maps for the tiled mixing kernel
 
     // graph replay of pairs of iterations (small, launch-bound problems)
-    uint64_t* d_k = nullptr;                 // device iteration counter
+    uint64_t* d_k = nullptr;                 // device iteration counter (two slots, see capture_pair)
     const uint64_t* k_dev_active = nullptr;  // non-NULL only while a graph is captured
+    uint64_t* k_dev_next = nullptr;          // capture of a self-advancing step kernel: where it leaves k + 1
     cudaGraphExec_t graph_exec = nullptr;
     cudaStream_t capture_stream = nullptr;   // private stream the pair is recorded on
     int graph_cur = 0;                       // value of `cur` the graph was captured at
@@ -132,7 +133,7 @@ cudaError_t launch_mix_uniform(dpsgd_ctx* c, const float* X, const float* G, flo
 cudaError_t launch_mix_gather(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
 cudaError_t launch_mix_rowpar(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
 bool mix_is_small(const dpsgd_ctx* c);
-cudaError_t launch_mix_tiled(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
+cudaError_t launch_mix_tiled(dpsgd_ctx* c, const float* X, const float* G, float* Xn, double* stats_out = nullptr);
 bool mix_tiled_supported(const dpsgd_ctx* c);
 // One CTA that waits, with the kernels' bounded wait cut to max_polls polls, on an mbarrier nothing arrives at.
 cudaError_t launch_wait_probe(dpsgd_ctx* c, uint32_t max_polls);
@@ -153,6 +154,7 @@ cudaError_t launch_set_k(dpsgd_ctx* c, uint64_t v);
 cudaError_t launch_advance_k(dpsgd_ctx* c);
 cudaError_t launch_grad_linear(dpsgd_ctx* c, uint64_t k, const float* X, float* G);
 bool linear_step_fuses(const dpsgd_ctx* c);
+bool linear_node_step_fuses(const dpsgd_ctx* c);   // the one-launch variant (its kernel advances the replay counter itself)
 cudaError_t launch_linear_step(dpsgd_ctx* c, uint64_t k, const float* X, float* G, float* Xn);
 // Xn != NULL: weight blocks whose product runs on the fused kernel are written to Xn after the gossip
 // step instead of to G, and listed in c->fused_blocks.
@@ -165,6 +167,11 @@ cudaError_t run_tcw_fused(dpsgd_ctx* c, const float* h, int din, const float* de
                           int64_t w_off, const float* X, float* Xn);
 // Gossip step on the columns of [0, ld) outside c->fused_blocks.
 cudaError_t launch_mix_rest(dpsgd_ctx* c, const float* X, const float* G, float* Xn);
+// 3x3 convolution forward with every node's own filters (conv_fwd.cu).  *why names what is unsupported
+// when the result is cudaErrorNotSupported.
+const char* conv3x3_forward_unsupported(int batch, int c_in, int h, int w, int c_out, int stride);
+cudaError_t launch_conv3x3_forward(dpsgd_ctx* c, const float* x, int batch, int c_in, int h, int w, int c_out, int stride,
+                                   int64_t w_off, int64_t b_off, int relu, float* y, const char** why);
 size_t mlp_act_floats(const dpsgd_ctx* c);
 size_t mlp_delta_floats(const dpsgd_ctx* c);
 

@@ -321,6 +321,141 @@ glm_rows_reduce_mix_kernel(const float4* __restrict__ X, float4* __restrict__ G,
     Xn[(int64_t)node * ld4 + c] = a;
 }
 
+// ---- one launch per iteration for small linear models ----
+//
+// One CTA per node does the node's whole iteration of Algorithm 1: draws the B indices (step 2), stages the
+// sampled rows and the node's own x in shared memory, forms the B dot products and coefficients and the
+// gradient row (step 3), writes it to G, and applies the gossip step X_next[i] = sum_j W_ij X[j] - gamma g_i
+// (steps 4-5).  The update is out of place (neighbours are read from X_k, results go to X_{k+1}), so no CTA
+// waits for another.  Every reduction runs in the order of glm_forward_kernel / glm_backward_kernel /
+// mix_rowpar_kernel (lanes of a 32-wide xor tree, warps in order, eight interleaved slices of the minibatch
+// in order), so the result is bit-identical to the three-launch path.
+// With k_next != NULL the kernel reads the iteration number from *k_ptr and leaves k + 1 in *k_next (two
+// slots used alternately by consecutive launches: a replayed graph needs no counter kernel in between).
+constexpr int kNodeThreads = 256;
+
+__global__ void __launch_bounds__(kNodeThreads)
+glm_node_step_kernel(const float4* __restrict__ X, float4* __restrict__ G, float4* __restrict__ Xn, int64_t ld,
+                     const float* __restrict__ A, const float* __restrict__ y, int64_t m, int d, int B, uint64_t seed,
+                     uint64_t k, const uint64_t* __restrict__ k_ptr, uint64_t* __restrict__ k_next, int model, float l2,
+                     int32_t* __restrict__ idx, float* __restrict__ coef_out, const int32_t* __restrict__ node_batch,
+                     const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col,
+                     const float* __restrict__ val, float ngamma) {
+    extern __shared__ __align__(16) unsigned char node_smem[];
+    const int node = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int d4 = d / 4;
+    const int64_t ld4 = ld / 4;
+    float4* rows = reinterpret_cast<float4*>(node_smem);                   // [B][d4]
+    float4* xs = rows + (size_t)B * d4;                                    // [ld4] the node's own row
+    float4* gs = xs + ld4;                                                 // [ld4] its gradient row
+    float4* red = gs + ld4;                                                // [8][32]
+    float* scoef = reinterpret_cast<float*>(red + 8 * 32);                 // [B]
+    int32_t* sj = reinterpret_cast<int32_t*>(scoef + B);                   // [B]
+    if (k_ptr) k = *k_ptr;
+    if (k_next && node == 0 && tid == 0) *k_next = k + 1;
+    const int Bi = node_batch ? __ldg(node_batch + node) : B;
+    for (int b = tid; b < B; b += kNodeThreads) {
+        const int32_t j = sample_index(seed, k, (uint32_t)node, (uint32_t)b, (uint32_t)m);
+        sj[b] = j;
+        idx[node * B + b] = j;
+    }
+    for (int64_t c = tid; c < ld4; c += kNodeThreads) xs[c] = __ldg(X + (int64_t)node * ld4 + c);
+    __syncthreads();
+    for (int e = tid; e < B * d4; e += kNodeThreads) {
+        const int b = e / d4, c = e - b * d4;
+        rows[e] = b < Bi ? __ldg(reinterpret_cast<const float4*>(A + ((int64_t)node * m + sj[b]) * d) + c)
+                         : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    __syncthreads();
+    // forward: a warp per draw; lane l of pass w stands for thread 32 w + l of the per-sample CTA
+    for (int b = warp; b < B; b += kNodeThreads / 32) {
+        float cf = 0.f;
+        if (b < Bi) {
+            float dot = 0.f;
+#pragma unroll 1
+            for (int w = 0; w < 8; ++w) {
+                const int c = w * 32 + lane;
+                float acc = 0.f;
+                if (c < d4) {
+                    const float4 a = rows[b * d4 + c], v = xs[c];
+                    acc = fmaf(a.x, v.x, acc); acc = fmaf(a.y, v.y, acc);
+                    acc = fmaf(a.z, v.z, acc); acc = fmaf(a.w, v.w, acc);
+                }
+                dot += warp_allsum(acc);
+            }
+            const float yv = __ldg(y + (int64_t)node * m + sj[b]);
+            if (model == DPSGD_MODEL_LSQ) {
+                cf = (dot - yv) / (float)Bi;
+            } else {
+                const float z = dot + reinterpret_cast<const float*>(xs)[d];
+                const float s = 1.f / (1.f + expf(yv * z));
+                cf = -yv * s / (float)Bi;
+            }
+        }
+        if (lane == 0) { scoef[b] = cf; coef_out[node * B + b] = cf; }
+    }
+    __syncthreads();
+    // backward: 32 column groups x 8 interleaved slices of the minibatch, slices added in order
+    const int tx = lane, ty = warp;
+    for (int c0 = 0; c0 < d4; c0 += 32) {
+        const int cg = c0 + tx;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (cg < d4) {
+            for (int b = ty; b < Bi; b += 8) {
+                const float w = scoef[b];
+                const float4 a = rows[b * d4 + cg];
+                acc.x = fmaf(w, a.x, acc.x); acc.y = fmaf(w, a.y, acc.y);
+                acc.z = fmaf(w, a.z, acc.z); acc.w = fmaf(w, a.w, acc.w);
+            }
+        }
+        red[ty * 32 + tx] = acc;
+        __syncthreads();
+        if (ty == 0 && cg < d4) {
+            float4 s = red[tx];
+#pragma unroll
+            for (int t = 1; t < 8; ++t) {
+                const float4 r = red[t * 32 + tx];
+                s.x += r.x; s.y += r.y; s.z += r.z; s.w += r.w;
+            }
+            if (model == DPSGD_MODEL_LOGISTIC) {
+                const float4 x = xs[cg];
+                s.x = fmaf(l2, x.x, s.x); s.y = fmaf(l2, x.y, s.y); s.z = fmaf(l2, x.z, s.z); s.w = fmaf(l2, x.w, s.w);
+            }
+            gs[cg] = s;
+        }
+        __syncthreads();
+    }
+    if (ty == 1) {          // bias gradient (logistic) and zero padding: columns [d, ld)
+        for (int64_t c = d + tx; c < ld; c += 32) {
+            float s = 0.f;
+            if (model == DPSGD_MODEL_LOGISTIC && c == d)
+                for (int b = 0; b < Bi; ++b) s += scoef[b];
+            reinterpret_cast<float*>(gs)[c] = s;
+        }
+    }
+    __syncthreads();
+    // gradient row out, then the gossip step on this node's row
+    const int p0 = __ldg(row_ptr + node), pe = __ldg(row_ptr + node + 1);
+    for (int64_t c = tid; c < ld4; c += kNodeThreads) {
+        const float4 g = gs[c];
+        G[(int64_t)node * ld4 + c] = g;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int p = p0; p < pe; ++p) {
+            const float w = __ldg(val + p);
+            const float4 v = __ldg(X + (int64_t)__ldg(col + p) * ld4 + c);
+            a.x = fmaf(w, v.x, a.x); a.y = fmaf(w, v.y, a.y);
+            a.z = fmaf(w, v.z, a.z); a.w = fmaf(w, v.w, a.w);
+        }
+        a.x = fmaf(ngamma, g.x, a.x); a.y = fmaf(ngamma, g.y, a.y);
+        a.z = fmaf(ngamma, g.z, a.z); a.w = fmaf(ngamma, g.w, a.w);
+        Xn[(int64_t)node * ld4 + c] = a;
+    }
+}
+
+size_t node_step_smem(const dpsgd_ctx* c) {
+    return sizeof(float) * ((size_t)c->batch * c->d + 2 * (size_t)c->ld + 8 * 32 * 4 + 2 * (size_t)c->batch);
+}
+
 bool rows_path(const dpsgd_ctx* c) {
     return c->d % 4 == 0 && c->d >= 1024 && c->d <= 16 * kRowsThreads * kRowsMaxR / 4 && c->n <= 65535;
 }
@@ -347,14 +482,34 @@ cudaError_t launch_rows(dpsgd_ctx* c, uint64_t k, const float* X, int* groups_ou
 
 }  // namespace
 
-// Whole iteration of a linear model in two launches: shares of the gradient, then their reduction and the
-// gossip step together.  False when the shapes or the options call for the separate stages.
+// Narrow rows on a small matrix: the whole iteration in ONE launch (a CTA per node).
+bool linear_node_step_fuses(const dpsgd_ctx* c) {
+    return c->model != DPSGD_MODEL_MLP && !rows_path(c) && c->d % 4 == 0 && c->d < 1024 && c->batch <= 1024 &&
+           (int64_t)c->batch * c->d <= 8192 && c->ld <= 2048 && !c->kind_forced && mix_is_small(c) && !c->swapped &&
+           c->V == nullptr && c->n <= 65535;
+}
+
+// Whole iteration of a linear model in one launch (narrow rows) or two (wide rows: shares of the gradient,
+// then their reduction and the gossip step together).  False when the shapes or the options call for the
+// separate stages.
 bool linear_step_fuses(const dpsgd_ctx* c) {
+    if (linear_node_step_fuses(c)) return true;
     return c->model != DPSGD_MODEL_MLP && rows_path(c) && !c->kind_forced && mix_is_small(c) && !c->swapped &&
            c->V == nullptr;
 }
 
 cudaError_t launch_linear_step(dpsgd_ctx* c, uint64_t k, const float* X, float* G, float* Xn) {
+    if (linear_node_step_fuses(c)) {
+        const size_t smem = node_step_smem(c);
+        cudaError_t e = cudaFuncSetAttribute(glm_node_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        glm_node_step_kernel<<<c->n, kNodeThreads, smem, c->stream>>>(
+            reinterpret_cast<const float4*>(X), reinterpret_cast<float4*>(G), reinterpret_cast<float4*>(Xn), c->ld, c->A,
+            static_cast<const float*>(c->y), c->m, c->d, c->batch, c->seed, k, c->k_dev_active, c->k_dev_next, c->model,
+            c->l2, c->d_idx, c->d_coef, c->d_node_batch, c->W.row_ptr, c->W.col, c->W.val, -c->gamma);
+        c->launches++;
+        return cudaGetLastError();
+    }
     int groups = 0;
     cudaError_t e = launch_rows(c, k, X, &groups);
     if (e != cudaSuccess) return e;

@@ -47,6 +47,8 @@ struct TiledState {
     int csr_in_smem = 0;
     int x_tma = 1;
     int swapped = 0;
+    int stats = 0;        // this launch also accumulates the consensus statistics
+    int last_grid = 0;    // CTAs of the last launch (= partials written)
     int* d_status = nullptr;
     PackedNz* d_nz = nullptr;
 };
@@ -96,29 +98,41 @@ __device__ __forceinline__ void cp_async_arrive(uint64_t* bar) {
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// Shared memory: S x { X tile [n][T] | G tile [n][T] }, S mbarriers, then (when it fits) a copy of
-// row_ptr and of the packed nonzeros so that the gather loop never leaves the SM.
+// Shared memory: S x { X tile [n][T] | G tile [n][T] }, S mbarriers, two scratch buffers for the consensus
+// statistics, then (when it fits) a copy of row_ptr and of the packed nonzeros so that the gather loop
+// never leaves the SM.
 // X arrives by TMA (one box per tile) or, with X_TMA = false, by per-thread 16-byte async copies
 // like G always does; each stage's mbarrier counts the TMA transaction plus one arrival per thread.
-// SWAPPED (footnote c of Algorithm 1): the staged X tile is first turned into X - gamma G in place,
-// then gathered: X_next[i] = sum_j W_ij (X[j] - gamma G[j]).
-template <int T, int S, bool X_TMA, bool SWAPPED>
+// SWAPPED (footnote c of Algorithm 1): X_next[i] = sum_j W_ij (X[j] - gamma G[j]); every neighbour's term
+// is formed on the fly from the two staged tiles (no rewrite of the X tile, no extra barrier).
+// STATS (Theorem 4, Eq. 10): also accumulates sum_i ||xbar - x_i||^2 of the NEW rows while they are in
+// registers.  Per column the new values are shifted by the staged old X[0][c] (any common shift cancels),
+// d_i = x'_i - X[0][c]; the rows of a column sit in different threads, so per-thread sums of d and d^2 are
+// combined by shuffles inside a warp and through shared memory across warps (in a fixed order), the
+// column's sum d^2 - (sum d)^2 / n is formed in fp64, and every CTA leaves one fp64 partial.
+constexpr int kWarps = kThreads / 32;
+__host__ __device__ constexpr size_t stats_scratch_bytes(int T) { return (size_t)2 * 2 * kWarps * T * sizeof(float); }
+
+template <int T, int S, bool X_TMA, bool SWAPPED, bool STATS>
 __global__ void __launch_bounds__(kThreads)
 mix_tiled_kernel(const __grid_constant__ CUtensorMap mapX, const float4* __restrict__ X,
                  const float4* __restrict__ G, float4* __restrict__ Xn, const int32_t* row_ptr,
                  const PackedNz* nz, int n, int64_t ld4, int64_t tiles, float ngamma, int csr_in_smem,
-                 int* __restrict__ status) {
+                 int* __restrict__ status, double* __restrict__ partials) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     constexpr int kGroups = T / 4;                 // float4 column groups per tile
     constexpr int kRowStep = kThreads / kGroups;   // rows processed concurrently by the CTA
+    constexpr int kGW = kGroups < 32 ? kGroups : 32;   // column groups one warp covers
     const uint32_t tile_bytes = (uint32_t)n * T * sizeof(float);
     const uint32_t stage_bytes = 2 * tile_bytes;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + (size_t)S * stage_bytes);
+    // statistics scratch: [2 buffers][sum d | sum d^2][warp][column group of the warp] float4
+    float4* scratch = reinterpret_cast<float4*>(reinterpret_cast<unsigned char*>(full) + 16 * ((S * 8 + 15) / 16));
 
     const int tid = threadIdx.x;
     if (csr_in_smem) {
         const int nnz = __ldg(row_ptr + n);
-        PackedNz* s_nz = reinterpret_cast<PackedNz*>(full + S);
+        PackedNz* s_nz = reinterpret_cast<PackedNz*>(reinterpret_cast<unsigned char*>(scratch) + stats_scratch_bytes(T));
         int32_t* s_rp = reinterpret_cast<int32_t*>(s_nz + nnz);
         for (int t = tid; t <= n; t += kThreads) s_rp[t] = __ldg(row_ptr + t);
         for (int t = tid; t < nnz; t += kThreads) s_nz[t] = nz[t];
@@ -136,6 +150,7 @@ mix_tiled_kernel(const __grid_constant__ CUtensorMap mapX, const float4* __restr
     const int64_t my_tiles = first < tiles ? (tiles - first + step - 1) / step : 0;
     const int cg = tid % kGroups;
     const int r0 = tid / kGroups;
+    double col_acc = 0.0;                          // STATS: threads tid < T, one column of the tile each
 
     // every thread takes part: rows r0, r0 + kRowStep, ... of its own column group
     auto issue = [&](int64_t it, int s) {
@@ -168,30 +183,29 @@ mix_tiled_kernel(const __grid_constant__ CUtensorMap mapX, const float4* __restr
                 const int sj = (s + j) % S;
                 if (it + j < my_tiles) mbar_wait(full + sj, sj > s ? parity : parity ^ 1u);
             }
+            // the result is void (the status word says so); leave a defined partial and go, as threads that
+            // have exited do not hold up the CTA's barriers
+            if (STATS) partials[blockIdx.x] = 0.0;
             return;
         }
         unsigned char* xs = smem_raw + (size_t)s * stage_bytes + cg * 16;   // this thread's column group
         const unsigned char* gs = xs + tile_bytes;
         const int64_t c4 = (first + it * step) * kGroups + cg;
-        if (SWAPPED) {
-            for (int i = r0; i < n; i += kRowStep) {
-                float4* xp = reinterpret_cast<float4*>(xs + (uint32_t)i * (T * 4u));
-                const float4 g = *reinterpret_cast<const float4*>(gs + (uint32_t)i * (T * 4u));
-                float4 v = *xp;
-                v.x = fmaf(ngamma, g.x, v.x); v.y = fmaf(ngamma, g.y, v.y);
-                v.z = fmaf(ngamma, g.z, v.z); v.w = fmaf(ngamma, g.w, v.w);
-                *xp = v;
-            }
-            __syncthreads();
-        }
+        float4 s1 = make_float4(0.f, 0.f, 0.f, 0.f), s2 = make_float4(0.f, 0.f, 0.f, 0.f);
         if (c4 < ld4) {
             float4* out = Xn + c4;
+            const float4 sh = STATS ? *reinterpret_cast<const float4*>(xs) : make_float4(0.f, 0.f, 0.f, 0.f);
             for (int i = r0; i < n; i += kRowStep) {
                 float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
                 const int pe = row_ptr[i + 1];
                 for (int p = row_ptr[i]; p < pe; ++p) {
                     const PackedNz e = nz[p];
-                    const float4 v = *reinterpret_cast<const float4*>(xs + e.row_bytes);
+                    float4 v = *reinterpret_cast<const float4*>(xs + e.row_bytes);
+                    if (SWAPPED) {
+                        const float4 g = *reinterpret_cast<const float4*>(gs + e.row_bytes);
+                        v.x = fmaf(ngamma, g.x, v.x); v.y = fmaf(ngamma, g.y, v.y);
+                        v.z = fmaf(ngamma, g.z, v.z); v.w = fmaf(ngamma, g.w, v.w);
+                    }
                     a.x = fmaf(e.w, v.x, a.x); a.y = fmaf(e.w, v.y, a.y);
                     a.z = fmaf(e.w, v.z, a.z); a.w = fmaf(e.w, v.w, a.w);
                 }
@@ -201,14 +215,59 @@ mix_tiled_kernel(const __grid_constant__ CUtensorMap mapX, const float4* __restr
                     a.z = fmaf(ngamma, g.z, a.z); a.w = fmaf(ngamma, g.w, a.w);
                 }
                 __stcs(out + (int64_t)i * ld4, a);
+                if (STATS) {
+                    const float dx = a.x - sh.x, dy = a.y - sh.y, dz = a.z - sh.z, dw = a.w - sh.w;
+                    s1.x += dx; s1.y += dy; s1.z += dz; s1.w += dw;
+                    s2.x = fmaf(dx, dx, s2.x); s2.y = fmaf(dy, dy, s2.y);
+                    s2.z = fmaf(dz, dz, s2.z); s2.w = fmaf(dw, dw, s2.w);
+                }
             }
         }
-        // the swapped order rewrote the X tile with ordinary stores; order them before the bulk copy that
-        // refills the stage (generic-proxy writes against the async proxy)
-        if (SWAPPED) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncthreads();                       // everyone is done reading stage s
+        float4* sc = scratch + (size_t)(it & 1) * (2 * kWarps * kGW);
+        if (STATS) {
+            // lanes of a warp that share a column group (kGroups < 32: rows r0 differ), then one entry per warp
+#pragma unroll
+            for (int o = kGW; o < 32; o <<= 1) {
+                s1.x += __shfl_xor_sync(0xffffffffu, s1.x, o); s1.y += __shfl_xor_sync(0xffffffffu, s1.y, o);
+                s1.z += __shfl_xor_sync(0xffffffffu, s1.z, o); s1.w += __shfl_xor_sync(0xffffffffu, s1.w, o);
+                s2.x += __shfl_xor_sync(0xffffffffu, s2.x, o); s2.y += __shfl_xor_sync(0xffffffffu, s2.y, o);
+                s2.z += __shfl_xor_sync(0xffffffffu, s2.z, o); s2.w += __shfl_xor_sync(0xffffffffu, s2.w, o);
+            }
+            const int lane = tid & 31, warp = tid >> 5;
+            if (lane < kGW) {
+                sc[warp * kGW + lane] = s1;
+                sc[(kWarps + warp) * kGW + lane] = s2;
+            }
+        }
+        __syncthreads();                       // everyone is done reading stage s (and has left its statistics)
         if (it + S < my_tiles) issue(it + S, s);
+        if (STATS && tid < T) {
+            // column tid of the tile: its group is covered by the warps w with (w * 32 / kGroups ...) - for
+            // kGroups >= 32 a warp covers groups [32 (w % (kGroups / 32)), +32); otherwise every warp covers all
+            const int grp = tid >> 2, comp = tid & 3;
+            double a1 = 0.0, a2 = 0.0;
+            for (int w = 0; w < kWarps; ++w) {
+                if (kGroups > 32 && (w % (kGroups / 32)) != grp / 32) continue;
+                const float* e1 = reinterpret_cast<const float*>(sc + w * kGW + (grp % kGW));
+                const float* e2 = reinterpret_cast<const float*>(sc + (kWarps + w) * kGW + (grp % kGW));
+                a1 += (double)e1[comp];
+                a2 += (double)e2[comp];
+            }
+            col_acc += a2 - a1 * a1 / (double)n;
+        }
         if (++s == S) { s = 0; parity ^= 1u; }
+    }
+    if (STATS) {
+        // one fp64 partial per CTA, added in thread order
+        double* red = reinterpret_cast<double*>(scratch);
+        __syncthreads();
+        if (tid < T) red[tid] = col_acc;
+        __syncthreads();
+        if (tid == 0) {
+            double r = 0.0;
+            for (int t = 0; t < T; ++t) r += red[t];
+            partials[blockIdx.x] = r;
+        }
     }
 }
 
@@ -240,7 +299,7 @@ bool make_map(CUtensorMap* map, const float* base, int n, int64_t ld, int T) {
 }
 
 size_t smem_need(int n, int nnz, int T, int S, bool with_csr) {
-    size_t b = (size_t)S * 2 * n * T * sizeof(float) + S * sizeof(uint64_t);
+    size_t b = (size_t)S * 2 * n * T * sizeof(float) + 16 * ((S * sizeof(uint64_t) + 15) / 16) + stats_scratch_bytes(T);
     if (with_csr) b += sizeof(PackedNz) * (size_t)nnz + sizeof(int32_t) * (n + 1);
     return b;
 }
@@ -262,28 +321,31 @@ bool pick_shape(int n, int nnz, int* T_out, int* S_out, int* ctas_out) {
     return false;
 }
 
-template <int T, int S, bool X_TMA, bool SWAPPED>
+template <int T, int S, bool X_TMA, bool SWAPPED, bool STATS>
 cudaError_t launch_tsx(dpsgd_ctx* c, TiledState* st, int which, const float* G, float* Xn) {
     // per device and cheap: set on every launch rather than remembered in a process-wide flag
-    cudaError_t ea = cudaFuncSetAttribute(mix_tiled_kernel<T, S, X_TMA, SWAPPED>,
+    cudaError_t ea = cudaFuncSetAttribute(mix_tiled_kernel<T, S, X_TMA, SWAPPED, STATS>,
                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)(kSmemPerSm - kSmemPerCtaReserve));
     if (ea != cudaSuccess) return ea;
     const int64_t ld4 = c->ld / 4;
     const int64_t tiles = (c->ld + T - 1) / T;
     const int grid = (int)std::min<int64_t>(tiles, st->grid);
-    mix_tiled_kernel<T, S, X_TMA, SWAPPED><<<grid, kThreads, st->smem, c->stream>>>(
+    mix_tiled_kernel<T, S, X_TMA, SWAPPED, STATS><<<grid, kThreads, st->smem, c->stream>>>(
         st->mapX[which], reinterpret_cast<const float4*>(c->X[which]), reinterpret_cast<const float4*>(G),
         reinterpret_cast<float4*>(Xn), c->W.row_ptr, st->d_nz, c->n, ld4, tiles, -c->gamma, st->csr_in_smem,
-        st->d_status);
+        st->d_status, c->d_partials);
+    st->last_grid = grid;
     return cudaGetLastError();
 }
 
 template <int T, int S>
 cudaError_t launch_ts(dpsgd_ctx* c, TiledState* st, int which, const float* G, float* Xn) {
-    if (st->swapped)
-        return st->x_tma ? launch_tsx<T, S, true, true>(c, st, which, G, Xn) : launch_tsx<T, S, false, true>(c, st, which, G, Xn);
-    return st->x_tma ? launch_tsx<T, S, true, false>(c, st, which, G, Xn) : launch_tsx<T, S, false, false>(c, st, which, G, Xn);
+#define DPSGD_TILED_PICK(XT, SW) \
+    (st->stats ? launch_tsx<T, S, XT, SW, true>(c, st, which, G, Xn) : launch_tsx<T, S, XT, SW, false>(c, st, which, G, Xn))
+    if (st->swapped) return st->x_tma ? DPSGD_TILED_PICK(true, true) : DPSGD_TILED_PICK(false, true);
+    return st->x_tma ? DPSGD_TILED_PICK(true, false) : DPSGD_TILED_PICK(false, false);
+#undef DPSGD_TILED_PICK
 }
 
 template <int T>
@@ -315,7 +377,9 @@ cudaError_t launch_wait_probe(dpsgd_ctx* c, uint32_t max_polls) {
     return cudaGetLastError();
 }
 
-cudaError_t launch_mix_tiled(dpsgd_ctx* c, const float* X, const float* G, float* Xn) {
+// stats_out != NULL: the kernel also accumulates the consensus distance of X_next, and a fixed-order
+// reduction of the per-CTA partials leaves it in *stats_out (device).
+cudaError_t launch_mix_tiled(dpsgd_ctx* c, const float* X, const float* G, float* Xn, double* stats_out) {
     TiledState* st = static_cast<TiledState*>(c->tma_state);
     if (!st) {
         st = new TiledState();
@@ -351,13 +415,16 @@ cudaError_t launch_mix_tiled(dpsgd_ctx* c, const float* X, const float* G, float
     }
     const int which = (X == c->X[0]) ? 0 : 1;
     st->swapped = c->swapped ? 1 : 0;
+    st->stats = stats_out ? 1 : 0;
     cudaError_t e;
+    if (stats_out && (e = ensure_partials(c, st->grid)) != cudaSuccess) return e;
     switch (st->T) {
         case 128: e = launch_t<128>(c, st, which, G, Xn); break;
         case 64: e = launch_t<64>(c, st, which, G, Xn); break;
         default: e = launch_t<32>(c, st, which, G, Xn); break;
     }
     c->launches++;
+    if (e == cudaSuccess && stats_out) e = launch_consensus_final(c, st->last_grid, stats_out);
     return e;
 }
 

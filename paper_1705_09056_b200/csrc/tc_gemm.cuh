@@ -98,6 +98,14 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// TF32 head of v: the 10-bit-mantissa value NEAREST to v (ties away from zero; truncation would leave a
+// remainder twice as large).  The remainder v - head is exact in fp32 and at most half a TF32 ulp, so the
+// tensor core's own truncation of it costs at most 2^-22 |v|.  Finite values within 2^-12 of the largest
+// float round to infinity.
+__device__ __forceinline__ float tf32_head(float v) {
+    return __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xFFFFE000u);
+}
+
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
     uint32_t r[16];
     asm volatile(
@@ -188,10 +196,10 @@ struct OperandLoader {
     static __device__ __forceinline__ void put(unsigned char* hi, unsigned char* lo, uint32_t off, float4 v) {
         if (PRECISE) {
             float4 h, l;
-            h.x = __uint_as_float(__float_as_uint(v.x) & 0xFFFFE000u); l.x = v.x - h.x;
-            h.y = __uint_as_float(__float_as_uint(v.y) & 0xFFFFE000u); l.y = v.y - h.y;
-            h.z = __uint_as_float(__float_as_uint(v.z) & 0xFFFFE000u); l.z = v.z - h.z;
-            h.w = __uint_as_float(__float_as_uint(v.w) & 0xFFFFE000u); l.w = v.w - h.w;
+            h.x = tf32_head(v.x); l.x = v.x - h.x;
+            h.y = tf32_head(v.y); l.y = v.y - h.y;
+            h.z = tf32_head(v.z); l.z = v.z - h.z;
+            h.w = tf32_head(v.w); l.w = v.w - h.w;
             *reinterpret_cast<float4*>(hi + off) = h;
             *reinterpret_cast<float4*>(lo + off) = l;
         } else {

@@ -86,10 +86,10 @@ template <bool PRECISE>
 __device__ __forceinline__ void put(uint32_t hi, uint32_t lo, uint32_t off, float4 v) {
     if (PRECISE) {
         float4 h, l;
-        h.x = __uint_as_float(__float_as_uint(v.x) & 0xFFFFE000u); l.x = v.x - h.x;
-        h.y = __uint_as_float(__float_as_uint(v.y) & 0xFFFFE000u); l.y = v.y - h.y;
-        h.z = __uint_as_float(__float_as_uint(v.z) & 0xFFFFE000u); l.z = v.z - h.z;
-        h.w = __uint_as_float(__float_as_uint(v.w) & 0xFFFFE000u); l.w = v.w - h.w;
+        h.x = tc::tf32_head(v.x); l.x = v.x - h.x;
+        h.y = tc::tf32_head(v.y); l.y = v.y - h.y;
+        h.z = tc::tf32_head(v.z); l.z = v.z - h.z;
+        h.w = tc::tf32_head(v.w); l.w = v.w - h.w;
         asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(hi + off), "f"(h.x), "f"(h.y), "f"(h.z), "f"(h.w) : "memory");
         asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(lo + off), "f"(l.x), "f"(l.y), "f"(l.z), "f"(l.w) : "memory");
     } else {
@@ -109,8 +109,9 @@ __device__ __forceinline__ float lds32(uint32_t addr) {
 
 // TF32 head and remainder of one value.
 __device__ __forceinline__ void split(float v, uint32_t& hi, uint32_t& lo) {
-    hi = __float_as_uint(v) & 0xFFFFE000u;
-    lo = __float_as_uint(v - __uint_as_float(hi));
+    const float h = tc::tf32_head(v);
+    hi = __float_as_uint(h);
+    lo = __float_as_uint(v - h);
 }
 
 // 16 consecutive columns of this thread's TMEM lane.

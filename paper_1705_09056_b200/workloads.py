@@ -290,6 +290,45 @@ def stress_matrix(n: int, ld: int, N: int, seed: int, device) -> torch.Tensor:
     return M
 
 
+# --------------------------------------------------------------------------------------
+# Convolution layer family (stand-in for the paper's CIFAR-10 residual networks, Sections 5.1 / 5.3)
+# --------------------------------------------------------------------------------------
+
+# (C_in, C_out, stride) of the 3x3 convolutions: 32x32x3 inputs, widths 16 / 32 / 64, a stride-2 layer
+# where the width doubles (one layer of each kind a 20- or 32-layer residual network is built from).
+CIFAR_PLAN = ((3, 16, 1), (16, 16, 1), (16, 32, 2), (32, 32, 1), (32, 64, 2), (64, 64, 1))
+
+
+def conv_param_count(plan) -> int:
+    """Row layout [w_1 (C_out x C_in x 3 x 3, row-major) | b_1 | w_2 | b_2 | ...]."""
+    return sum(o * c * 9 + o for c, o, _ in plan)
+
+
+@dataclass
+class ConvWorkload:
+    """Per-node image minibatches and per-node filter banks (fp32 torch tensors on one device)."""
+    n: int
+    batch: int
+    plan: Tuple[Tuple[int, int, int], ...]
+    inputs: torch.Tensor       # [n][B][3][32][32], N(0,1)
+    params: torch.Tensor       # [n][conv_param_count(plan)], He-scaled filters, small non-zero biases
+
+
+def conv_workload(n=8, batch=32, plan=CIFAR_PLAN, hw=32, seed=170509061, device="cpu") -> ConvWorkload:
+    """CIFAR-shaped synthetic inputs (3 x hw x hw, N(0,1)) and, per node, its own He-initialised filters
+    (the nodes' models differ between synchronisations, so every node convolves with its own weights)."""
+    g = _gen(device, seed)
+    inputs = _randn((n, batch, plan[0][0], hw, hw), g, device)
+    rows = []
+    for _ in range(n):
+        parts = []
+        for (cin, cout, _) in plan:
+            parts.append((_randn((cout, cin, 3, 3), g, device) * math.sqrt(2.0 / (cin * 9))).reshape(-1))
+            parts.append(0.05 * _randn((cout,), g, device))
+        rows.append(torch.cat(parts))
+    return ConvWorkload(n, batch, tuple(tuple(p) for p in plan), inputs.contiguous(), torch.stack(rows).contiguous())
+
+
 def config(idx: int, device="cpu", **over) -> Workload:
     """The five benchmark configurations (0-based)."""
     if idx == 0:

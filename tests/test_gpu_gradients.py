@@ -231,3 +231,47 @@ def test_graph_replayed_run_is_bit_identical_to_steps(model):
     c.ctx.run(0, 29)
     assert row_rel_err(c.x(), o.X) <= TOL_TRAJ
     a.close(); b.close(); c.close()
+
+
+@pytest.mark.parametrize("model,n,d,m,B,batches", [
+    (binding.MODEL_LSQ, 8, 64, 1024, 16, None),           # config 1
+    (binding.MODEL_LOGISTIC, 6, 260, 300, 24, None),      # rows of more than one 32-lane pass, bias column
+    (binding.MODEL_LSQ, 5, 300, 200, 27, None),           # minibatch not a multiple of the eight slices
+    (binding.MODEL_LOGISTIC, 4, 128, 64, 16, [16, 1, 9, 4]),   # per-node minibatch sizes
+    (binding.MODEL_LSQ, 3, 4, 20, 3, None),
+])
+def test_one_launch_step_is_bit_identical_to_the_three_launches(model, n, d, m, B, batches):
+    """Small linear models: dpsgd_step runs sample, gradient and gossip step as ONE kernel (a CTA per
+    node).  X, G and the indices must equal those of the separate launches bit for bit, and the step takes
+    one launch."""
+    w = _linear_workload(model, n, d, m, B)
+    A, y = w.A.numpy(), w.y.numpy()
+    rng = np.random.default_rng(d)
+    X = (0.3 * rng.standard_normal((n, w.N))).astype(np.float32)
+    runs = []
+    for mode in (0, 1):
+        run = GpuRun(n, w.N, w.csr(), w.gamma, seed=11, X=X)
+        _attach(run, w, A, y)
+        if batches:
+            run.ctx.set_node_batches(batches)
+        run.ctx.set_fused_step(mode)
+        runs.append(run)
+    for k in range(5):
+        before = [r.ctx.launch_count() for r in runs]
+        for r in runs:
+            r.G.fill_(7.0)
+            r.ctx.step(k)
+        assert runs[0].ctx.launch_count() - before[0] == 3
+        assert runs[1].ctx.launch_count() - before[1] == 1
+        assert np.array_equal(runs[0].g(), runs[1].g()), k
+        assert np.array_equal(runs[0].x(), runs[1].x()), k
+        assert torch.equal(runs[0].G, runs[1].G)                      # padding columns too
+    o = orc.Oracle(n, w.N, *w.csr(), w.gamma, 11, w.model, w.dims, B, w.l2_lambda, A, y)
+    if not batches:
+        o.set_x(X)
+        for k in range(5):
+            o.step(k)
+        assert row_rel_err(runs[1].x(), o.X) <= 5 * TOL_STEP
+    for r in runs:
+        r.check_pads()
+        r.close()

@@ -71,11 +71,22 @@ def test_dense_w_swapped_order_is_centralized_sgd_on_the_gpu():
     run.close()
 
 
-@pytest.mark.parametrize("topo,n,N,swapped", [("ring", 16, 4097, False), ("ring", 112, 20011, False),
-                                              ("ring", 8, 333, True), ("dense", 64, 30000, False),
-                                              ("dense", 5, 77, False), ("torus", 16, 2500, False),
-                                              ("torus", 16, 2500, True), ("ring", 3, 5, False)])
-def test_fused_consensus_matches_oracle(topo, n, N, swapped):
+TILED = binding.MIX_TILED_CSR
+
+
+@pytest.mark.parametrize("topo,n,N,swapped,kind", [
+    ("ring", 16, 4097, False, -1), ("ring", 112, 20011, False, -1), ("ring", 8, 333, True, -1),
+    ("dense", 64, 30000, False, -1), ("dense", 5, 77, False, -1), ("torus", 16, 2500, False, -1),
+    ("torus", 16, 2500, True, -1), ("ring", 3, 5, False, -1),
+    # any sparse W on the tile-staging kernel: the statistics come out of the gossip pass itself
+    ("torus", 64, 40007, False, -1),            # beyond the small-problem switch: tiles of 64 columns, ragged tail
+    ("torus", 64, 40007, True, -1),
+    ("torus", 16, 2500, False, TILED), ("torus", 16, 2500, True, TILED),      # tiles of 128 columns
+    ("torus", 100, 3001, False, TILED),         # one CTA per SM, 64-column tiles
+    ("torus", 9, 1000, False, TILED), ("ring+antipode", 8, 70001, True, TILED),
+    ("ring", 200, 777, False, TILED),           # 200 rows per tile: one stage fills most of the shared memory
+])
+def test_fused_consensus_matches_oracle(topo, n, N, swapped, kind):
     rng = np.random.default_rng(N)
     csr = wl.topology(topo, n)
     X = (2.0 + 0.05 * rng.standard_normal((n, N))).astype(np.float32)     # small spread on an offset
@@ -83,8 +94,13 @@ def test_fused_consensus_matches_oracle(topo, n, N, swapped):
     run = GpuRun(n, N, csr, 0.1, X=X)
     run.set_g(G)
     run.ctx.set_order(swapped)
+    if kind >= 0:
+        run.ctx.mix_kind(kind)
     out = torch.full((1,), -1.0, dtype=torch.float64, device="cuda")
+    before = run.ctx.launch_count()
     run.ctx.mix_update_consensus(out)
+    if kind == TILED or (topo == "torus" and n * N * 4 > 8 << 20):
+        assert run.ctx.launch_count() - before == 2            # gossip kernel + the fixed-order sum of its partials
     ref = (orc.mix_update_swapped if swapped else orc.mix_update)(X, G, *csr, 0.1)
     assert row_rel_err(run.x(), ref) <= TOL_STEP
     c_ref = orc.consensus_dist(ref)
