@@ -341,11 +341,62 @@ def mlp_iterations(torch, binding, wl, dev, peak, cpu_legs, steps=20, warmup=3):
     return out
 
 
+def conv_layers(torch, binding, wl, dev, peak, cpu_legs, n=32, batch=32, reps=20):
+    """The convolution layer family of the paper's image workloads (3x3, CIFAR-shaped 32x32x3 inputs, widths
+    16/32/64): forward pass of the six layers for n nodes, every node with the filters of its own row."""
+    w = wl.conv_workload(n=n, batch=batch, device=dev)
+    N = w.params.shape[1]
+    X0 = torch.zeros((n, wl.padded_ld(N)), device=dev)
+    X0[:, :N] = w.params
+    X1, G = torch.zeros_like(X0), torch.zeros_like(X0)
+    ctx = binding.Dpsgd(n, N, *wl.ring(n), gamma=0.1)
+    ctx.bind(X0, X1, G)
+    offs, off = [], 0
+    for (cin, cout, _) in w.plan:
+        offs.append((off, off + cout * cin * 9))
+        off += cout * cin * 9 + cout
+    acts, hw = [w.inputs], 32
+    for (cin, cout, stride) in w.plan:
+        hw = (hw - 1) // stride + 1
+        acts.append(torch.empty((n, batch, cout, hw, hw), device=dev))
+
+    def forward(r):
+        for _ in range(r):
+            for l, ((cin, cout, stride), (wo, bo)) in enumerate(zip(w.plan, offs)):
+                ctx.conv3x3_forward(acts[l], cout, stride, wo, bo, True, acts[l + 1])
+
+    forward(3)
+    l0 = ctx.launch_count()
+    ms = _event_ms(torch, forward, reps)
+    launches = (ctx.launch_count() - l0) / reps
+    flops = sum(2.0 * 9 * cin * cout * acts[l + 1].shape[3] * acts[l + 1].shape[4] * n * batch
+                for l, (cin, cout, _) in enumerate(w.plan))
+    bytes_step = 4 * sum(a.numel() for a in acts[:-1]) + 4 * sum(a.numel() for a in acts[1:])   # every layer reads its input, writes its output
+    res = {"n": n, "batch": batch, "layers": [list(p) for p in w.plan], "ms_per_forward": ms, "launches_per_forward": launches,
+           "images_per_s": n * batch / (ms * 1e-3), "fp32_equivalent_TFLOPs": flops / (ms * 1e-3) / 1e12,
+           "algorithmic_bytes_per_forward": bytes_step, "GBps": bytes_step / (ms * 1e-3) / 1e9,
+           "frac_of_measured_peak": bytes_step / (ms * 1e-3) / 1e9 / peak}
+    ctx.sync()
+    if cpu_legs:
+        from oracle import conv_oracle as co
+        x = w.inputs[0, :4].cpu().numpy()
+        prm = w.params[0].cpu().numpy()
+        t0 = time.perf_counter()
+        co.layers_forward(x, prm, w.plan)
+        dt = time.perf_counter() - t0
+        res["cpu_baseline"] = {"value": 4 / dt, "unit": "images/s", "cores": 1, "kind": "oracle",
+                               "host_cores_available": os.cpu_count(),
+                               "sample": "the six layers on 4 images of one node (fp64 einsum per filter tap)"}
+    ctx.close()
+    return res
+
+
 def whole_iterations(torch, binding, wl, dev, peak, cpu_legs=True):
     """Whole D-PSGD iterations (sample + gradient + mix + update) of the four model configurations.
     Context for the headline line, which times the gossip step alone on configuration 4."""
     out = linear_iterations(torch, binding, wl, dev, peak, cpu_legs)
     out.update(mlp_iterations(torch, binding, wl, dev, peak, cpu_legs))
+    out["conv3x3_forward_cifar_layers_n32"] = conv_layers(torch, binding, wl, dev, peak, cpu_legs)
     return out
 
 

@@ -348,7 +348,8 @@ glm_node_step_kernel(const float4* __restrict__ X, float4* __restrict__ G, float
     float4* rows = reinterpret_cast<float4*>(node_smem);                   // [B][d4]
     float4* xs = rows + (size_t)B * d4;                                    // [ld4] the node's own row
     float4* gs = xs + ld4;                                                 // [ld4] its gradient row
-    float4* red = gs + ld4;                                                // [8][32]
+    float4* ms = gs + ld4;                                                 // [ld4] sum_j W_ij X[j], formed while the rows load
+    float4* red = ms + ld4;                                                // [8][32]
     float* scoef = reinterpret_cast<float*>(red + 8 * 32);                 // [B]
     int32_t* sj = reinterpret_cast<int32_t*>(scoef + B);                   // [B]
     if (k_ptr) k = *k_ptr;
@@ -359,7 +360,19 @@ glm_node_step_kernel(const float4* __restrict__ X, float4* __restrict__ G, float
         sj[b] = j;
         idx[node * B + b] = j;
     }
-    for (int64_t c = tid; c < ld4; c += kNodeThreads) xs[c] = __ldg(X + (int64_t)node * ld4 + c);
+    const int p0 = __ldg(row_ptr + node), pe = __ldg(row_ptr + node + 1);
+    for (int64_t c = tid; c < ld4; c += kNodeThreads) {
+        xs[c] = __ldg(X + (int64_t)node * ld4 + c);
+        // the mixing half of the gossip step needs X_k only: its loads overlap the gathers of the sampled rows
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int p = p0; p < pe; ++p) {
+            const float w = __ldg(val + p);
+            const float4 v = __ldg(X + (int64_t)__ldg(col + p) * ld4 + c);
+            a.x = fmaf(w, v.x, a.x); a.y = fmaf(w, v.y, a.y);
+            a.z = fmaf(w, v.z, a.z); a.w = fmaf(w, v.w, a.w);
+        }
+        ms[c] = a;
+    }
     __syncthreads();
     for (int e = tid; e < B * d4; e += kNodeThreads) {
         const int b = e / d4, c = e - b * d4;
@@ -434,18 +447,11 @@ glm_node_step_kernel(const float4* __restrict__ X, float4* __restrict__ G, float
         }
     }
     __syncthreads();
-    // gradient row out, then the gossip step on this node's row
-    const int p0 = __ldg(row_ptr + node), pe = __ldg(row_ptr + node + 1);
+    // gradient row out, then the update half of the gossip step on this node's row
     for (int64_t c = tid; c < ld4; c += kNodeThreads) {
         const float4 g = gs[c];
         G[(int64_t)node * ld4 + c] = g;
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int p = p0; p < pe; ++p) {
-            const float w = __ldg(val + p);
-            const float4 v = __ldg(X + (int64_t)__ldg(col + p) * ld4 + c);
-            a.x = fmaf(w, v.x, a.x); a.y = fmaf(w, v.y, a.y);
-            a.z = fmaf(w, v.z, a.z); a.w = fmaf(w, v.w, a.w);
-        }
+        float4 a = ms[c];
         a.x = fmaf(ngamma, g.x, a.x); a.y = fmaf(ngamma, g.y, a.y);
         a.z = fmaf(ngamma, g.z, a.z); a.w = fmaf(ngamma, g.w, a.w);
         Xn[(int64_t)node * ld4 + c] = a;
@@ -453,7 +459,7 @@ glm_node_step_kernel(const float4* __restrict__ X, float4* __restrict__ G, float
 }
 
 size_t node_step_smem(const dpsgd_ctx* c) {
-    return sizeof(float) * ((size_t)c->batch * c->d + 2 * (size_t)c->ld + 8 * 32 * 4 + 2 * (size_t)c->batch);
+    return sizeof(float) * ((size_t)c->batch * c->d + 3 * (size_t)c->ld + 8 * 32 * 4 + 2 * (size_t)c->batch);
 }
 
 bool rows_path(const dpsgd_ctx* c) {

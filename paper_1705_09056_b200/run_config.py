@@ -7,6 +7,8 @@ timings as one JSON line.  Also the command to put under a profiler for a single
       4 MLP 1024-2048-2048-10)
   python -m paper_1705_09056_b200.run_config --config 3 --n 64 --N 2000000 --topology ring --steps 3
       the gossip step alone on supplied N(0,1) gradients (the bandwidth configuration, any shape)
+  python -m paper_1705_09056_b200.run_config --conv --n 32 --batch 32 --steps 5
+      forward pass of the CIFAR-shaped 3x3 convolution layers, every node with its own filters
 """
 from __future__ import annotations
 
@@ -57,6 +59,51 @@ def gossip_step_alone(args, dev):
     ctx.close()
 
 
+def conv_layers(args, dev):
+    """dpsgd_conv3x3_forward on the six CIFAR-shaped layers: total and per-layer CUDA-event times."""
+    n = args.n or 32
+    w = wl.conv_workload(n=n, batch=args.batch, device=dev)
+    N = w.params.shape[1]
+    X0 = torch.zeros((n, wl.padded_ld(N)), device=dev)
+    X0[:, :N] = w.params
+    ctx = binding.Dpsgd(n, N, *wl.ring(n), gamma=0.1)
+    ctx.bind(X0, torch.zeros_like(X0), torch.zeros_like(X0))
+    offs, off = [], 0
+    for (cin, cout, _) in w.plan:
+        offs.append((off, off + cout * cin * 9))
+        off += cout * cin * 9 + cout
+    acts, hw = [w.inputs], 32
+    for (cin, cout, stride) in w.plan:
+        hw = (hw - 1) // stride + 1
+        acts.append(torch.empty((n, args.batch, cout, hw, hw), device=dev))
+
+    def layer(l):
+        (cin, cout, stride), (wo, bo) = w.plan[l], offs[l]
+        ctx.conv3x3_forward(acts[l], cout, stride, wo, bo, True, acts[l + 1])
+
+    for _ in range(args.warmup):
+        for l in range(len(w.plan)):
+            layer(l)
+    per_layer = []
+    for l, (cin, cout, stride) in enumerate(w.plan):
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(args.steps):
+            layer(l)
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / args.steps
+        flops = 2.0 * 9 * cin * cout * acts[l + 1].shape[3] * acts[l + 1].shape[4] * n * args.batch
+        moved = 4 * (acts[l].numel() + acts[l + 1].numel())
+        per_layer.append({"layer": [cin, cout, stride], "ms": ms, "fp32_equivalent_TFLOPs": flops / ms / 1e9,
+                          "GBps": moved / ms / 1e6})
+    ctx.sync()
+    print(json.dumps({"workload": "conv3x3 forward, CIFAR-shaped layers", "n": n, "batch": args.batch,
+                      "ms_per_forward": sum(p["ms"] for p in per_layer), "layers": per_layer}))
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", type=int, default=2, choices=[0, 1, 2, 3, 4])
@@ -65,6 +112,8 @@ def main():
     ap.add_argument("--n", type=int, default=0, help="override the node count")
     ap.add_argument("--N", type=int, default=0, help="config 3: parameters per replica (default 25,000,000)")
     ap.add_argument("--kind", type=int, default=-1, help="config 3: force a DPSGD_MIX_* kernel")
+    ap.add_argument("--conv", action="store_true", help="time the convolution layer family instead of a configuration")
+    ap.add_argument("--batch", type=int, default=32, help="--conv: images per node")
     ap.add_argument("--momentum", type=float, default=0.0,
                     help="config 3: momentum of the Section 5.3 runs (one more matrix)")
     ap.add_argument("--m", type=int, default=0, help="override the local dataset size")
@@ -82,6 +131,8 @@ def main():
 
     build.build()
     dev = torch.device("cuda", 0)
+    if args.conv:
+        return conv_layers(args, dev)
     if args.config == 3:
         return gossip_step_alone(args, dev)
     over = {}

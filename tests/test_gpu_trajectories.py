@@ -76,12 +76,12 @@ def oracle_mlp_step(o, k):
     return oracle_mix_update_blocks(o, np.stack(rows))
 
 
-def _context(w, seed, mode=None):
+def _context(w, seed, mode=None, precision=0):
     X0 = wl.stack_rows(w.x0, w.n, w.ld)
     X1, G = torch.zeros_like(X0), torch.zeros_like(X0)
     ctx = binding.Dpsgd(w.n, w.N, *w.csr(), gamma=w.gamma, seed=seed)
     ctx.bind(X0, X1, G)
-    ctx.set_model(w.model, w.dims, w.l2_lambda, w.batch, 0)
+    ctx.set_model(w.model, w.dims, w.l2_lambda, w.batch, precision)
     ctx.set_data(w.A, w.y)
     if mode is not None:
         ctx.set_fused_step(mode)
@@ -147,7 +147,7 @@ def match_gate_decisions(dims, x, A_i, y_i, idx_i, g_gpu, g_or):
     chosen, best = [], g_or
     ref_norm = np.linalg.norm(g_or.astype(np.float64))
     best_err = np.linalg.norm(diff)
-    for t in ties[:24]:
+    for t in ties[:96]:
         if best_err <= 2e-5 * ref_norm:
             break
         cand = orc.grad_mlp(x, dims, A_i, y_i, idx_i, flip=chosen + [t]).astype(np.float32)
@@ -157,7 +157,54 @@ def match_gate_decisions(dims, x, A_i, y_i, idx_i, g_gpu, g_or):
     return best, chosen
 
 
-def run_mlp_trajectory(w, seed, free_modes, consensus_every_step, label, explain_every=1, rows_always=False):
+def _resync_step(sync, o, X_k, G_or, A, y, idx, k, N, n, dev, label, explain_every, flips, first_flip, worst):
+    """One iteration of the resynchronised leg of run_mlp_trajectory: the context `sync` holds the oracle's X_k and
+    its gradient of iteration k; o.X already is the oracle's X_{k+1}."""
+    Gs = sync._bufs[2]
+    G_ref = torch.from_numpy(G_or).to(dev)
+    gerr = _rows_rel_err_dev(Gs[:, :N], G_ref)
+    sync.mix_update()
+    X_cmp = torch.from_numpy(o.X).to(dev)
+    xerr_rows = _rows_rel_err_dev(sync.current()[:, :N], X_cmp)
+    explain = (k % explain_every == 0) or k < 4
+    bad = [i for i in range(n) if float(gerr[i]) > 5e-5 and
+           (explain or float(gerr[i]) > 1e-3 or float(xerr_rows[i]) > 1e-5)]
+    unexplained = int((gerr > 5e-5).sum()) - len(bad)
+
+    def resolve(i):                      # a ReLU decision at an fp32 tie went the other way?
+        g_gpu = Gs[i, :N].cpu().numpy().astype(np.float64)
+        best, chosen = match_gate_decisions(o.dims, X_k[i], A[i], y[i], idx[i], g_gpu, G_or[i])
+        _, _, pre = orc._mlp_forward(X_k[i], o.dims, A[i], idx[i])
+        return best, [(l, b, u, float(pre[l][b, u])) for (l, b, u) in chosen], oracle_mix_update_row(o, X_k, i, best)
+
+    for i, (best, chosen, x_row) in zip(bad, POOL.map(resolve, bad)):
+        assert chosen, (label, k, i, float(gerr[i]), "gradient differs and no near-zero pre-activation explains it")
+        for (l, b, u, z) in chosen:
+            flips.append({"k": k, "node": i, "layer": l, "sample": b, "unit": u, "z": z,
+                          "G_err_unmatched": float(gerr[i])})
+        G_ref[i] = torch.from_numpy(best).to(dev)
+        X_cmp[i] = torch.from_numpy(x_row).to(dev)     # the step with the kernel's gate decisions
+    if bad or unexplained:
+        if first_flip is None:
+            first_flip = k
+    if bad:
+        gerr_fixed = _rows_rel_err_dev(Gs[:, :N], G_ref)
+        for i in bad:
+            assert float(gerr_fixed[i]) <= 5e-5, (label, k, i, float(gerr_fixed[i]))
+            gerr[i] = gerr_fixed[i]
+    within = gerr[gerr <= 5e-5]                          # rows in tolerance, natively or with flips resolved
+    if within.numel():
+        worst["G"] = max(worst["G"], float(within.max()))
+    worst["unresolved"] = worst.get("unresolved", 0) + unexplained
+    assert float(gerr.max()) <= 1e-3, (label, k, float(gerr.max()))
+    xerr = float(_rows_rel_err_dev(sync.current()[:, :N], X_cmp).max())
+    worst["X"] = max(worst["X"], xerr)
+    assert xerr <= 1e-5, (label, k, xerr)
+    return first_flip, worst
+
+
+def run_mlp_trajectory(w, seed, free_modes, consensus_every_step, label, explain_every=1, rows_always=False,
+                       resync=True, blas_threads=1):
     """Algorithm 1 for T = w.iterations iterations of an MLP configuration, three ways at once:
 
       oracle ........ free-running, its own fp64 arithmetic throughout (the reference trajectory);
@@ -182,64 +229,37 @@ def run_mlp_trajectory(w, seed, free_modes, consensus_every_step, label, explain
     T, N, n = w.iterations, w.N, w.n
     dev = w.A.device
     sync = _context(w, seed, 0)
-    free = {name: _context(w, seed, mode) for name, mode in free_modes.items()}
+    # free_modes: name -> fused-step mode, or (mode, mlp_precision)
+    free = {name: _context(w, seed, *(mode if isinstance(mode, tuple) else (mode,))) for name, mode in free_modes.items()}
     A, y = w.A.cpu().numpy(), w.y.cpu().numpy()
     o = orc.Oracle(n, N, *w.csr(), w.gamma, seed, w.model, w.dims, w.batch, 0.0, A, y)
     o.set_x(np.tile(w.x0.cpu().numpy(), (n, 1)))
     log = {name: torch.zeros(T, dtype=torch.float64, device=dev) for name in free}
     flips, first_flip, worst = [], None, {"G": 0.0, "X": 0.0}
-    Gs = sync._bufs[2]
+    spent = {"oracle_gradients": 0.0, "oracle_gossip": 0.0, "resync": 0.0, "free": 0.0}
     t0 = time.time()
-    with threadpool_limits(limits=1):            # one BLAS thread per node: the pool supplies the parallelism
+    with threadpool_limits(limits=blas_threads):   # few BLAS threads per node: the pool supplies the parallelism
         for k in range(T):
             idx = o.sample(k)
-            assert np.array_equal(sync.sample(k).cpu().numpy(), idx), k
-            # ---- resynchronised leg: same start, one iteration
+            assert np.array_equal(next(iter(free.values())).sample(k).cpu().numpy(), idx), k
             X_k = o.X
-            sync.current()[:, :N] = torch.from_numpy(X_k).to(dev)
-            sync.grad(k)
+            t1 = time.time()
+            if resync:
+                sync.current()[:, :N] = torch.from_numpy(X_k).to(dev)
+                sync.grad(k)
             rows = list(POOL.map(lambda i: orc.grad_mlp(X_k[i], o.dims, A[i], y[i], idx[i]).astype(np.float32), range(n)))
             G_or = np.stack(rows)
-            G_ref = torch.from_numpy(G_or).to(dev)
-            gerr = _rows_rel_err_dev(Gs[:, :N], G_ref)
-            sync.mix_update()
+            t2 = time.time()
             oracle_mix_update_blocks(o, G_or)                    # the oracle's own next point
-            X_cmp = torch.from_numpy(o.X).to(dev)
-            xerr_rows = _rows_rel_err_dev(sync.current()[:, :N], X_cmp)
-            explain = (k % explain_every == 0) or k < 4
-            bad = [i for i in range(n) if float(gerr[i]) > 5e-5 and
-                   (explain or float(gerr[i]) > 1e-3 or float(xerr_rows[i]) > 1e-5)]
-            unexplained = int((gerr > 5e-5).sum()) - len(bad)
-
-            def resolve(i):                      # a ReLU decision at an fp32 tie went the other way?
-                g_gpu = Gs[i, :N].cpu().numpy().astype(np.float64)
-                best, chosen = match_gate_decisions(o.dims, X_k[i], A[i], y[i], idx[i], g_gpu, G_or[i])
-                _, _, pre = orc._mlp_forward(X_k[i], o.dims, A[i], idx[i])
-                return best, [(l, b, u, float(pre[l][b, u])) for (l, b, u) in chosen], oracle_mix_update_row(o, X_k, i, best)
-
-            for i, (best, chosen, x_row) in zip(bad, POOL.map(resolve, bad)):
-                assert chosen, (label, k, i, float(gerr[i]), "gradient differs and no near-zero pre-activation explains it")
-                for (l, b, u, z) in chosen:
-                    flips.append({"k": k, "node": i, "layer": l, "sample": b, "unit": u, "z": z,
-                                  "G_err_unmatched": float(gerr[i])})
-                G_ref[i] = torch.from_numpy(best).to(dev)
-                X_cmp[i] = torch.from_numpy(x_row).to(dev)     # the step with the kernel's gate decisions
-            if bad or unexplained:
-                if first_flip is None:
-                    first_flip = k
-            if bad:
-                gerr_fixed = _rows_rel_err_dev(Gs[:, :N], G_ref)
-                for i in bad:
-                    assert float(gerr_fixed[i]) <= 5e-5, (label, k, i, float(gerr_fixed[i]))
-                    gerr[i] = gerr_fixed[i]
-            within = gerr[gerr <= 5e-5]                          # rows in tolerance, natively or with flips resolved
-            if within.numel():
-                worst["G"] = max(worst["G"], float(within.max()))
-            worst["unresolved"] = worst.get("unresolved", 0) + unexplained
-            assert float(gerr.max()) <= 1e-3, (label, k, float(gerr.max()))
-            xerr = float(_rows_rel_err_dev(sync.current()[:, :N], X_cmp).max())
-            worst["X"] = max(worst["X"], xerr)
-            assert xerr <= 1e-5, (label, k, xerr)
+            t3 = time.time()
+            if resync:
+                # ---- resynchronised leg: same start, one iteration
+                first_flip, worst = _resync_step(sync, o, X_k, G_or, A, y, idx, k, N, n, dev, label, explain_every,
+                                                 flips, first_flip, worst)
+            t4 = time.time()
+            spent["oracle_gradients"] += t2 - t1
+            spent["oracle_gossip"] += t3 - t2
+            spent["resync"] += t4 - t3
             # ---- free-running legs
             for name, ctx in free.items():
                 if consensus_every_step:
@@ -261,17 +281,20 @@ def run_mlp_trajectory(w, seed, free_modes, consensus_every_step, label, explain
                         rec["consensus"] = float(log[name][k])
                         rec["consensus_oracle"] = c_or
                     _log(rec)
-                    if first_flip is None:
+                    if resync and first_flip is None:
                         assert e <= TOL_TRAJ and a <= TOL_AVG, (label, name, k, e, a)
                     if rows_always:
                         assert e <= TOL_TRAJ, (label, name, k, e)
-                    if consensus_every_step and (first_flip is None or rows_always):
+                    if consensus_every_step and resync and first_flip is None:
                         assert abs(rec["consensus"] - c_or) <= 2e-2 * c_or
+                    if consensus_every_step:          # logged by every iteration; close to the oracle's all along
+                        assert abs(rec["consensus"] - c_or) <= 0.1 * c_or, (label, name, k, rec["consensus"], c_or)
                     # sanity from the first flip on: neighbours on the same path, nothing blown up
                     assert e <= SANITY_ROWS and a <= SANITY_AVG, (label, name, k, e, a)
     _log({"config": label, "flips": flips[:200], "n_flips": len(flips), "first_flip": first_flip,
           "resync_worst_G": worst["G"], "resync_worst_X": worst["X"],
-          "gradient_rows_over_5e-5_not_resolved": worst.get("unresolved", 0)})
+          "gradient_rows_over_5e-5_not_resolved": worst.get("unresolved", 0), "seconds_spent": spent,
+          "seconds_total": time.time() - t0})
     for ctx in list(free.values()) + [sync]:
         ctx.sync()
         ctx.close()
@@ -345,8 +368,13 @@ def test_config4_stress_50_steps_fresh_gradients(topology):
 def test_config5_mlp_300_iterations_consensus_every_step(topology):
     """MLP 1024-2048-2048-10 (6,316,042 parameters per node), 4096 samples per node, minibatch 64,
     gamma 0.02, T = 300, consensus distance reported by every iteration (dpsgd_step_consensus); the ring
-    beside the averaging matrix of C-PSGD.  n = 8 nodes: what the oracle finishes in a few minutes."""
+    beside the averaging matrix of C-PSGD.  n = 4 nodes: what the oracle finishes in a few minutes.  The ring
+    run is also followed step by step (flips resolved every 25th iteration) and free-runs a second time on the
+    exact fp32 FMA kernels (mlp_precision = 2), whose pre-activations are ten times closer to the oracle's."""
     _need(8)
-    w = wl.config(4, device="cuda", n=8, topology=topology)
+    w = wl.config(4, device="cuda", n=4, topology=topology)
     assert w.iterations == 300 and w.batch == 64 and w.dims == (1024, 2048, 2048, 10)
-    run_mlp_trajectory(w, 20254, {"default": 1}, True, "5-" + topology, explain_every=10, rows_always=True)
+    ring = topology == "ring"
+    modes = {"default": 1, "fp32_fma": (1, 2)} if ring else {"default": 1}
+    run_mlp_trajectory(w, 20254, modes, True, "5-" + topology, explain_every=25, rows_always=True, resync=ring,
+                       blas_threads=4)
