@@ -278,6 +278,30 @@ DPSGD_API dpsgd_status dpsgd_conv3x3_forward(dpsgd_ctx* ctx, const float* in_dev
                                              int32_t w, int32_t c_out, int32_t stride, int64_t w_off, int64_t b_off,
                                              int32_t relu, float* out_dev);
 
+/*
+ * Backward of dpsgd_conv3x3_forward for the same layer, all nodes at once (gradient half of Algorithm 1 step 3
+ * for the image workloads of Sections 5.1 / 5.3).  With dym = dout * [out > 0] for a ReLU layer (ReLU'(0) = 0),
+ * dym = dout otherwise:
+ *   G[i][b_off + o]                      <- sum_{b,p,q} dym[i][b][o][p][q]
+ *   G[i][w_off + ((o c_in + c) 3 + kh) 3 + kw] <- sum_{b,p,q} dym[i][b][o][p][q] * in[i][b][c][stride p + kh - 1][stride q + kw - 1]
+ *   din[i][b][c][y][x] <- sum_{o,kh,kw} w_i[o][c][kh][kw] * dym[i][b][o][p][q] over stride p + kh - 1 = y, stride q + kw - 1 = x
+ * i.e. the filter and bias blocks of node i's row of the bound gradient matrix G receive SUMS over the minibatch
+ * (the caller's dout carries the 1/B of a mean loss), and din (optional, NULL = not wanted) receives the
+ * gradient at the layer's input.  Filters are read from the current X.
+ *   in_dev / out_dev   the layer's input and its output as dpsgd_conv3x3_forward wrote it (out_dev only read for
+ *                      relu != 0); dout_dev: gradient at the output, same shape as out_dev; all fp32, device,
+ *                      16-byte aligned, caller-owned.
+ * The contractions run on the tensor-core kernels (three TF32 MMAs per product); the library keeps a scratch
+ * buffer of about (9 c_in + c_out) x the size of dout (allocated on the first call, grown when a larger layer
+ * comes, released by dpsgd_destroy).  Asynchronous on the bound stream; results are bit-reproducible.
+ * din needs c_in to be a multiple of 16 and the shape limits of dpsgd_conv3x3_forward on the input's size;
+ * n * batch <= 65535.  Errors: DPSGD_ERR_ARG, DPSGD_ERR_ALIGN, DPSGD_ERR_UNSUPPORTED, DPSGD_ERR_CUDA.
+ */
+DPSGD_API dpsgd_status dpsgd_conv3x3_backward(dpsgd_ctx* ctx, const float* in_dev, const float* out_dev,
+                                              const float* dout_dev, int32_t batch, int32_t c_in, int32_t h, int32_t w,
+                                              int32_t c_out, int32_t stride, int64_t w_off, int64_t b_off, int32_t relu,
+                                              float* din_dev);
+
 /* Output of Algorithm 1: xbar = (1/n) sum_i x_i into xbar_dev (fp32 [ld], 16-byte aligned). */
 DPSGD_API dpsgd_status dpsgd_average(dpsgd_ctx* ctx, float* xbar_dev);
 

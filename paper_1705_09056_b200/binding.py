@@ -51,6 +51,7 @@ SIGNATURES = {
     "dpsgd_selftest_wait": [_vp, ctypes.c_uint32],
     "dpsgd_average": [_vp, _vp],
     "dpsgd_conv3x3_forward": [_vp, _vp, _i32, _i32, _i32, _i32, _i32, _i32, _i64, _i64, _i32, _vp],
+    "dpsgd_conv3x3_backward": [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32, _i32, _i64, _i64, _i32, _vp],
     "dpsgd_mix_update_host": [_vp, _vp, _i64, ctypes.POINTER(ctypes.c_double)],
     "dpsgd_consensus_dist_noalloc": [_vp, _i32, _i64, _i64, _vp, _vp],
     "dpsgd_current": [_vp, ctypes.POINTER(_vp)],
@@ -269,6 +270,18 @@ class Dpsgd:
         self._check(self._lib.dpsgd_conv3x3_forward(self._h, _ptr(x), B, C, H, W, c_out, stride, w_off, b_off,
                                                     1 if relu else 0, _ptr(out)))
         return out
+
+    def conv3x3_backward(self, x: torch.Tensor, y: Optional[torch.Tensor], dy: torch.Tensor, stride: int, w_off: int,
+                         b_off: int, relu: bool = True, want_dx: bool = True) -> Optional[torch.Tensor]:
+        """Backward of conv3x3_forward: filter and bias gradients (sums over the minibatch) into the bound G at
+        columns w_off / b_off; returns the gradient at the layer's input (None when want_dx is False)."""
+        assert x.is_cuda and x.is_contiguous() and dy.is_cuda and dy.is_contiguous() and x.dim() == 5 and dy.dim() == 5
+        _, B, C, H, W = x.shape
+        c_out = dy.shape[2]
+        dx = torch.empty_like(x) if want_dx else None
+        self._check(self._lib.dpsgd_conv3x3_backward(self._h, _ptr(x), _ptr(y), _ptr(dy), B, C, H, W, c_out, stride,
+                                                     w_off, b_off, 1 if relu else 0, _ptr(dx)))
+        return dx
 
     def average(self, xbar: Optional[torch.Tensor] = None) -> torch.Tensor:
         if xbar is None:

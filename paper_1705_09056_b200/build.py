@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdpsgd.so")
 SOURCES = ["api.cu", "mix_update.cu", "mix_variants.cu", "mix_tiled.cu", "consensus.cu", "sampler.cu",
-           "grad_linear.cu", "grad_mlp.cu", "tc_wgrad_fused.cu", "conv_fwd.cu"]
+           "grad_linear.cu", "grad_mlp.cu", "tc_wgrad_fused.cu", "conv_fwd.cu", "conv_bwd.cu"]
 FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
          "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--use_fast_math=false"]
 

@@ -138,6 +138,7 @@ void release(dpsgd_ctx* c) {
     cudaFree(c->d_act);
     cudaFree(c->d_delta);
     cudaFree(c->d_partials);
+    cudaFree(c->d_conv_ws);
     cudaFree(c->d_result);
     if (c->h_result) cudaFreeHost(c->h_result);
     delete c;
@@ -745,6 +746,27 @@ DPSGD_API dpsgd_status dpsgd_conv3x3_forward(dpsgd_ctx* c, const float* in_dev, 
     cudaError_t e = launch_conv3x3_forward(c, in_dev, batch, c_in, h, w, c_out, stride, w_off, b_off, relu, out_dev, &why);
     if (e == cudaErrorNotSupported && why) return fail(c, DPSGD_ERR_UNSUPPORTED, why);
     return e == cudaSuccess ? DPSGD_OK : cuda_fail(c, e, "convolution kernel");
+}
+
+DPSGD_API dpsgd_status dpsgd_conv3x3_backward(dpsgd_ctx* c, const float* in_dev, const float* out_dev,
+                                              const float* dout_dev, int32_t batch, int32_t c_in, int32_t h, int32_t w,
+                                              int32_t c_out, int32_t stride, int64_t w_off, int64_t b_off, int32_t relu,
+                                              float* din_dev) {
+    dpsgd_status s = need_bound(c);
+    if (s != DPSGD_OK) return s;
+    if (!in_dev || !dout_dev || (relu && !out_dev)) return fail(c, DPSGD_ERR_ARG, "in_dev, dout_dev (and out_dev of a ReLU layer) must not be NULL");
+    if (!aligned(in_dev, 16) || !aligned(dout_dev, 16) || !aligned(out_dev, 16) || !aligned(din_dev, 16))
+        return fail(c, DPSGD_ERR_ALIGN, "activation and gradient buffers must be 16-byte aligned");
+    if (batch < 1 || c_in < 1 || h < 1 || w < 1 || c_out < 1) return fail(c, DPSGD_ERR_ARG, "sizes must be positive");
+    if (stride != 1 && stride != 2) return fail(c, DPSGD_ERR_UNSUPPORTED, "stride must be 1 or 2");
+    const int64_t wsz = (int64_t)c_out * c_in * 9;
+    if (w_off < 0 || b_off < 0 || w_off + wsz > c->N || b_off + c_out > c->N)
+        return fail(c, DPSGD_ERR_ARG, "filter or bias block lies outside the parameter row");
+    const char* why = nullptr;
+    cudaError_t e = launch_conv3x3_backward(c, in_dev, out_dev, dout_dev, batch, c_in, h, w, c_out, stride, w_off, b_off,
+                                            relu, din_dev, &why);
+    if (e == cudaErrorNotSupported && why) return fail(c, DPSGD_ERR_UNSUPPORTED, why);
+    return e == cudaSuccess ? DPSGD_OK : cuda_fail(c, e, "convolution backward kernels");
 }
 
 DPSGD_API dpsgd_status dpsgd_average(dpsgd_ctx* c, float* xbar) {

@@ -55,7 +55,7 @@ constexpr uint32_t kTmemCols = 256;  // accumulator + two converted blocks, roun
 
 struct Args {
     const float* W;          // first filter of node 0 (inside its parameter row); node stride ld_w
-    const float* bias;       // first bias of node 0; same stride
+    const float* bias;       // first bias of node 0; same stride (NULL: no bias)
     int64_t ld_w;
     float* Y;                // [n][B][C_out_total][Ho][Wo]
     int n, B, C_in, C_out_total, o0;   // this launch computes channels [o0, o0 + ROWS_B)
@@ -217,14 +217,14 @@ conv3x3_fwd_kernel(const __grid_constant__ CUtensorMap mapX, Args g) {
             const bool live = pg < total_pos;
             const int img = pg / pos_per_img, pin_g = pg - img * pos_per_img;
             float* yb = g.Y + (((int64_t)node * g.B + img) * g.C_out_total + g.o0) * pos_per_img + pin_g;
-            const float* bn = g.bias + (int64_t)node * g.ld_w + g.o0;
+            const float* bn = g.bias ? g.bias + (int64_t)node * g.ld_w + g.o0 : nullptr;
 #pragma unroll 1
             for (int c0 = 0; c0 < ROWS_B; c0 += 16) {
                 float v[16];
                 tc::tmem_ld16(lane_base + (uint32_t)c0, v);
 #pragma unroll
                 for (int u = 0; u < 16; ++u) {
-                    float x = v[u] + __ldg(bn + c0 + u);
+                    float x = bn ? v[u] + __ldg(bn + c0 + u) : v[u];
                     if (g.relu && !(x > 0.f)) x = 0.f;
                     if (live) yb[(int64_t)(c0 + u) * pos_per_img] = x;
                 }
@@ -329,6 +329,13 @@ const char* conv3x3_forward_unsupported(int batch, int c_in, int h, int w, int c
 
 cudaError_t launch_conv3x3_forward(dpsgd_ctx* c, const float* x, int batch, int c_in, int h, int w, int c_out, int stride,
                                    int64_t w_off, int64_t b_off, int relu, float* y, const char** why) {
+    return launch_conv3x3_forward_on(c, x, batch, c_in, h, w, c_out, stride, c->X[c->cur] + w_off, c->X[c->cur] + b_off,
+                                     c->ld, relu, y, why);
+}
+
+cudaError_t launch_conv3x3_forward_on(dpsgd_ctx* c, const float* x, int batch, int c_in, int h, int w, int c_out,
+                                      int stride, const float* W, const float* bias, int64_t ld_w, int relu, float* y,
+                                      const char** why) {
     using namespace conv;
     *why = nullptr;
     Args a{};
@@ -345,7 +352,7 @@ cudaError_t launch_conv3x3_forward(dpsgd_ctx* c, const float* x, int batch, int 
     a.patch_stride = (a.patch_bytes + 127u) & ~127u;
     a.log2_wo = ilog2(a.Wo);
     a.log2_img = ilog2(std::min(pos, kTileP));
-    a.W = c->X[c->cur] + w_off; a.bias = c->X[c->cur] + b_off; a.ld_w = c->ld;
+    a.W = W; a.bias = bias; a.ld_w = ld_w;
     a.Y = y;
     a.status = &c->d_result->status;
     if (a.rows_patch > 256) { *why = "the input patch of a tile is taller than a TMA box"; return cudaErrorNotSupported; }

@@ -121,6 +121,10 @@ struct dpsgd_ctx {
     int fuse_step = 1;         // 0 off, 1 where it pays (default), 2 wherever a fused kernel applies, 3 as 2 without the ring kernel
     std::vector<std::pair<int64_t, int64_t>> fused_blocks;   // [begin, end) columns already written to X_next
 
+    // convolution backward: masked output gradient, unfolded input, per-image filter gradients, flipped filters
+    float* d_conv_ws = nullptr;
+    size_t conv_ws_floats = 0;
+
     int64_t launches = 0;
     std::string err;
 };
@@ -172,6 +176,18 @@ cudaError_t launch_mix_rest(dpsgd_ctx* c, const float* X, const float* G, float*
 const char* conv3x3_forward_unsupported(int batch, int c_in, int h, int w, int c_out, int stride);
 cudaError_t launch_conv3x3_forward(dpsgd_ctx* c, const float* x, int batch, int c_in, int h, int w, int c_out, int stride,
                                    int64_t w_off, int64_t b_off, int relu, float* y, const char** why);
+// Backward of the same layer (conv_bwd.cu): filter and bias gradients into G, optionally the input gradient.
+cudaError_t launch_conv3x3_backward(dpsgd_ctx* c, const float* x, const float* y, const float* dy, int batch, int c_in,
+                                    int h, int w, int c_out, int stride, int64_t w_off, int64_t b_off, int relu,
+                                    float* dx, const char** why);
+// Forward kernel on filters outside the parameter matrix (W: first filter of node 0, rows ld_w apart; bias may be
+// NULL = none): what the input gradient runs on.
+cudaError_t launch_conv3x3_forward_on(dpsgd_ctx* c, const float* x, int batch, int c_in, int h, int w, int c_out,
+                                      int stride, const float* W, const float* bias, int64_t ld_w, int relu, float* y,
+                                      const char** why);
+cudaError_t launch_tc_gemm_kmajor(dpsgd_ctx* c, const float* A, int64_t a_problem, int64_t a_pitch, const float* B,
+                                  int64_t b_problem, int64_t b_pitch, float* C, int64_t c_problem, int64_t c_pitch,
+                                  int M, int N, int K, int problems);
 size_t mlp_act_floats(const dpsgd_ctx* c);
 size_t mlp_delta_floats(const dpsgd_ctx* c);
 

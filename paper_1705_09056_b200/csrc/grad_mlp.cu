@@ -211,28 +211,28 @@ void run_gemm(dpsgd_ctx* c, const GemmArgs& g) {
 }
 
 template <int NT, bool A_K, bool B_K, bool VEC, bool PRECISE>
-cudaError_t launch_tc_inst(dpsgd_ctx* c, const tc::Args& a, int n_tiles) {
+cudaError_t launch_tc_inst(dpsgd_ctx* c, const tc::Args& a, int n_tiles, int problems) {
     auto kernel = tc::tc_gemm_kernel<NT, A_K, B_K, VEC, PRECISE>;
     constexpr size_t smem = tc::smem_bytes<NT, A_K, B_K, PRECISE>();
     // per device and cheap: set on every launch rather than remembered in a process-wide flag
     cudaError_t ea = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (ea != cudaSuccess) return ea;
-    dim3 grid((a.M + tc::kTileM - 1) / tc::kTileM, (n_tiles + a.n_per_cta - 1) / a.n_per_cta, c->n);
+    dim3 grid((a.M + tc::kTileM - 1) / tc::kTileM, (n_tiles + a.n_per_cta - 1) / a.n_per_cta, problems);
     kernel<<<grid, tc::kThreads, smem, c->stream>>>(a);
     c->launches++;
     return cudaGetLastError();
 }
 
 template <int NT, bool VEC>
-cudaError_t launch_tc_nt(dpsgd_ctx* c, const tc::Args& a, int n_tiles) {
+cudaError_t launch_tc_nt(dpsgd_ctx* c, const tc::Args& a, int n_tiles, int problems) {
     if (a.precise) {
-        if (a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, true, true, VEC, true>(c, a, n_tiles);
-        if (!a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, false, true, VEC, true>(c, a, n_tiles);
-        if (!a.a_kcontig && !a.b_kcontig) return launch_tc_inst<NT, false, false, VEC, true>(c, a, n_tiles);
+        if (a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, true, true, VEC, true>(c, a, n_tiles, problems);
+        if (!a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, false, true, VEC, true>(c, a, n_tiles, problems);
+        if (!a.a_kcontig && !a.b_kcontig) return launch_tc_inst<NT, false, false, VEC, true>(c, a, n_tiles, problems);
     } else {
-        if (a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, true, true, VEC, false>(c, a, n_tiles);
-        if (!a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, false, true, VEC, false>(c, a, n_tiles);
-        if (!a.a_kcontig && !a.b_kcontig) return launch_tc_inst<NT, false, false, VEC, false>(c, a, n_tiles);
+        if (a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, true, true, VEC, false>(c, a, n_tiles, problems);
+        if (!a.a_kcontig && a.b_kcontig) return launch_tc_inst<NT, false, true, VEC, false>(c, a, n_tiles, problems);
+        if (!a.a_kcontig && !a.b_kcontig) return launch_tc_inst<NT, false, false, VEC, false>(c, a, n_tiles, problems);
     }
     return cudaErrorInvalidValue;
 }
@@ -245,30 +245,33 @@ bool vec_ok(const float* p, int64_t pitch, int64_t node_stride, int contig_exten
 }
 
 // C[n][m] = epi(sum_k A(m,k) B(n,k)); max_tile = widest column tile (multiple of 16, <= 128).
-cudaError_t run_tc(dpsgd_ctx* c, tc::Args a, int max_tile) {
+// problems: independent problems in the launch (blockIdx.z), one per node unless given; force_precise: three
+// MMAs per product whatever the model's precision setting.
+cudaError_t run_tc(dpsgd_ctx* c, tc::Args a, int max_tile, int problems = -1, bool force_precise = false) {
+    if (problems < 0) problems = c->n;
     const bool vec = vec_ok(a.A, a.a_pitch, a.a_node, a.a_kcontig ? a.K : a.M) &&
                      vec_ok(a.B, a.b_pitch, a.b_node, a.b_kcontig ? a.K : a.N);
     a.a_vec = a.b_vec = vec;
-    a.precise = c->mlp_precision == 0;
+    a.precise = force_precise || c->mlp_precision == 0;
     a.status = &c->d_result->status;
     const int want = a.N < max_tile ? a.N : max_tile;
     {   // column tiles per CTA: up to 8 (keeps the A tile staged), but never so many that the grid
         // falls under about four CTAs per CTA slot of the device
         const int tile = want <= 16 ? 16 : (want <= 32 ? 32 : (want <= 64 ? 64 : 128));
-        const long long tiles = (long long)((a.M + tc::kTileM - 1) / tc::kTileM) * ((a.N + tile - 1) / tile) * c->n;
+        const long long tiles = (long long)((a.M + tc::kTileM - 1) / tc::kTileM) * ((a.N + tile - 1) / tile) * problems;
         const long long per = tiles / (4LL * 2 * 148);
         a.n_per_cta = (int)(per < 1 ? 1 : (per > 8 ? 8 : per));
     }
     if (vec) {
-        if (want <= 16) return launch_tc_nt<1, true>(c, a, (a.N + 15) / 16);
-        if (want <= 32) return launch_tc_nt<2, true>(c, a, (a.N + 31) / 32);
-        if (want <= 64) return launch_tc_nt<4, true>(c, a, (a.N + 63) / 64);
-        return launch_tc_nt<8, true>(c, a, (a.N + 127) / 128);
+        if (want <= 16) return launch_tc_nt<1, true>(c, a, (a.N + 15) / 16, problems);
+        if (want <= 32) return launch_tc_nt<2, true>(c, a, (a.N + 31) / 32, problems);
+        if (want <= 64) return launch_tc_nt<4, true>(c, a, (a.N + 63) / 64, problems);
+        return launch_tc_nt<8, true>(c, a, (a.N + 127) / 128, problems);
     }
-    if (want <= 16) return launch_tc_nt<1, false>(c, a, (a.N + 15) / 16);
-    if (want <= 32) return launch_tc_nt<2, false>(c, a, (a.N + 31) / 32);
-    if (want <= 64) return launch_tc_nt<4, false>(c, a, (a.N + 63) / 64);
-    return launch_tc_nt<8, false>(c, a, (a.N + 127) / 128);
+    if (want <= 16) return launch_tc_nt<1, false>(c, a, (a.N + 15) / 16, problems);
+    if (want <= 32) return launch_tc_nt<2, false>(c, a, (a.N + 31) / 32, problems);
+    if (want <= 64) return launch_tc_nt<4, false>(c, a, (a.N + 63) / 64, problems);
+    return launch_tc_nt<8, false>(c, a, (a.N + 127) / 128, problems);
 }
 
 // ---- weight-streaming kernel (tc_stream.cuh): forward and input-gradient products ----
@@ -407,6 +410,22 @@ cudaError_t run_tc_weights(dpsgd_ctx* c, const tc::Args& a) {
 }
 
 }  // namespace
+
+// Batched GEMM with both operands contiguous along k, for callers outside this file:
+//     C[p][nn * c_pitch + m] = sum_k A[p][m * a_pitch + k] * B[p][nn * b_pitch + k],   p < problems,
+// on the register-staged tensor-core kernel (tc_gemm.cuh), three TF32 MMAs per product.
+cudaError_t launch_tc_gemm_kmajor(dpsgd_ctx* c, const float* A, int64_t a_problem, int64_t a_pitch, const float* B,
+                                  int64_t b_problem, int64_t b_pitch, float* C, int64_t c_problem, int64_t c_pitch,
+                                  int M, int N, int K, int problems) {
+    tc::Args a{};
+    a.A = A; a.a_node = a_problem; a.a_pitch = a_pitch; a.a_kcontig = 1;
+    a.B = B; a.b_node = b_problem; a.b_pitch = b_pitch; a.b_kcontig = 1;
+    a.C = C; a.c_node = c_problem; a.c_pitch = c_pitch;
+    a.aux = nullptr; a.aux_node = 0; a.aux_pitch = 0;
+    a.M = M; a.N = N; a.K = K;
+    a.epi = tc::EPI_STORE;
+    return run_tc(c, a, 128, problems, true);
+}
 
 size_t mlp_act_floats(const dpsgd_ctx* c) {
     size_t a = 0;

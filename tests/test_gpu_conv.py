@@ -116,3 +116,77 @@ def test_filters_follow_the_current_parameter_buffer_and_bad_shapes_are_refused(
     assert e.value.status == binding.ERR_UNSUPPORTED
     ctx.sync()
     ctx.close()
+
+
+def _backward_reference(x, params, w_off, b_off, cin, cout, stride, relu, dy):
+    """Oracle: (dw, db, dx) of one node's layer, sums over the minibatch."""
+    w = params[w_off:w_off + cout * cin * 9].reshape(cout, cin, 3, 3)
+    b = params[b_off:b_off + cout]
+    _, pre = co.conv3x3_forward(x, w, b, stride, relu)
+    d = co.relu_backward(dy, pre) if relu else np.asarray(dy, dtype=np.float64)
+    dw, db = co.conv3x3_weight_grad(d, x, stride)
+    dx = co.conv3x3_input_grad(d, w, x.shape[2:], stride)
+    return dw, db, dx
+
+
+@pytest.mark.parametrize("n,batch", [(3, 4), (2, 16)])
+def test_backward_of_every_cifar_layer_matches_the_oracle(n, batch):
+    """Filter, bias and input gradients of each layer of the family, from the oracle's activations and a random
+    gradient at the layer's output.  The first layer (3 input channels) needs no input gradient."""
+    w = wl.conv_workload(n=n, batch=batch, seed=12)
+    ctx = _context(w.params)
+    Gdev = ctx._keep[2]
+    rng = np.random.default_rng(batch)
+    acts = [co.layers_forward(w.inputs[i].numpy(), w.params[i].numpy(), w.plan) for i in range(n)]
+    for l, ((cin, cout, stride), (w_off, b_off)) in enumerate(zip(w.plan, _offsets(w.plan))):
+        x_l = np.stack([acts[i][l] for i in range(n)])
+        y_l = np.stack([acts[i][l + 1] for i in range(n)])
+        dy = rng.standard_normal(y_l.shape).astype(np.float32)
+        Gdev.fill_(7.0)
+        want_dx = cin % 16 == 0
+        dx = ctx.conv3x3_backward(torch.from_numpy(x_l).cuda(), torch.from_numpy(y_l).cuda(), torch.from_numpy(dy).cuda(),
+                                  stride, w_off, b_off, relu=True, want_dx=want_dx)
+        G = Gdev.cpu().numpy().astype(np.float64)
+        refs = [_backward_reference(x_l[i], w.params[i].numpy(), w_off, b_off, cin, cout, stride, True, dy[i]) for i in range(n)]
+        dw = G[:, w_off:w_off + cout * cin * 9]
+        db = G[:, b_off:b_off + cout]
+        dw_ref = np.stack([r[0].reshape(-1) for r in refs])
+        db_ref = np.stack([r[1] for r in refs])
+        assert np.linalg.norm(dw - dw_ref, axis=1).max() <= 1e-5 * np.linalg.norm(dw_ref, axis=1).min(), ("dw", l)
+        assert np.abs(dw - dw_ref).max() <= 2e-5 * np.abs(dw_ref).max(), ("dw", l)
+        assert np.abs(db - db_ref).max() <= 2e-5 * np.abs(db_ref).max() + 1e-6, ("db", l)
+        # nothing but the layer's own blocks of G is written
+        keep = np.ones(G.shape[1], dtype=bool)
+        keep[w_off:w_off + cout * cin * 9] = False
+        keep[b_off:b_off + cout] = False
+        assert np.all(G[:, keep] == 7.0), l
+        if want_dx:
+            _check(dx, np.stack([r[2] for r in refs]), ("dx", l))
+    ctx.sync()
+    ctx.close()
+
+
+def test_backward_without_relu_ragged_batch_and_refusals():
+    n, B, cin, cout, h, wd, stride = 2, 3, 16, 32, 8, 8, 2
+    rng = np.random.default_rng(9)
+    N = cout * cin * 9 + cout
+    params = torch.from_numpy(rng.standard_normal((n, N)).astype(np.float32) / np.sqrt(cin * 9))
+    x = rng.standard_normal((n, B, cin, h, wd)).astype(np.float32)
+    dy = rng.standard_normal((n, B, cout, 4, 4)).astype(np.float32)
+    ctx = _context(params)
+    dx = ctx.conv3x3_backward(torch.from_numpy(x).cuda(), None, torch.from_numpy(dy).cuda(), stride, 0, cout * cin * 9,
+                              relu=False)
+    G = ctx._keep[2].cpu().numpy().astype(np.float64)
+    refs = [_backward_reference(x[i], params[i].numpy(), 0, cout * cin * 9, cin, cout, stride, False, dy[i]) for i in range(n)]
+    dw_ref = np.stack([r[0].reshape(-1) for r in refs])
+    assert np.abs(G[:, :cout * cin * 9] - dw_ref).max() <= 2e-5 * np.abs(dw_ref).max()
+    assert np.abs(G[:, cout * cin * 9:N] - np.stack([r[1] for r in refs])).max() <= 2e-5 * np.abs(dw_ref).max()
+    _check(dx, np.stack([r[2] for r in refs]), "dx without relu")
+    with pytest.raises(binding.DpsgdError) as e:           # a ReLU layer needs its output for the mask
+        ctx.conv3x3_backward(torch.from_numpy(x).cuda(), None, torch.from_numpy(dy).cuda(), stride, 0, cout * cin * 9, relu=True)
+    assert e.value.status == binding.ERR_ARG
+    with pytest.raises(binding.DpsgdError) as e:           # filters outside the row
+        ctx.conv3x3_backward(torch.from_numpy(x).cuda(), None, torch.from_numpy(dy).cuda(), stride, cout + 1, cout * cin * 9, relu=False)
+    assert e.value.status == binding.ERR_ARG
+    ctx.sync()
+    ctx.close()
