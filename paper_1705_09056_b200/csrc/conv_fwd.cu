@@ -13,7 +13,7 @@
 //                   (W_in, rows, C_in, images, node) of the NCHW input with one halo row above and below.
 //                   Rows outside the image are zero-filled by the TMA unit (the box starts at row -1);
 //                   the box always starts at column 0, so the copy is 16-byte aligned whatever the tap.
-//   converter warps (4) thread p owns output position p.  Per block of 32 k it gathers its row of the
+//   converter warps (8) two threads own an output position, 16 of a block's 32 k each.  Per block a thread gathers its part of the row of the
 //                   unfolded matrix from the patch in shared memory (a table gives, for every k, the offset
 //                   of tap (c, kh, kw) inside the patch; the left / right zero border is a predicate),
 //                   splits each value into its TF32 head and remainder and writes both to its TENSOR
@@ -22,8 +22,10 @@
 //                   shared-memory layout of the MMA descriptors (heads and remainders), for all of K.
 //   MMA warp        one thread issues, per block of 32 k, three TF32 MMAs per 8 k (lo*hi + hi*lo + hi*hi,
 //                   fp32 accumulation in tensor memory), A from tensor memory, B through descriptors.
-//   epilogue        the converter warps read the finished accumulator (tcgen05.ld), add the bias, apply the
-//                   ReLU and store with the positions contiguous across lanes (NCHW: 128-byte lines).
+//   epilogue        the converter warps read a finished accumulator (tcgen05.ld), add the bias, apply the
+//                   ReLU and store with the positions contiguous across lanes (NCHW: 128-byte lines).  There are
+//                   two accumulators and the epilogue of a tile runs after the NEXT tile's blocks have been
+//                   converted, so the tensor core never waits for it.
 //
 // CTAs are persistent and take CONTIGUOUS ranges of (node, tile), so a node's filters are converted once
 // per CTA that touches the node.  Every mbarrier wait is bounded; a wait that runs out raises the status
@@ -45,13 +47,14 @@ using tc::smem_u32;
 using tcs::lds32;
 using tcs::mbar_expect_tx;
 
-constexpr int kThreads = 192;        // 4 converter / epilogue warps, MMA warp, TMA warp
-constexpr int kConvThreads = 128;
+constexpr int kThreads = 320;        // 8 converter / epilogue warps, MMA warp, TMA warp
+constexpr int kConvThreads = 256;    // two threads per output position: 16 of a block's 32 k each
+constexpr int kMmaWarp = 8, kTmaWarp = 9;
 constexpr int kTileP = 128;          // output positions per tile
 constexpr int kBK = 32;              // k per converted block
 constexpr uint32_t kACols = 2 * kBK; // heads, then remainders
-constexpr uint32_t kAccCols = 64;
-constexpr uint32_t kTmemCols = 256;  // accumulator + two converted blocks, rounded to a power of two
+constexpr uint32_t kAccCols = 64;    // per accumulator; two of them, so that a tile's epilogue runs under the next tile's MMAs
+constexpr uint32_t kTmemCols = 256;  // two accumulators + two converted blocks
 
 struct Args {
     const float* W;          // first filter of node 0 (inside its parameter row); node stride ld_w
@@ -84,8 +87,11 @@ __device__ __forceinline__ uint32_t lds32u(uint32_t addr) {
 // Shared memory: [patch stages][B heads | B remainders][tap table][barriers].
 __host__ __device__ inline uint32_t b_copy_bytes(int kb, int rows) { return (uint32_t)kb * (kBK / 4) * rows * 16; }
 
-template <int NT>
-__global__ void __launch_bounds__(kThreads, 1)
+// TAPMAJOR (C_in a multiple of 16): the contraction index runs tap-major, k = (kh, kw) C_in + c, so that the 16
+// values a thread gathers per block share one tap: one border predicate, addresses one channel plane apart, no
+// table.  Otherwise k = c 9 + (kh, kw) as the filters lie in memory, through the tap table.
+template <int NT, bool TAPMAJOR>
+__global__ void __launch_bounds__(kThreads, 2)
 conv3x3_fwd_kernel(const __grid_constant__ CUtensorMap mapX, Args g) {
     constexpr int ROWS_B = 16 * NT;                       // output channels of this launch
     constexpr uint32_t B_LBO = (uint32_t)ROWS_B * 16, SBO = 128;
@@ -102,8 +108,8 @@ conv3x3_fwd_kernel(const __grid_constant__ CUtensorMap mapX, Args g) {
     uint64_t* patch_empty = bars + 2;            // [2]
     uint64_t* conv_full = bars + 4;              // [2]
     uint64_t* conv_empty = bars + 6;             // [2]
-    uint64_t* acc_full = bars + 8;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 9);
+    uint64_t* acc_full = bars + 8;               // [2] one per accumulator
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -111,10 +117,10 @@ conv3x3_fwd_kernel(const __grid_constant__ CUtensorMap mapX, Args g) {
             mbar_init(patch_full + s, 1); mbar_init(patch_empty + s, kConvThreads);
             mbar_init(conv_full + s, kConvThreads); mbar_init(conv_empty + s, 1);
         }
-        mbar_init(acc_full, 1);
+        mbar_init(acc_full, 1); mbar_init(acc_full + 1, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 4) {
+    if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -139,23 +145,58 @@ conv3x3_fwd_kernel(const __grid_constant__ CUtensorMap mapX, Args g) {
     const int pos_per_img = g.Ho * g.Wo;
     const int total_pos = g.B * pos_per_img;              // per node
 
-    if (warp < 4) {
+    if (warp < 8) {
         // ------------------------------ converters, then epilogue ------------------------------
-        const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+        // thread = (output position p, half): lane quarter warp % 4 of tensor memory, columns 16 half .. of a block
+        const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+        const uint32_t half = (uint32_t)warp >> 2;
         bool ok = true;
         uint32_t q = 0, done = 0;
         int cur_node = -1;
         // position of this thread inside a tile: image, output row, output column (all local to the tile)
-        const int p = tid;
+        const int p = tid & 127;
         const int img_l = p >> g.log2_img, pin = p & ((1 << g.log2_img) - 1);
         const int i_l = pin >> g.log2_wo, j = pin & (g.Wo - 1);
         const int jj0 = g.stride * j - 1;                                   // input column under tap kw = 0
         const uint32_t base_p = (uint32_t)(((img_l * g.C_in) * g.rows_patch + g.stride * i_l) * g.W_in + g.stride * j);
+
+        // Epilogue of the tile whose MMAs went into accumulator `slot`: bias, ReLU, NCHW store (positions contiguous
+        // across lanes).  It is run one tile late, after the next tile's blocks have been converted, so that the MMAs
+        // it waits for have had that long to finish and the tensor core works on the next tile meanwhile.
+        auto epilogue = [&](int t_done, uint32_t idx) -> bool {
+            const uint32_t slot = idx & 1u;
+            bool fine = mbar_wait(acc_full + slot, (idx >> 1) & 1u);
+            fine = __all_sync(0xffffffffu, fine);                            // tcgen05.ld needs the whole warp
+            if (!fine) return false;
+            tc::tc_fence_after();
+            const int node = t_done / g.tiles_per_node, tile = t_done - node * g.tiles_per_node;
+            const int pg = tile * kTileP + p;                                // position inside the node
+            const bool live = pg < total_pos;
+            const int img = pg / pos_per_img, pin_g = pg - img * pos_per_img;
+            float* yb = g.Y + (((int64_t)node * g.B + img) * g.C_out_total + g.o0) * pos_per_img + pin_g;
+            const float* bn = g.bias ? g.bias + (int64_t)node * g.ld_w + g.o0 : nullptr;
+#pragma unroll 1
+            for (int c0 = 16 * (int)half; c0 < ROWS_B; c0 += 32) {
+                float v[16];
+                tc::tmem_ld16(lane_base + slot * kAccCols + (uint32_t)c0, v);
+#pragma unroll
+                for (int u = 0; u < 16; ++u) {
+                    float x = bn ? v[u] + __ldg(bn + c0 + u) : v[u];
+                    if (g.relu && !(x > 0.f)) x = 0.f;
+                    if (live) yb[(int64_t)(c0 + u) * pos_per_img] = x;
+                }
+            }
+            tc::tc_fence_before();          // these accumulator reads precede the MMAs of the tile after next
+            return true;
+        };
+
+        int pending = -1;                                                    // tile whose epilogue is still owed
         for (int t = t_begin; t < t_end && ok; ++t, ++done) {
-            const int node = t / g.tiles_per_node, tile = t - node * g.tiles_per_node;
+            const int node = t / g.tiles_per_node;
             if (node != cur_node) {
-                // this node's filters for channels [o0, o0 + ROWS_B): every MMA of the previous tile has
-                // completed (its accumulator was drained), so the buffers are free
+                // this node's filters for channels [o0, o0 + ROWS_B): the buffers are free once every MMA of the
+                // previous tile has completed, i.e. once its accumulator is full
+                if (pending >= 0) { ok = epilogue(pending, done - 1); pending = -1; if (!ok) break; }
                 const float* wn = g.W + (int64_t)node * g.ld_w + (int64_t)g.o0 * g.K;
                 const int chunks = g.KB * (kBK / 4);
                 const bool vec = (g.K & 3) == 0 && (reinterpret_cast<uintptr_t>(wn) & 15) == 0;
@@ -164,7 +205,13 @@ conv3x3_fwd_kernel(const __grid_constant__ CUtensorMap mapX, Args g) {
                     const int k = 4 * c;
                     const float* src = wn + (int64_t)o * g.K + k;
                     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (vec) {
+                    if (TAPMAJOR) {
+                        if (k < g.K) {      // four consecutive channels of one tap: nine floats apart in memory
+                            const int tap = k / g.C_in, ch = k - tap * g.C_in;
+                            const float* sp = wn + (int64_t)o * g.K + ch * 9 + tap;
+                            v = make_float4(__ldg(sp), __ldg(sp + 9), __ldg(sp + 18), __ldg(sp + 27));
+                        }
+                    } else if (vec) {
                         if (k < g.K) v = __ldg(reinterpret_cast<const float4*>(src));
                     } else {
                         if (k < g.K) v.x = __ldg(src);
@@ -183,10 +230,22 @@ conv3x3_fwd_kernel(const __grid_constant__ CUtensorMap mapX, Args g) {
                 const uint32_t buf = q & 1u;
                 if (!__all_sync(0xffffffffu, mbar_wait(conv_empty + buf, ((q >> 1) & 1u) ^ 1u))) { ok = false; break; }
                 tc::tc_fence_after();
-                const uint32_t a_cols = lane_base + kAccCols + buf * kACols;
+                const uint32_t a_cols = lane_base + 2 * kAccCols + buf * kACols;
+                uint32_t hi[16], lo[16];
+                if (TAPMAJOR) {
+                    const int k0 = kb * kBK + (int)half * 16;            // 16 consecutive channels of one tap
+                    const int tap = k0 / g.C_in, ch = k0 - tap * g.C_in;
+                    const int kh = (tap * 11) >> 5, kw = tap - 3 * kh;   // tap / 3 for tap < 9
+                    const int jj = jj0 + kw;
+                    const bool in = k0 < g.K && jj >= 0 && jj < g.W_in;
+                    const uint32_t plane = (uint32_t)(g.rows_patch * g.W_in) * 4;
+                    const uint32_t src = patch + (uint32_t)((ch * g.rows_patch + kh) * g.W_in + kw) * 4 - 4;
 #pragma unroll
-                for (uint32_t half = 0; half < 2; ++half) {
-                    uint32_t hi[16], lo[16];
+                    for (int u = 0; u < 16; ++u) {
+                        const float v = in ? lds32(src + (uint32_t)u * plane) : 0.f;
+                        tcs::split(v, hi[u], lo[u]);
+                    }
+                } else {
 #pragma unroll
                     for (int u = 0; u < 16; ++u) {
                         const uint32_t e = lds32u(table + (uint32_t)(kb * kBK + half * 16 + u) * 4);
@@ -197,9 +256,9 @@ conv3x3_fwd_kernel(const __grid_constant__ CUtensorMap mapX, Args g) {
                         const float v = in ? lds32(patch + (e >> 2) * 4 - 4) : 0.f;
                         tcs::split(v, hi[u], lo[u]);
                     }
-                    tcs::tmem_st16(a_cols + 16 * half, hi);
-                    tcs::tmem_st16(a_cols + kBK + 16 * half, lo);
                 }
+                tcs::tmem_st16(a_cols + 16 * half, hi);
+                tcs::tmem_st16(a_cols + kBK + 16 * half, lo);
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 tc::tc_fence_before();
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the filters written above, first block
@@ -207,62 +266,45 @@ conv3x3_fwd_kernel(const __grid_constant__ CUtensorMap mapX, Args g) {
             }
             if (!ok) break;
             mbar_arrive(patch_empty + ps);                                   // the patch has been read
-            if (!mbar_wait(acc_full, done & 1u)) ok = false;
-            ok = __all_sync(0xffffffffu, ok);                                // tcgen05.ld needs the whole warp
-            if (!ok) break;
-            tc::tc_fence_after();
-            // ---- epilogue: bias, ReLU, NCHW store (positions contiguous across lanes) ----
-            const int pos0 = tile * kTileP;                                  // first position of the tile inside the node
-            const int pg = pos0 + p;
-            const bool live = pg < total_pos;
-            const int img = pg / pos_per_img, pin_g = pg - img * pos_per_img;
-            float* yb = g.Y + (((int64_t)node * g.B + img) * g.C_out_total + g.o0) * pos_per_img + pin_g;
-            const float* bn = g.bias ? g.bias + (int64_t)node * g.ld_w + g.o0 : nullptr;
-#pragma unroll 1
-            for (int c0 = 0; c0 < ROWS_B; c0 += 16) {
-                float v[16];
-                tc::tmem_ld16(lane_base + (uint32_t)c0, v);
-#pragma unroll
-                for (int u = 0; u < 16; ++u) {
-                    float x = bn ? v[u] + __ldg(bn + c0 + u) : v[u];
-                    if (g.relu && !(x > 0.f)) x = 0.f;
-                    if (live) yb[(int64_t)(c0 + u) * pos_per_img] = x;
-                }
-            }
-            tc::tc_fence_before();          // the accumulator reads precede the next tile's first MMA
+            if (pending >= 0) ok = epilogue(pending, done - 1);              // the tile before this one
+            pending = t;
         }
+        if (ok && pending >= 0) ok = epilogue(pending, done - 1);
         if (!ok && lane == 0) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
-    } else if (warp == 4) {
+    } else if (warp == kMmaWarp) {
         if (lane == 0) {
             // ------------------------------ MMA issuer ------------------------------
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(ROWS_B >> 3) << 17) |
                                    ((uint32_t)(kTileP >> 4) << 24);
             bool ok = true;
-            uint32_t q = 0;
-            for (int t = t_begin; t < t_end && ok; ++t) {
+            uint32_t q = 0, done = 0;
+            for (int t = t_begin; t < t_end && ok; ++t, ++done) {
                 uint32_t acc = 0;
+                // accumulator done & 1: its previous contents (tile done - 2) were read before the converters wrote
+                // the first block of this tile
+                const uint32_t d_acc = tmem_base + (done & 1u) * kAccCols;
                 for (int kb = 0; kb < g.KB; ++kb, ++q) {
                     const uint32_t buf = q & 1u;
                     if (!mbar_wait(conv_full + buf, (q >> 1) & 1u)) { ok = false; break; }
                     tc::tc_fence_after();
-                    const uint32_t a_hi = tmem_base + kAccCols + buf * kACols, a_lo = a_hi + kBK;
+                    const uint32_t a_hi = tmem_base + 2 * kAccCols + buf * kACols, a_lo = a_hi + kBK;
 #pragma unroll
                     for (uint32_t kk = 0; kk < kBK / 8; ++kk) {
                         if ((int)(kb * kBK + kk * 8) >= g.K) break;          // zero padding only from here on
                         const uint32_t boff = (uint32_t)(kb * (kBK / 8) + kk) * 2 * B_LBO;
                         const uint64_t dbh = tc::smem_desc(b_hi + boff, B_LBO, SBO);
                         const uint64_t dbl = tc::smem_desc(b_lo + boff, B_LBO, SBO);
-                        tcs::mma_tf32_ts(tmem_base, a_lo + kk * 8, dbh, idesc, acc); acc = 1;
-                        tcs::mma_tf32_ts(tmem_base, a_hi + kk * 8, dbl, idesc, acc);
-                        tcs::mma_tf32_ts(tmem_base, a_hi + kk * 8, dbh, idesc, acc);
+                        tcs::mma_tf32_ts(d_acc, a_lo + kk * 8, dbh, idesc, acc); acc = 1;
+                        tcs::mma_tf32_ts(d_acc, a_hi + kk * 8, dbl, idesc, acc);
+                        tcs::mma_tf32_ts(d_acc, a_hi + kk * 8, dbh, idesc, acc);
                     }
                     tc::mma_commit(conv_empty + buf);
                 }
-                if (ok) tc::mma_commit(acc_full);
+                if (ok) tc::mma_commit(acc_full + (done & 1u));
             }
             if (!ok) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
         }
-    } else if (lane == 0) {
+    } else if (warp == kTmaWarp && lane == 0) {
         // ------------------------------ TMA: input patches ------------------------------
         bool ok = true;
         uint32_t done = 0;
@@ -289,16 +331,19 @@ conv3x3_fwd_kernel(const __grid_constant__ CUtensorMap mapX, Args g) {
     }
     tc::tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == kMmaWarp) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 }
 
+template <int NT>
+cudaError_t launch_nt(dpsgd_ctx* c, const CUtensorMap& map, const Args& a, size_t smem);
+
 int ilog2(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
 
-template <int NT>
-cudaError_t launch_nt(dpsgd_ctx* c, const CUtensorMap& map, const Args& a, size_t smem) {
-    auto kernel = conv3x3_fwd_kernel<NT>;
+template <int NT, bool TAPMAJOR>
+cudaError_t launch_nt_k(dpsgd_ctx* c, const CUtensorMap& map, const Args& a, size_t smem) {
+    auto kernel = conv3x3_fwd_kernel<NT, TAPMAJOR>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int sms = 0;
@@ -308,6 +353,11 @@ cudaError_t launch_nt(dpsgd_ctx* c, const CUtensorMap& map, const Args& a, size_
     kernel<<<grid, kThreads, smem, c->stream>>>(map, a);
     c->launches++;
     return cudaGetLastError();
+}
+
+template <int NT>
+cudaError_t launch_nt(dpsgd_ctx* c, const CUtensorMap& map, const Args& a, size_t smem) {
+    return a.C_in % 16 == 0 ? launch_nt_k<NT, true>(c, map, a, smem) : launch_nt_k<NT, false>(c, map, a, smem);
 }
 
 }  // namespace conv

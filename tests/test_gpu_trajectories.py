@@ -369,12 +369,12 @@ def test_config5_mlp_300_iterations_consensus_every_step(topology):
     """MLP 1024-2048-2048-10 (6,316,042 parameters per node), 4096 samples per node, minibatch 64,
     gamma 0.02, T = 300, consensus distance reported by every iteration (dpsgd_step_consensus); the ring
     beside the averaging matrix of C-PSGD.  n = 4 nodes: what the oracle finishes in a few minutes.  The ring
-    run is also followed step by step (flips resolved every 25th iteration) and free-runs a second time on the
+    run is also followed step by step (flips resolved every 50th iteration) and free-runs a second time on the
     exact fp32 FMA kernels (mlp_precision = 2), whose pre-activations are ten times closer to the oracle's."""
     _need(8)
     w = wl.config(4, device="cuda", n=4, topology=topology)
     assert w.iterations == 300 and w.batch == 64 and w.dims == (1024, 2048, 2048, 10)
     ring = topology == "ring"
     modes = {"default": 1, "fp32_fma": (1, 2)} if ring else {"default": 1}
-    run_mlp_trajectory(w, 20254, modes, True, "5-" + topology, explain_every=25, rows_always=True, resync=ring,
+    run_mlp_trajectory(w, 20254, modes, True, "5-" + topology, explain_every=50, rows_always=True, resync=ring,
                        blas_threads=4)
