@@ -198,28 +198,50 @@ conv3x3_fwd_kernel(const __grid_constant__ CUtensorMap mapX, Args g) {
                 // previous tile has completed, i.e. once its accumulator is full
                 if (pending >= 0) { ok = epilogue(pending, done - 1); pending = -1; if (!ok) break; }
                 const float* wn = g.W + (int64_t)node * g.ld_w + (int64_t)g.o0 * g.K;
-                const int chunks = g.KB * (kBK / 4);
                 const bool vec = (g.K & 3) == 0 && (reinterpret_cast<uintptr_t>(wn) & 15) == 0;
-                for (int idx = tid; idx < chunks * ROWS_B; idx += kConvThreads) {
-                    const int o = idx % ROWS_B, c = idx / ROWS_B;            // lanes run along o: conflict-free stores
-                    const int k = 4 * c;
-                    const float* src = wn + (int64_t)o * g.K + k;
-                    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (TAPMAJOR) {
-                        if (k < g.K) {      // four consecutive channels of one tap: nine floats apart in memory
-                            const int tap = k / g.C_in, ch = k - tap * g.C_in;
-                            const float* sp = wn + (int64_t)o * g.K + ch * 9 + tap;
-                            v = make_float4(__ldg(sp), __ldg(sp + 9), __ldg(sp + 18), __ldg(sp + 27));
+                if (TAPMAJOR) {
+                    // read the filters as they lie in memory (o, c, tap: coalesced, all loads of a thread in flight)
+                    // and scatter every value to its tap-major place k = tap C_in + c of the MMA layout
+                    const int quads = g.K >> 2;                              // K = 9 C_in is a multiple of 16
+                    for (int idx = tid; idx < quads * ROWS_B; idx += kConvThreads) {
+                        const int o = idx / quads, m0 = 4 * (idx - o * quads);
+                        const float* src = wn + (int64_t)o * g.K + m0;
+                        float v[4];
+                        if (vec) {
+                            const float4 t = __ldg(reinterpret_cast<const float4*>(src));
+                            v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+                        } else {
+                            v[0] = __ldg(src); v[1] = __ldg(src + 1); v[2] = __ldg(src + 2); v[3] = __ldg(src + 3);
                         }
-                    } else if (vec) {
-                        if (k < g.K) v = __ldg(reinterpret_cast<const float4*>(src));
-                    } else {
-                        if (k < g.K) v.x = __ldg(src);
-                        if (k + 1 < g.K) v.y = __ldg(src + 1);
-                        if (k + 2 < g.K) v.z = __ldg(src + 2);
-                        if (k + 3 < g.K) v.w = __ldg(src + 3);
+                        const uint32_t row = (uint32_t)(o >> 3) * SBO + (uint32_t)(o & 7) * 16;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int m = m0 + e, ch = m / 9, tap = m - 9 * ch;
+                            const uint32_t k = (uint32_t)(tap * g.C_in + ch);
+                            const uint32_t off = (k >> 2) * B_LBO + row + (k & 3u) * 4;
+                            uint32_t hi, lo;
+                            tcs::split(v[e], hi, lo);
+                            asm volatile("st.shared.b32 [%0], %1;" ::"r"(b_hi + off), "r"(hi) : "memory");
+                            asm volatile("st.shared.b32 [%0], %1;" ::"r"(b_lo + off), "r"(lo) : "memory");
+                        }
                     }
-                    tcs::put<true>(b_hi, b_lo, (uint32_t)c * B_LBO + (uint32_t)(o >> 3) * SBO + (uint32_t)(o & 7) * 16, v);
+                } else {
+                    const int chunks = g.KB * (kBK / 4);
+                    for (int idx = tid; idx < chunks * ROWS_B; idx += kConvThreads) {
+                        const int o = idx % ROWS_B, c = idx / ROWS_B;        // lanes run along o: conflict-free stores
+                        const int k = 4 * c;
+                        const float* src = wn + (int64_t)o * g.K + k;
+                        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (vec) {
+                            if (k < g.K) v = __ldg(reinterpret_cast<const float4*>(src));
+                        } else {
+                            if (k < g.K) v.x = __ldg(src);
+                            if (k + 1 < g.K) v.y = __ldg(src + 1);
+                            if (k + 2 < g.K) v.z = __ldg(src + 2);
+                            if (k + 3 < g.K) v.w = __ldg(src + 3);
+                        }
+                        tcs::put<true>(b_hi, b_lo, (uint32_t)c * B_LBO + (uint32_t)(o >> 3) * SBO + (uint32_t)(o & 7) * 16, v);
+                    }
                 }
                 cur_node = node;
             }

@@ -352,6 +352,7 @@ glm_node_step_kernel(const float4* __restrict__ X, float4* __restrict__ G, float
     float4* red = ms + ld4;                                                // [8][32]
     float* scoef = reinterpret_cast<float*>(red + 8 * 32);                 // [B]
     int32_t* sj = reinterpret_cast<int32_t*>(scoef + B);                   // [B]
+    float* sy = reinterpret_cast<float*>(sj + B);                          // [B] targets / labels of the draws
     if (k_ptr) k = *k_ptr;
     if (k_next && node == 0 && tid == 0) *k_next = k + 1;
     const int Bi = node_batch ? __ldg(node_batch + node) : B;
@@ -379,14 +380,16 @@ glm_node_step_kernel(const float4* __restrict__ X, float4* __restrict__ G, float
         rows[e] = b < Bi ? __ldg(reinterpret_cast<const float4*>(A + ((int64_t)node * m + sj[b]) * d) + c)
                          : make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    for (int b = tid; b < B; b += kNodeThreads) sy[b] = __ldg(y + (int64_t)node * m + sj[b]);   // with the rows, not after the dots
     __syncthreads();
     // forward: a warp per draw; lane l of pass w stands for thread 32 w + l of the per-sample CTA
     for (int b = warp; b < B; b += kNodeThreads / 32) {
         float cf = 0.f;
         if (b < Bi) {
             float dot = 0.f;
+            // passes beyond the row's last 16-byte column would add 0.0f to dot, which changes nothing: skipped
 #pragma unroll 1
-            for (int w = 0; w < 8; ++w) {
+            for (int w = 0; w * 32 < d4; ++w) {
                 const int c = w * 32 + lane;
                 float acc = 0.f;
                 if (c < d4) {
@@ -396,7 +399,7 @@ glm_node_step_kernel(const float4* __restrict__ X, float4* __restrict__ G, float
                 }
                 dot += warp_allsum(acc);
             }
-            const float yv = __ldg(y + (int64_t)node * m + sj[b]);
+            const float yv = sy[b];
             if (model == DPSGD_MODEL_LSQ) {
                 cf = (dot - yv) / (float)Bi;
             } else {
@@ -459,7 +462,7 @@ glm_node_step_kernel(const float4* __restrict__ X, float4* __restrict__ G, float
 }
 
 size_t node_step_smem(const dpsgd_ctx* c) {
-    return sizeof(float) * ((size_t)c->batch * c->d + 3 * (size_t)c->ld + 8 * 32 * 4 + 2 * (size_t)c->batch);
+    return sizeof(float) * ((size_t)c->batch * c->d + 3 * (size_t)c->ld + 8 * 32 * 4 + 3 * (size_t)c->batch);
 }
 
 bool rows_path(const dpsgd_ctx* c) {
