@@ -230,8 +230,8 @@ DPSGD_API dpsgd_status dpsgd_step_consensus(dpsgd_ctx* ctx, uint64_t k, double* 
 DPSGD_API dpsgd_status dpsgd_step(dpsgd_ctx* ctx, uint64_t k);
 
 /* The loop of Algorithm 1: iterations k_first, k_first + 1, ... (dpsgd_step each), enqueued in one
- * call.  For launch-bound sizes (linear models, matrices of at most 8 MB, at least 8 iterations) a
- * pair of iterations is captured once into a CUDA graph that reads the iteration number from
+ * call.  For launch-bound sizes (linear models, matrices of at most 8 MB, at least 32 iterations) a
+ * chain of 16 iterations is captured once into a CUDA graph that reads the iteration number from
  * device memory, and replayed; results are identical to repeated dpsgd_step calls.  The bound
  * stream must not be used by other threads during the call. */
 DPSGD_API dpsgd_status dpsgd_run(dpsgd_ctx* ctx, uint64_t k_first, int64_t iterations);

@@ -621,8 +621,10 @@ DPSGD_API dpsgd_status dpsgd_step(dpsgd_ctx* c, uint64_t k) {
     return DPSGD_OK;
 }
 
-// Captures two iterations (the X buffers swap back) that read the iteration number from device
-// memory and advance it, so that one graph can be replayed for any k.
+// Captures kGraphChain iterations (an even number: the X buffers swap back) that read the iteration number from
+// device memory and advance it, so that one graph can be replayed for any k.  A longer chain means fewer graph
+// launches, whose boundaries cost more than the dependency between two kernels inside a graph.
+constexpr int kGraphChain = 16;
 dpsgd_status capture_pair(dpsgd_ctx* c) {
     cudaError_t e = cudaSuccess;
     if (!c->d_k) e = cudaMalloc(&c->d_k, 2 * sizeof(uint64_t));
@@ -637,19 +639,22 @@ dpsgd_status capture_pair(dpsgd_ctx* c) {
     e = cudaStreamBeginCapture(c->capture_stream, cudaStreamCaptureModeThreadLocal);
     if (e != cudaSuccess) return cuda_fail(c, e, "begin capture");
     c->stream = c->capture_stream;
-    // The one-launch step kernel reads the iteration number from one slot and leaves the next number in the
-    // other, so the two captured iterations alternate slots (the replay starts from slot 0) and need no
-    // counter kernel; every other path reads slot 0 and a one-thread kernel advances it.
+    // The one-launch step kernel reads the iteration number from its slot and leaves k + 2 there for the launch
+    // after next; consecutive iterations alternate between the two slots (set to k and k + 1 before the replay),
+    // need no counter kernel and can be programmatic dependents of one another.  Every other path reads slot 0
+    // and a one-thread kernel advances it.
     const bool self = c->fuse_step && linear_node_step_fuses(c);
     dpsgd_status s = DPSGD_OK;
-    for (int t = 0; t < 2 && s == DPSGD_OK; ++t) {
-        c->k_dev_active = c->d_k + (self ? t : 0);
-        c->k_dev_next = self ? c->d_k + (t ^ 1) : nullptr;
+    for (int t = 0; t < kGraphChain && s == DPSGD_OK; ++t) {
+        c->k_dev_active = c->d_k + (self ? (t & 1) : 0);
+        c->k_dev_next = self ? c->d_k + (t & 1) : nullptr;
+        c->chain_pos = t;
         s = dpsgd_step(c, 0);
         if (!self && s == DPSGD_OK && launch_advance_k(c) != cudaSuccess) s = DPSGD_ERR_CUDA;
     }
     c->k_dev_active = nullptr;
     c->k_dev_next = nullptr;
+    c->chain_pos = 0;
     c->stream = bound_stream;
     cudaGraph_t graph = nullptr;
     e = cudaStreamEndCapture(c->capture_stream, &graph);
@@ -673,11 +678,11 @@ DPSGD_API dpsgd_status dpsgd_run(dpsgd_ctx* c, uint64_t k_first, int64_t iterati
     if ((s = need_model(c)) != DPSGD_OK) return s;
     if (iterations < 0) return fail(c, DPSGD_ERR_ARG, "iterations must be >= 0");
     int64_t t = 0;
-    // Launch-bound sizes only: replay a captured pair of iterations.  The first two iterations always
+    // Launch-bound sizes only: replay a captured chain of iterations.  The first two iterations always
     // run directly, which also completes any first-use set-up before a capture starts.
     // (rows of 4 KB and more make the gradient kernels long enough to hide the launches: replay measured
     // slower there, 29 against 24 us per iteration on the 4096-feature logistic configuration)
-    const bool small = mix_is_small(c) && c->model != DPSGD_MODEL_MLP && c->d < 1024 && iterations >= 8;
+    const bool small = mix_is_small(c) && c->model != DPSGD_MODEL_MLP && c->d < 1024 && iterations >= 2 * kGraphChain;
     if (small) {
         for (; t < 2; ++t)
             if ((s = dpsgd_step(c, k_first + (uint64_t)t)) != DPSGD_OK) return s;
@@ -688,7 +693,7 @@ DPSGD_API dpsgd_status dpsgd_run(dpsgd_ctx* c, uint64_t k_first, int64_t iterati
                 ++t;
             }
             cudaError_t e = launch_set_k(c, k_first + (uint64_t)t);
-            for (; e == cudaSuccess && t + 2 <= iterations; t += 2) {
+            for (; e == cudaSuccess && t + kGraphChain <= iterations; t += kGraphChain) {
                 e = cudaGraphLaunch(c->graph_exec, c->stream);
                 c->launches += c->graph_launches;
             }

@@ -50,6 +50,7 @@ using tcs::mbar_expect_tx;
 constexpr int kThreads = 320;        // 8 converter / epilogue warps, MMA warp, TMA warp
 constexpr int kConvThreads = 256;    // two threads per output position: 16 of a block's 32 k each
 constexpr int kMmaWarp = 8, kTmaWarp = 9;
+constexpr int kMaxPatchStages = 4;   // input patches in flight: a TMA copy takes longer than a small tile's work
 constexpr int kTileP = 128;          // output positions per tile
 constexpr int kBK = 32;              // k per converted block
 constexpr uint32_t kACols = 2 * kBK; // heads, then remainders
@@ -104,19 +105,17 @@ conv3x3_fwd_kernel(const __grid_constant__ CUtensorMap mapX, Args g) {
     const uint32_t b_hi = patch0 + S * g.patch_stride, b_lo = b_hi + B_COPY;
     const uint32_t table = b_lo + B_COPY;
     uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + S * g.patch_stride + 2 * B_COPY + (uint32_t)g.KB * kBK * 4);
-    uint64_t* patch_full = bars;                 // [2]
-    uint64_t* patch_empty = bars + 2;            // [2]
-    uint64_t* conv_full = bars + 4;              // [2]
-    uint64_t* conv_empty = bars + 6;             // [2]
-    uint64_t* acc_full = bars + 8;               // [2] one per accumulator
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+    uint64_t* patch_full = bars;                 // [kMaxPatchStages]
+    uint64_t* patch_empty = bars + kMaxPatchStages;
+    uint64_t* conv_full = bars + 2 * kMaxPatchStages;            // [2]
+    uint64_t* conv_empty = conv_full + 2;        // [2]
+    uint64_t* acc_full = conv_full + 4;          // [2] one per accumulator
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(conv_full + 6);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(patch_full + s, 1); mbar_init(patch_empty + s, kConvThreads);
-            mbar_init(conv_full + s, kConvThreads); mbar_init(conv_empty + s, 1);
-        }
+        for (int s = 0; s < kMaxPatchStages; ++s) { mbar_init(patch_full + s, 1); mbar_init(patch_empty + s, kConvThreads); }
+        for (int s = 0; s < 2; ++s) { mbar_init(conv_full + s, kConvThreads); mbar_init(conv_empty + s, 1); }
         mbar_init(acc_full, 1); mbar_init(acc_full + 1, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -456,12 +455,16 @@ cudaError_t launch_conv3x3_forward_on(dpsgd_ctx* c, const float* x, int batch, i
         uint32_t stages = 2;
         for (;;) {
             const size_t fixed = 2 * (size_t)b_copy_bytes(a.KB, rows) + (size_t)a.KB * kBK * 4 + 128 + 256;
-            stages = 2;
-            need = fixed + 2 * (size_t)a.patch_stride;
-            if (need <= budget) break;
-            stages = 1;
-            need = fixed + (size_t)a.patch_stride;
-            if (need <= budget) break;
+            // as many patches in flight (up to four) as leave room for two CTAs per SM when one patch does;
+            // otherwise as many as fit beside the filters with one CTA per SM
+            const size_t two_ctas = (size_t)110 * 1024;
+            const size_t limit = fixed + (size_t)a.patch_stride <= two_ctas ? two_ctas : budget;
+            bool fits = false;
+            for (uint32_t st = kMaxPatchStages; st >= 1 && !fits; --st) {
+                need = fixed + st * (size_t)a.patch_stride;
+                if (need <= limit) { stages = st; fits = true; }
+            }
+            if (fits) break;
             if (rows == 16) { *why = "a tile's input patch and the filters do not fit shared memory"; return cudaErrorNotSupported; }
             rows /= 2;
         }

@@ -102,7 +102,8 @@ struct dpsgd_ctx {
     // graph replay of pairs of iterations (small, launch-bound problems)
     uint64_t* d_k = nullptr;                 // device iteration counter (two slots, see capture_pair)
     const uint64_t* k_dev_active = nullptr;  // non-NULL only while a graph is captured
-    uint64_t* k_dev_next = nullptr;          // capture of a self-advancing step kernel: where it leaves k + 1
+    uint64_t* k_dev_next = nullptr;          // capture of a self-advancing step kernel: the slot it leaves k + 2 in
+    int chain_pos = 0;                       // position of the iteration being captured inside its chain
     cudaGraphExec_t graph_exec = nullptr;
     cudaStream_t capture_stream = nullptr;   // private stream the pair is recorded on
     int graph_cur = 0;                       // value of `cur` the graph was captured at

@@ -330,8 +330,12 @@ glm_rows_reduce_mix_kernel(const float4* __restrict__ X, float4* __restrict__ G,
 // waits for another.  Every reduction runs in the order of glm_forward_kernel / glm_backward_kernel /
 // mix_rowpar_kernel (lanes of a 32-wide xor tree, warps in order, eight interleaved slices of the minibatch
 // in order), so the result is bit-identical to the three-launch path.
-// With k_next != NULL the kernel reads the iteration number from *k_ptr and leaves k + 1 in *k_next (two
-// slots used alternately by consecutive launches: a replayed graph needs no counter kernel in between).
+// Replayed graphs: with k_next != NULL the kernel reads the iteration number from *k_ptr and leaves k + 2 there
+// for the launch after next (two slots used alternately by consecutive launches, so no counter kernel runs in
+// between and a launch never reads a slot its predecessor writes).  That, and the fact that everything before
+// griddepcontrol.wait reads only the dataset (never written by this library), lets consecutive launches of a
+// captured chain be programmatic dependents: launch t + 1 draws its indices and gathers its rows while launch
+// t is still computing, and touches X, G and the index buffer only after launch t has completed.
 constexpr int kNodeThreads = 256;
 
 __global__ void __launch_bounds__(kNodeThreads)
@@ -353,14 +357,21 @@ glm_node_step_kernel(const float4* __restrict__ X, float4* __restrict__ G, float
     float* scoef = reinterpret_cast<float*>(red + 8 * 32);                 // [B]
     int32_t* sj = reinterpret_cast<int32_t*>(scoef + B);                   // [B]
     float* sy = reinterpret_cast<float*>(sj + B);                          // [B] targets / labels of the draws
-    if (k_ptr) k = *k_ptr;
-    if (k_next && node == 0 && tid == 0) *k_next = k + 1;
+    if (k_ptr) k = *k_ptr;                 // written two launches ago: complete before this launch could start
     const int Bi = node_batch ? __ldg(node_batch + node) : B;
-    for (int b = tid; b < B; b += kNodeThreads) {
-        const int32_t j = sample_index(seed, k, (uint32_t)node, (uint32_t)b, (uint32_t)m);
-        sj[b] = j;
-        idx[node * B + b] = j;
+    for (int b = tid; b < B; b += kNodeThreads) sj[b] = sample_index(seed, k, (uint32_t)node, (uint32_t)b, (uint32_t)m);
+    __syncthreads();
+    for (int e = tid; e < B * d4; e += kNodeThreads) {
+        const int b = e / d4, c = e - b * d4;
+        rows[e] = b < Bi ? __ldg(reinterpret_cast<const float4*>(A + ((int64_t)node * m + sj[b]) * d) + c)
+                         : make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    for (int b = tid; b < B; b += kNodeThreads) sy[b] = __ldg(y + (int64_t)node * m + sj[b]);   // with the rows, not after the dots
+    // ---- everything above read the dataset only; from here on X, G and the scratch of the previous launch ----
+    asm volatile("griddepcontrol.wait;" ::: "memory");              // no-op unless launched as a programmatic dependent
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); // the next launch may begin its own gathers
+    if (k_next && node == 0 && tid == 0) *k_next = k + 2;
+    for (int b = tid; b < B; b += kNodeThreads) idx[node * B + b] = sj[b];
     const int p0 = __ldg(row_ptr + node), pe = __ldg(row_ptr + node + 1);
     for (int64_t c = tid; c < ld4; c += kNodeThreads) {
         xs[c] = __ldg(X + (int64_t)node * ld4 + c);
@@ -374,13 +385,6 @@ glm_node_step_kernel(const float4* __restrict__ X, float4* __restrict__ G, float
         }
         ms[c] = a;
     }
-    __syncthreads();
-    for (int e = tid; e < B * d4; e += kNodeThreads) {
-        const int b = e / d4, c = e - b * d4;
-        rows[e] = b < Bi ? __ldg(reinterpret_cast<const float4*>(A + ((int64_t)node * m + sj[b]) * d) + c)
-                         : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    for (int b = tid; b < B; b += kNodeThreads) sy[b] = __ldg(y + (int64_t)node * m + sj[b]);   // with the rows, not after the dots
     __syncthreads();
     // forward: a warp per draw; lane l of pass w stands for thread 32 w + l of the per-sample CTA
     for (int b = warp; b < B; b += kNodeThreads / 32) {
@@ -512,12 +516,20 @@ cudaError_t launch_linear_step(dpsgd_ctx* c, uint64_t k, const float* X, float* 
         const size_t smem = node_step_smem(c);
         cudaError_t e = cudaFuncSetAttribute(glm_node_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        glm_node_step_kernel<<<c->n, kNodeThreads, smem, c->stream>>>(
-            reinterpret_cast<const float4*>(X), reinterpret_cast<float4*>(G), reinterpret_cast<float4*>(Xn), c->ld, c->A,
-            static_cast<const float*>(c->y), c->m, c->d, c->batch, c->seed, k, c->k_dev_active, c->k_dev_next, c->model,
-            c->l2, c->d_idx, c->d_coef, c->d_node_batch, c->W.row_ptr, c->W.col, c->W.val, -c->gamma);
+        // inside a captured chain (k_dev_next set) every launch after the first is a programmatic dependent of the one before
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)c->n); cfg.blockDim = dim3(kNodeThreads); cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = (c->k_dev_next && c->chain_pos > 0) ? 1 : 0;
+        e = cudaLaunchKernelEx(&cfg, glm_node_step_kernel, reinterpret_cast<const float4*>(X), reinterpret_cast<float4*>(G),
+                               reinterpret_cast<float4*>(Xn), c->ld, c->A, static_cast<const float*>(c->y), c->m, c->d,
+                               c->batch, c->seed, k, c->k_dev_active, c->k_dev_next, c->model, c->l2, c->d_idx, c->d_coef,
+                               (const int32_t*)c->d_node_batch, c->W.row_ptr, c->W.col, c->W.val, -c->gamma);
         c->launches++;
-        return cudaGetLastError();
+        return e != cudaSuccess ? e : cudaGetLastError();
     }
     int groups = 0;
     cudaError_t e = launch_rows(c, k, X, &groups);

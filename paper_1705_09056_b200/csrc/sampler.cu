@@ -12,7 +12,7 @@ __global__ void sample_kernel(uint64_t seed, uint64_t k, int n, int B, uint32_t 
     idx[t] = sample_index(seed, k, (uint32_t)node, (uint32_t)b, m);
 }
 
-__global__ void set_k_kernel(uint64_t* k, uint64_t v) { *k = v; }
+__global__ void set_k_kernel(uint64_t* k, uint64_t v) { k[0] = v; k[1] = v + 1; }   // the two slots of a replayed chain
 __global__ void advance_k_kernel(uint64_t* k) { *k += 1; }
 
 }  // namespace

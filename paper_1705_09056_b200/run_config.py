@@ -98,9 +98,26 @@ def conv_layers(args, dev):
         moved = 4 * (acts[l].numel() + acts[l + 1].numel())
         per_layer.append({"layer": [cin, cout, stride], "ms": ms, "fp32_equivalent_TFLOPs": flops / ms / 1e9,
                           "GBps": moved / ms / 1e6})
+    out = {"workload": "conv3x3 forward, CIFAR-shaped layers", "n": n, "batch": args.batch,
+           "ms_per_forward": sum(p["ms"] for p in per_layer), "layers": per_layer}
+    if args.backward:
+        # filter, bias and input gradients of every layer from a random gradient at its output (layer 1: no input gradient)
+        for l, (cin, cout, stride) in enumerate(w.plan):
+            dy = torch.randn_like(acts[l + 1])
+            run = lambda: ctx.conv3x3_backward(acts[l], acts[l + 1], dy, stride, offs[l][0], offs[l][1], True, cin % 16 == 0)
+            for _ in range(args.warmup):
+                run()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(args.steps):
+                run()
+            b.record()
+            torch.cuda.synchronize()
+            per_layer[l]["ms_backward"] = a.elapsed_time(b) / args.steps
+        out["ms_per_backward"] = sum(p["ms_backward"] for p in per_layer)
     ctx.sync()
-    print(json.dumps({"workload": "conv3x3 forward, CIFAR-shaped layers", "n": n, "batch": args.batch,
-                      "ms_per_forward": sum(p["ms"] for p in per_layer), "layers": per_layer}))
+    print(json.dumps(out))
     ctx.close()
 
 
@@ -114,6 +131,7 @@ def main():
     ap.add_argument("--kind", type=int, default=-1, help="config 3: force a DPSGD_MIX_* kernel")
     ap.add_argument("--conv", action="store_true", help="time the convolution layer family instead of a configuration")
     ap.add_argument("--batch", type=int, default=32, help="--conv: images per node")
+    ap.add_argument("--backward", action="store_true", help="--conv: also time the backward of every layer")
     ap.add_argument("--momentum", type=float, default=0.0,
                     help="config 3: momentum of the Section 5.3 runs (one more matrix)")
     ap.add_argument("--m", type=int, default=0, help="override the local dataset size")

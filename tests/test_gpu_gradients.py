@@ -195,19 +195,19 @@ def test_run_equals_repeated_steps():
     X0 = np.zeros((w.n, w.N), dtype=np.float32)
     a = GpuRun(w.n, w.N, w.csr(), w.gamma, seed=5, X=X0)
     _attach(a, w, A, y)
-    for k in range(3, 33):
+    for k in range(3, 63):
         a.ctx.step(k)
     b = GpuRun(w.n, w.N, w.csr(), w.gamma, seed=5, X=X0)
     _attach(b, w, A, y)
-    b.ctx.run(3, 30)
+    b.ctx.run(3, 60)
     assert np.array_equal(a.x(), b.x())
     a.close(); b.close()
 
 
 @pytest.mark.parametrize("model", [binding.MODEL_LSQ, binding.MODEL_LOGISTIC])
 def test_graph_replayed_run_is_bit_identical_to_steps(model):
-    """dpsgd_run replays a captured pair of iterations for small problems; odd counts, several
-    calls in a row and a change of gamma in between must all equal plain stepping."""
+    """dpsgd_run replays a captured chain of 16 iterations for small problems (runs of at least 32); short
+    and odd counts, several calls in a row and a change of gamma in between must all equal plain stepping."""
     w = _linear_workload(model, 8, 64, 256, 16)
     A, y = w.A.numpy(), w.y.numpy()
     X0 = np.zeros((w.n, w.N), dtype=np.float32)
@@ -216,7 +216,8 @@ def test_graph_replayed_run_is_bit_identical_to_steps(model):
     b = GpuRun(w.n, w.N, w.csr(), w.gamma, seed=5, X=X0)
     _attach(b, w, A, y)
     k = 0
-    for count, gamma in ((9, w.gamma), (20, w.gamma), (3, w.gamma), (31, 0.5 * w.gamma), (8, 0.5 * w.gamma)):
+    for count, gamma in ((9, w.gamma), (40, w.gamma), (3, w.gamma), (71, 0.5 * w.gamma), (33, 0.5 * w.gamma),
+                         (32, w.gamma)):
         a.ctx.set_gamma(gamma); b.ctx.set_gamma(gamma)
         for t in range(count):
             a.ctx.step(k + t)
@@ -224,11 +225,11 @@ def test_graph_replayed_run_is_bit_identical_to_steps(model):
         k += count
         assert np.array_equal(a.x(), b.x()), (count, gamma)
     o = orc.Oracle(w.n, w.N, *w.csr(), w.gamma, 5, w.model, w.dims, w.batch, w.l2_lambda, A, y)
-    for t in range(29):
+    for t in range(53):
         o.step(t)
     c = GpuRun(w.n, w.N, w.csr(), w.gamma, seed=5, X=X0)
     _attach(c, w, A, y)
-    c.ctx.run(0, 29)
+    c.ctx.run(0, 53)
     assert row_rel_err(c.x(), o.X) <= TOL_TRAJ
     a.close(); b.close(); c.close()
 
