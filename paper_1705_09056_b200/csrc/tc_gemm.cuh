@@ -33,7 +33,7 @@ constexpr int kTileM = 128;
 constexpr int kBlockK = 64;            // fp32 elements per pipeline stage along k (8 MMAs of K = 8)
 constexpr int kChunks = kBlockK / 4;   // 16-byte chunk columns per stage
 constexpr int kStages = 1;            // one stage per CTA: four CTAs share an SM and overlap each other
-constexpr uint32_t kWaitSpins = 1u << 21;
+constexpr uint32_t kWaitSpins = 1u << 20;
 
 enum { EPI_BIAS_RELU = 0, EPI_BIAS = 1, EPI_STORE = 2, EPI_MASK = 3 };
 
@@ -57,22 +57,24 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// One poll of a phase.  The suspend-time hint lets the hardware park the thread until the phase completes (it is
+// woken at once) or the hint runs out, instead of returning after its short default slice: a thread that polls
+// in a tight loop keeps its SM partition's shared-memory queue busy, and the warps that share the partition
+// with a waiting single-thread role (MMA issuer, TMA issuer) then convert at half speed.
+constexpr uint32_t kSuspendNs = 2000;
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendNs) : "memory");
     return ok != 0;
 }
+// Bounded wait: kWaitSpins polls of at most kSuspendNs each (about two seconds), then false.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-    // try_wait itself blocks for a short hardware-defined slice, so plain polling is cheap; back
-    // off with nanosleep (coarse: it can cost a microsecond) only once the wait is clearly long
-    for (uint32_t spin = 0; spin < kWaitSpins; ++spin) {
+    for (uint32_t spin = 0; spin < kWaitSpins; ++spin)
         if (mbar_try_wait(bar, parity)) return true;
-        if (spin > 4096) __nanosleep(128);
-    }
     return false;
 }
 

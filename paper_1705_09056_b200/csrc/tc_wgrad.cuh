@@ -32,9 +32,11 @@
 //           take a staged tile, read the same tile of X from the node's neighbours with 128-bit loads
 //           (all but the first read of an element come from L2; the next node's tiles are prefetched
 //           into L2 one item ahead) and write X_next.  Two column tiles per item.
-//   kRing   (Theorem 3's ring): no epilogue warps and no staging; sixteen mixer warps read the
-//           accumulator in its own layout and keep the tiles of X_{i-1} and X_i in tensor memory, so
-//           X is read from memory once.  One column tile per item (the window holds one position).
+//   kRing   (Theorem 3's ring): no epilogue warps and no staging of the output; sixteen mixer warps read
+//           the accumulator in its own layout and keep the tiles of X_{i-1} and X_i in tensor memory, so
+//           X is read from memory once: the tile of X_{i+1}, which the TMA thread fetches one to two
+//           nodes ahead into two shared-memory stages (no mixer thread waits on HBM, no registers
+//           hold loads in flight).  One column tile per item (the window holds one position).
 //
 // One persistent CTA per SM; a work item is (node, 128-row block of m, run of column tiles).  Every
 // mbarrier wait is bounded; a wait that runs out raises the status word, the TMA thread waits
@@ -62,6 +64,7 @@ enum { kStore = 0, kGather = 1, kRing = 2 };
 constexpr int kTileM = 128;
 constexpr int kMaxK = 64;            // minibatch rows a raw tile holds
 constexpr int kStagesB = 3;
+constexpr int kStagesBRing = 2;      // kRing: one delta tile per item, and shared memory also holds two tiles of X
 constexpr uint32_t kAccStride = 64;  // TMEM columns per accumulator
 constexpr uint32_t kACols = 2 * kMaxK;   // heads, then remainders
 constexpr uint32_t A_COL0_ = 2 * kAccStride;   // first tensor-memory column of the converted h tiles
@@ -101,12 +104,12 @@ __host__ __device__ constexpr uint32_t b_lbo(int rows) { return (uint32_t)rows *
 __host__ __device__ constexpr uint32_t b_conv_bytes(int rows) { return (kMaxK / 4) * b_lbo(rows); }
 __host__ __device__ constexpr uint32_t stage_bytes(int rows) { return (uint32_t)rows * kTileM * 4; }
 
-// STAGED: two staging buffers for the output tile and one raw h tile; otherwise (kRing) no staging
-// and two raw h tiles.
+// STAGED: two staging buffers for the output tile and one raw h tile; otherwise (kRing) two raw h
+// tiles and two stages for the tile of X_{i+1}.
 template <int NT, bool PRECISE, bool STAGED = true>
 constexpr size_t smem_bytes() {
-    return 1024 + (STAGED ? 1 : 2) * a_raw_bytes() + kStagesB * b_raw_bytes(16 * NT) + 2 * (PRECISE ? 2 : 1) * b_conv_bytes(16 * NT) +
-           (STAGED ? 2 * stage_bytes(16 * NT) : 0) + 256;
+    return 1024 + (STAGED ? 1 : 2) * a_raw_bytes() + (STAGED ? kStagesB : kStagesBRing) * b_raw_bytes(16 * NT) +
+           2 * (PRECISE ? 2 : 1) * b_conv_bytes(16 * NT) + 2 * stage_bytes(16 * NT) + 256;
 }
 
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
@@ -191,31 +194,41 @@ __device__ __forceinline__ void mix_rows(const Mix& mx, int node, uint32_t st, i
     }
 }
 
-struct Item { int node, m0, t0, t1; };      // node < 0: past the end of a short last node range
-// Items this CTA walks (including the empty ones of a short last node range).
-__device__ __forceinline__ int cta_items(const Args& g) {
-    const int b = (int)blockIdx.x, grid = (int)gridDim.x;
-    return b < g.total_seqs ? ((g.total_seqs - b + grid - 1) / grid) * g.split_len : 0;
-}
-// The i-th item of this CTA.
-__device__ __forceinline__ Item cta_item(const Args& g, int i) {
-    const int round = i / g.split_len, j = i - round * g.split_len;
-    const int seq = (int)blockIdx.x + round * (int)gridDim.x;
-    const int per_split = g.m_tiles * g.chunks;
-    const int sp = seq / per_split, rem = seq - sp * per_split;
-    const int mt = rem / g.chunks, ch = rem - mt * g.chunks;
-    Item w;
-    w.node = sp * g.split_len + j;
-    if (w.node >= g.nodes) w.node = -1;
-    w.m0 = mt * kTileM;
-    w.t0 = ch * g.chunk;
-    w.t1 = min(g.n_tiles, w.t0 + g.chunk);
-    return w;
-}
+// The work items of this CTA in order.  The position (row block, run of column tiles, node range) is decoded
+// once per node range; inside a range the walk only counts nodes up, so that the per-item cost on the threads
+// that sit on the critical path (TMA, converters, MMA issuer) is an increment, not a chain of integer divisions.
+struct Walk {
+    int node, n1, m0, t0, t1;        // the current item: node, first row, column tiles [t0, t1)
+    int rd, rounds;
+    __device__ __forceinline__ explicit Walk(const Args& g) : node(0), n1(0), m0(0), t0(0), t1(0), rd(-1) {
+        const int b = (int)blockIdx.x, grid = (int)gridDim.x;
+        rounds = b < g.total_seqs ? (g.total_seqs - b + grid - 1) / grid : 0;
+    }
+    // Advances to the next item; false after the last one.
+    __device__ __forceinline__ bool next(const Args& g) {
+        if (++node < n1) return true;
+        while (++rd < rounds) {
+            const int seq = (int)blockIdx.x + rd * (int)gridDim.x;
+            const int per_split = g.m_tiles * g.chunks;
+            const int sp = seq / per_split, rem = seq - sp * per_split;
+            const int mt = rem / g.chunks, ch = rem - mt * g.chunks;
+            node = sp * g.split_len;
+            n1 = min(g.nodes, node + g.split_len);
+            m0 = mt * kTileM;
+            t0 = ch * g.chunk;
+            t1 = min(g.n_tiles, t0 + g.chunk);
+            if (node < n1) return true;
+        }
+        return false;
+    }
+    // The node of the next item when it belongs to the same range, else -1.
+    __device__ __forceinline__ int next_in_range() const { return node + 1 < n1 ? node + 1 : -1; }
+};
 
 // NT = column tile / 16 (16, 32 or 64 output units per tile); PRECISE: three split MMAs per product.
-// mapA: h as (m, k, node), box 128 x 64.  mapB: delta as (n, k, node), box 16 NT x 64.  mapC: the
-// gradient block as (m, n, node), box 128 x 16 NT (kStore only).
+// mapA: h as (m, k, node), box 128 x 64.  mapB: delta as (n, k, node), box 16 NT x 64.  mapC: as
+// (m, n, node) with box 128 x 16 NT, the gradient block (kStore, written) or this weight block of X
+// (kRing, read).
 //
 // Tensor memory columns: [0, 128) two accumulators, then two converted h tiles of 64 heads +
 // 64 remainders each.
@@ -231,7 +244,8 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     constexpr uint32_t NCOPY = PRECISE ? 2 : 1;
     constexpr uint32_t CONV_BUF = NCOPY * B_CONV;
     constexpr bool FUSE = MODE == kGather;            // staged tiles go to the mixer warps instead of a TMA store
-    constexpr uint32_t STAGE = MODE == kRing ? 0u : stage_bytes(ROWS_B);
+    constexpr uint32_t STAGE = stage_bytes(ROWS_B);     // kStore, kGather: output staging; kRing: the tile of X_{i+1}
+    constexpr int SB = MODE == kRing ? kStagesBRing : kStagesB;
     constexpr uint32_t WIN_COL0 = A_COL0_ + 2 * kACols;      // kRing: two 64-column slots of the X window
     constexpr uint32_t A_COL0 = A_COL0_;
     constexpr uint32_t TMEM_COLS = 512;
@@ -241,9 +255,9 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     constexpr uint32_t A_BUFS = MODE == kRing ? 2u : 1u;     // raw h tiles in flight (a new one every column tile in kRing)
     const uint32_t a_raw = base;
     const uint32_t b_raw = a_raw + A_BUFS * A_RAW;
-    const uint32_t b_conv = b_raw + kStagesB * B_RAW;
+    const uint32_t b_conv = b_raw + SB * B_RAW;
     const uint32_t stage = b_conv + 2 * CONV_BUF;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + A_BUFS * A_RAW + kStagesB * B_RAW + 2 * CONV_BUF + 2 * STAGE);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + A_BUFS * A_RAW + SB * B_RAW + 2 * CONV_BUF + 2 * STAGE);
     uint64_t* a_raw_full = bars;                 // [A_BUFS]
     uint64_t* a_raw_empty = bars + 2;            // [A_BUFS]
     uint64_t* a_conv_full = bars + 4;            // [2]
@@ -254,8 +268,8 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     uint64_t* b_conv_empty = b_conv_full + 2;    // [2]
     uint64_t* acc_full = b_conv_empty + 2;       // [2]
     uint64_t* acc_empty = acc_full + 2;          // [2]
-    uint64_t* stage_free = acc_empty + 2;        // [2] the TMA store that last read the buffer is done reading
-    uint64_t* stage_ready = stage_free + 2;      // [2] all epilogue threads have written the buffer
+    uint64_t* stage_free = acc_empty + 2;        // [2] the TMA store that last read the buffer is done reading (kRing: the mixers are)
+    uint64_t* stage_ready = stage_free + 2;      // [2] all epilogue threads have written the buffer (kRing: the tile of X has landed)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(stage_ready + 2);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -267,9 +281,9 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             mbar_init(a_conv_full + b, 128); mbar_init(a_conv_empty + b, 1);
             mbar_init(b_conv_full + b, 128); mbar_init(b_conv_empty + b, 1);
             mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, MODE == kRing ? 16 : 128);
-            mbar_init(stage_free + b, FUSE ? 32 * kMixWarps : 1); mbar_init(stage_ready + b, 128);
+            mbar_init(stage_free + b, MODE == kStore ? 1 : 32 * kMixWarps); mbar_init(stage_ready + b, MODE == kRing ? 1 : 128);
         }
-        for (int s = 0; s < kStagesB; ++s) { mbar_init(b_raw_full + s, 1); mbar_init(b_raw_empty + s, 128); }
+        for (int s = 0; s < SB; ++s) { mbar_init(b_raw_full + s, 1); mbar_init(b_raw_empty + s, 128); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 8) {
@@ -281,16 +295,13 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const int my_items = cta_items(g);
     bool ok = true;
 
     if (MODE != kRing && warp < 4) {
         // ------------------------------ epilogue: TMEM -> shared memory -> TMA store ------------------------------
         const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
         uint32_t q = 0;
-        for (int i = 0; i < my_items && ok; ++i) {
-            const Item w = cta_item(g, i);
-            if (w.node < 0) continue;
+        for (Walk w(g); ok && w.next(g);) {
             for (int t = w.t0; t < w.t1; ++t, ++q) {
                 const uint32_t ab = q & 1u, ph = (q >> 1) & 1u;
                 const uint32_t st = stage + ab * STAGE;
@@ -334,9 +345,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         const uint32_t ct = (uint32_t)tid - 128u, cw = (uint32_t)warp - 4u;
         const uint32_t lane_base = tmem_base + ((cw * 32u) << 16);
         uint32_t q = 0, it = 0;
-        for (int i = 0; i < my_items && ok; ++i) {
-            const Item w = cta_item(g, i);
-            if (w.node < 0) continue;
+        for (Walk w(g); ok && w.next(g);) {
             const uint32_t abuf = it & 1u;
             {   // h tile -> tensor memory: row ct of A is column ct of the raw [k][m] tile
                 const uint32_t rbuf = it % A_BUFS, a_tile = a_raw + rbuf * A_RAW;
@@ -363,8 +372,8 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 mbar_arrive(a_raw_empty + rbuf);
             }
             for (int t = w.t0; t < w.t1; ++t, ++q) {
-                const uint32_t s = q % kStagesB, bb = q & 1u;
-                if (!mbar_wait(b_raw_full + s, (q / kStagesB) & 1u) || !mbar_wait(b_conv_empty + bb, ((q >> 1) & 1u) ^ 1u)) {
+                const uint32_t s = q % SB, bb = q & 1u;
+                if (!mbar_wait(b_raw_full + s, (q / SB) & 1u) || !mbar_wait(b_conv_empty + bb, ((q >> 1) & 1u) ^ 1u)) {
                     ok = false;
                     break;
                 }
@@ -393,9 +402,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(ROWS_B >> 3) << 17) |
                                    ((uint32_t)(kTileM >> 4) << 24);
             uint32_t q = 0, it = 0;
-            for (int i = 0; i < my_items && ok; ++i) {
-                const Item w = cta_item(g, i);
-                if (w.node < 0) continue;
+            for (Walk w(g); ok && w.next(g);) {
                 const uint32_t abuf = it & 1u;
                 if (!mbar_wait(a_conv_full + abuf, (it >> 1) & 1u)) { ok = false; break; }
                 const uint32_t a_hi = tmem_base + A_COL0 + abuf * kACols, a_lo = a_hi + kMaxK;
@@ -425,20 +432,28 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         }
     } else if (warp == 9 && lane == 0) {
         // ------------------------------ TMA loads ------------------------------
-        uint32_t q = 0, it = 0;                  // delta tiles and h tiles issued so far
-        for (int i = 0; i < my_items && ok; ++i) {
-            const Item w = cta_item(g, i);
-            if (w.node < 0) continue;
+        uint32_t q = 0, it = 0, xq = 0;          // delta tiles, h tiles and tiles of X issued so far
+        for (Walk w(g); ok && w.next(g);) {
             const uint32_t rbuf = it % A_BUFS;
             if (!mbar_wait(a_raw_empty + rbuf, ((it / A_BUFS) & 1u) ^ 1u)) { ok = false; break; }
             mbar_expect_tx(a_raw_full + rbuf, A_RAW);
             tma_load_3d(a_raw + rbuf * A_RAW, &mapA, w.m0, 0, w.node, a_raw_full + rbuf);
             ++it;
             for (int t = w.t0; t < w.t1; ++t, ++q) {
-                const uint32_t s = q % kStagesB;
-                if (!mbar_wait(b_raw_empty + s, ((q / kStagesB) & 1u) ^ 1u)) { ok = false; break; }
+                const uint32_t s = q % SB;
+                if (!mbar_wait(b_raw_empty + s, ((q / SB) & 1u) ^ 1u)) { ok = false; break; }
                 mbar_expect_tx(b_raw_full + s, B_RAW);
                 tma_load_3d(b_raw + s * B_RAW, &mapB, t * ROWS_B, 0, w.node, b_raw_full + s);
+            }
+            if (MODE == kRing) {
+                // the tile of X_{node+1}: the one tile of X this node step reads from memory; after the loads the
+                // converters wait for, so that its gate (the mixers, two nodes back) never holds those up
+                const uint32_t xs = xq & 1u;
+                if (!ok || !mbar_wait(stage_free + xs, ((xq >> 1) & 1u) ^ 1u)) { ok = false; break; }
+                mbar_expect_tx(stage_ready + xs, STAGE);
+                tma_load_3d(stage + xs * STAGE, &mapC, w.m0, w.t0 * ROWS_B, w.node + 1 == g.nodes ? 0 : w.node + 1,
+                            stage_ready + xs);
+                ++xq;
             }
         }
         // loads still in flight (only when somebody gave up): let them land before the CTA leaves
@@ -446,9 +461,13 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             const uint32_t ii = it - 1 - j;
             mbar_wait(a_raw_full + ii % A_BUFS, (ii / A_BUFS) & 1u);
         }
-        for (uint32_t j = 0; j < (uint32_t)kStagesB && j < q; ++j) {
+        for (uint32_t j = 0; j < (uint32_t)SB && j < q; ++j) {
             const uint32_t qq = q - 1 - j;
-            mbar_wait(b_raw_full + qq % kStagesB, (qq / kStagesB) & 1u);
+            mbar_wait(b_raw_full + qq % SB, (qq / SB) & 1u);
+        }
+        for (uint32_t j = 0; MODE == kRing && j < 2u && j < xq; ++j) {
+            const uint32_t qq = xq - 1 - j;
+            mbar_wait(stage_ready + (qq & 1u), (qq >> 1) & 1u);
         }
         if (!ok) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
     }
@@ -466,6 +485,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const uint32_t win[2] = {lane_addr + WIN_COL0 + (uint32_t)cg * 16, lane_addr + WIN_COL0 + 64 + (uint32_t)cg * 16};
         const int64_t cstride = g.M;                         // one output unit further = din elements further
+        const uint32_t xt_off = (uint32_t)(cg * 16) * (kTileM * 4) + (uint32_t)m * 4;   // this thread's corner of a staged tile of X
         auto load16 = [&](const float* p, int ncols, float (&v)[16]) {
             if (ncols == 16) {
 #pragma unroll
@@ -475,12 +495,13 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 for (int j = 0; j < 16; ++j) v[j] = j < ncols ? __ldcg(p + j * cstride) : 0.f;
             }
         };
-        const int rounds = my_items / g.split_len;
+        const int b = (int)blockIdx.x, grid = (int)gridDim.x;
+        const int rounds = b < g.total_seqs ? (g.total_seqs - b + grid - 1) / grid : 0;
         const int per_split = g.m_tiles * g.chunks;
         uint32_t q = 0;
         for (int rd = 0; rd < rounds && ok; ++rd) {
-            // one node range at one tile position (decoded as in cta_item; chunk == 1: one column tile)
-            const int seq = (int)blockIdx.x + rd * (int)gridDim.x;
+            // one node range at one tile position (decoded as in Walk; chunk == 1: one column tile)
+            const int seq = b + rd * grid;
             const int sp = seq / per_split, rem = seq - sp * per_split;
             const int mt = rem / g.chunks, t = rem - mt * g.chunks;
             const int n0 = sp * g.split_len, n1 = min(g.nodes, n0 + g.split_len);
@@ -496,17 +517,20 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 float xr[16], tmp[16];
                 uint32_t bits[16];
                 const uint32_t jj = (uint32_t)(node - n0);
-                // X_{i+1}: the one tile read from memory; it was requested into L2 two nodes ago
-                load16(xpos + (int64_t)(node + 1 == g.nodes ? 0 : node + 1) * g.mix.ld, ncols, xr);
-                if (node + 2 < n1 && lane < ncols) {
-                    // lane j asks for the line that holds column j of the tile of X_{i+3} (this warp's 32 rows)
-                    const int ahead = node + 3 >= g.nodes ? node + 3 - g.nodes : node + 3;
-                    prefetch_l2(xpos - lane + (int64_t)ahead * g.mix.ld + lane * cstride);
+                // X_{i+1}: the one tile read from memory, staged by the TMA thread (zero outside the block)
+                {
+                    const uint32_t xs = q & 1u;
+                    const bool landed = mbar_wait(stage_ready + xs, (q >> 1) & 1u);
+                    if (!__all_sync(0xffffffffu, landed)) { ok = false; break; }
+                    const uint32_t xt = stage + xs * STAGE + xt_off;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) xr[j] = lds32(xt + (uint32_t)j * (kTileM * 4));
                 }
                 if (cold) load16(xpos + (int64_t)(node == 0 ? g.nodes - 1 : node - 1) * g.mix.ld, ncols, tmp);
                 else tc::tmem_ld16(win[(jj - 1) & 1u], tmp);                     // X_{i-1}
 #pragma unroll
                 for (int j = 0; j < 16; ++j) bits[j] = __float_as_uint(xr[j]);
+                mbar_arrive(stage_free + (q & 1u));                              // this thread's part of the stage is in registers
                 tcs::tmem_st16(cold ? win[1] : win[(jj - 1) & 1u], bits);        // X_{i+1} takes its place
 #pragma unroll
                 for (int j = 0; j < 16; ++j) xr[j] = fmaf(wr, xr[j], wl * tmp[j]);   // accumulated in place
@@ -546,11 +570,9 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         // ------------------------------ mixers: gossip step on staged tiles ------------------------------
         const int mw = warp - 10;
         uint32_t q = 0;
-        for (int i = 0; i < my_items && ok; ++i) {
-            const Item w = cta_item(g, i);
-            if (w.node < 0) continue;
+        for (Walk w(g); ok && w.next(g);) {
             // the next item of this CTA, when it is the next node of the same range
-            const int next_node = ((i + 1) % g.split_len != 0 && w.node + 1 < g.nodes) ? w.node + 1 : -1;
+            const int next_node = w.next_in_range();
             for (int t = w.t0; t < w.t1; ++t, ++q) {
                 const uint32_t ab = q & 1u, ph = (q >> 1) & 1u;
                 if (!mbar_wait(stage_ready + ab, ph)) { ok = false; break; }

@@ -58,7 +58,7 @@ cudaError_t launch(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap& map
 }
 
 template <bool PRECISE>
-cudaError_t launch_ring(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap& mapB, tcw::Args a) {
+cudaError_t launch_ring(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap& mapB, const CUtensorMap& mapX, tcw::Args a) {
     auto kernel = tcw::tc_wgrad_kernel<4, PRECISE, tcw::kRing, 0>;
     constexpr size_t smem = tcw::smem_bytes<4, PRECISE, false>();
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -71,7 +71,7 @@ cudaError_t launch_ring(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap
     a.chunks = a.n_tiles;
     choose_ranges(a, c->n, sms);
     const int grid = std::min(a.total_seqs, sms);                // one persistent CTA per SM
-    kernel<<<grid, tcw::kThreadsRing, smem, c->stream>>>(mapA, mapB, mapA, a);
+    kernel<<<grid, tcw::kThreadsRing, smem, c->stream>>>(mapA, mapB, mapX, a);
     c->launches++;
     return cudaGetLastError();
 }
@@ -114,14 +114,17 @@ cudaError_t run_tcw_ring(dpsgd_ctx* c, const float* h, int din, const float* del
     auto al = [](const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; };
     // w_off and din multiples of 4: the columns left to the mixing kernel are then whole groups of four
     if (!c->can_ring || !c->W.band || c->n < 3 || B > tcw::kMaxK || din % 4 != 0 || dpitch % 4 != 0 || w_off % 4 != 0 ||
-        !al(h) || !al(delta))
+        !al(h) || !al(delta) || !al(X + w_off) || c->ld % 4 != 0)
         return cudaErrorNotSupported;
     const uint64_t nodes = (uint64_t)c->n;
-    CUtensorMap mapA, mapB;
+    CUtensorMap mapA, mapB, mapX;
     bool ok = make_map_3d(&mapA, h, (uint64_t)din, (uint64_t)B, nodes, (uint64_t)din * 4, (uint64_t)B * din * 4,
                           tcw::kTileM, tcw::kMaxK, false);
     ok = ok && make_map_3d(&mapB, delta, (uint64_t)dout, (uint64_t)B, nodes, (uint64_t)dpitch * 4,
                            (uint64_t)B * dpitch * 4, 64u, tcw::kMaxK, false);
+    // this weight block of X as (input unit, output unit, node): the tile of X_{i+1} of every node step
+    ok = ok && make_map_3d(&mapX, X + w_off, (uint64_t)din, (uint64_t)dout, nodes, (uint64_t)din * 4, (uint64_t)c->ld * 4,
+                           tcw::kTileM, 64u, false);
     if (!ok) return cudaErrorNotSupported;
     tcw::Args a{};
     a.M = din; a.N = dout; a.K = B;
@@ -131,7 +134,7 @@ cudaError_t run_tcw_ring(dpsgd_ctx* c, const float* h, int din, const float* del
     a.mix.X = X; a.mix.Xn = Xn; a.mix.ld = c->ld; a.mix.ld_out = c->ld; a.mix.w_off = w_off;
     a.mix.row_ptr = c->W.row_ptr; a.mix.col = c->W.col; a.mix.val = c->W.val; a.mix.band = c->W.band;
     a.mix.ngamma = -c->gamma;
-    return c->mlp_precision == 0 ? launch_ring<true>(c, mapA, mapB, a) : launch_ring<false>(c, mapA, mapB, a);
+    return c->mlp_precision == 0 ? launch_ring<true>(c, mapA, mapB, mapX, a) : launch_ring<false>(c, mapA, mapB, mapX, a);
 }
 
 // Returns cudaErrorNotSupported when the shapes or alignments rule the kernel out (the caller then
