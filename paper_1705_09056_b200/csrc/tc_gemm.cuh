@@ -58,9 +58,9 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 // One poll of a phase.  The suspend-time hint lets the hardware park the thread until the phase completes (it is
-// woken at once) or the hint runs out, instead of returning after its short default slice: a thread that polls
-// in a tight loop keeps its SM partition's shared-memory queue busy, and the warps that share the partition
-// with a waiting single-thread role (MMA issuer, TMA issuer) then convert at half speed.
+// woken then) or the hint runs out, instead of returning after its short default slice.  Measured on the fused
+// weight-gradient kernel (22 warps, most of them waiting at any time): 4 % shorter per work item than tight polling,
+// which competes with the converting warps for their SM partition's issue slots and shared-memory queue.
 constexpr uint32_t kSuspendNs = 2000;
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;

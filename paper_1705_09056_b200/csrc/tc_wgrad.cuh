@@ -36,7 +36,10 @@
 //           the accumulator in its own layout and keep the tiles of X_{i-1} and X_i in tensor memory, so
 //           X is read from memory once: the tile of X_{i+1}, which the TMA thread fetches one to two
 //           nodes ahead into two shared-memory stages (no mixer thread waits on HBM, no registers
-//           hold loads in flight).  One column tile per item (the window holds one position).
+//           hold loads in flight).  One column tile per item (the window holds one position), hence
+//           one h tile AND one delta tile to convert per item: the four converter warps alone were the
+//           slowest stage (one warp per SM partition, ~500 dependent instructions per item), so here
+//           the mixer warps split the delta tile, one item ahead of the MMAs, two chunks per thread.
 //
 // One persistent CTA per SM; a work item is (node, 128-row block of m, run of column tiles).  Every
 // mbarrier wait is bounded; a wait that runs out raises the status word, the TMA thread waits
@@ -252,6 +255,9 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    // threads that split the delta tiles: the converter warps, or in kRing the sixteen mixer warps (the converters
+    // of a CTA with one h tile per column tile are the slowest stage otherwise)
+    constexpr uint32_t B_CONVERTERS = MODE == kRing ? 32u * kMixWarps : 128u;
     constexpr uint32_t A_BUFS = MODE == kRing ? 2u : 1u;     // raw h tiles in flight (a new one every column tile in kRing)
     const uint32_t a_raw = base;
     const uint32_t b_raw = a_raw + A_BUFS * A_RAW;
@@ -279,11 +285,11 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         for (uint32_t b = 0; b < A_BUFS; ++b) { mbar_init(a_raw_full + b, 1); mbar_init(a_raw_empty + b, 128); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(a_conv_full + b, 128); mbar_init(a_conv_empty + b, 1);
-            mbar_init(b_conv_full + b, 128); mbar_init(b_conv_empty + b, 1);
+            mbar_init(b_conv_full + b, B_CONVERTERS); mbar_init(b_conv_empty + b, 1);
             mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, MODE == kRing ? 16 : 128);
             mbar_init(stage_free + b, MODE == kStore ? 1 : 32 * kMixWarps); mbar_init(stage_ready + b, MODE == kRing ? 1 : 128);
         }
-        for (int s = 0; s < SB; ++s) { mbar_init(b_raw_full + s, 1); mbar_init(b_raw_empty + s, 128); }
+        for (int s = 0; s < SB; ++s) { mbar_init(b_raw_full + s, 1); mbar_init(b_raw_empty + s, B_CONVERTERS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 8) {
@@ -371,7 +377,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 mbar_arrive(a_conv_full + abuf);
                 mbar_arrive(a_raw_empty + rbuf);
             }
-            for (int t = w.t0; t < w.t1; ++t, ++q) {
+            for (int t = w.t0; MODE != kRing && t < w.t1; ++t, ++q) {
                 const uint32_t s = q % SB, bb = q & 1u;
                 if (!mbar_wait(b_raw_full + s, (q / SB) & 1u) || !mbar_wait(b_conv_empty + bb, ((q >> 1) & 1u) ^ 1u)) {
                     ok = false;
@@ -498,7 +504,35 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         const int b = (int)blockIdx.x, grid = (int)gridDim.x;
         const int rounds = b < g.total_seqs ? (g.total_seqs - b + grid - 1) / grid : 0;
         const int per_split = g.m_tiles * g.chunks;
+        uint32_t total_items = 0;
+        for (int rd = 0; rd < rounds; ++rd) {
+            const int n0 = ((b + rd * grid) / per_split) * g.split_len;
+            total_items += (uint32_t)max(0, min(g.nodes, n0 + g.split_len) - n0);
+        }
+        // The delta tile of item qb: raw [k][n] -> TF32 heads and remainders in the MMA's K-major layout, two
+        // 16-byte chunks (four samples of one output unit) per mixer thread.
+        const uint32_t mi = (uint32_t)(warp < 4 ? warp : warp - 6) * 32u + (uint32_t)lane;
+        auto convert_b = [&](uint32_t qb) -> bool {
+            const uint32_t s = qb % SB, bb = qb & 1u;
+            if (!mbar_wait(b_raw_full + s, (qb / SB) & 1u) || !mbar_wait(b_conv_empty + bb, ((qb >> 1) & 1u) ^ 1u)) return false;
+            const uint32_t rb = b_raw + s * B_RAW;
+            const uint32_t b_hi = b_conv + bb * CONV_BUF, b_lo = b_hi + B_CONV;
+#pragma unroll
+            for (uint32_t j = 0; j < (uint32_t)(ROWS_B * (kMaxK / 4)) / B_CONVERTERS; ++j) {
+                const uint32_t idx = mi + j * B_CONVERTERS;
+                const uint32_t n = idx % ROWS_B, c = idx / ROWS_B;
+                const uint32_t src = rb + (4 * c) * (ROWS_B * 4) + n * 4;
+                const float4 v = make_float4(lds32(src), lds32(src + ROWS_B * 4), lds32(src + 2 * ROWS_B * 4),
+                                             lds32(src + 3 * ROWS_B * 4));
+                tcs::put<PRECISE>(b_hi, b_lo, c * B_LBO + (n >> 3) * SBO + (n & 7) * 16, v);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_arrive(b_conv_full + bb);
+            mbar_arrive(b_raw_empty + s);
+            return true;
+        };
         uint32_t q = 0;
+        if (total_items > 0 && !convert_b(0)) ok = false;
         for (int rd = 0; rd < rounds && ok; ++rd) {
             // one node range at one tile position (decoded as in Walk; chunk == 1: one column tile)
             const int seq = b + rd * grid;
@@ -517,6 +551,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 float xr[16], tmp[16];
                 uint32_t bits[16];
                 const uint32_t jj = (uint32_t)(node - n0);
+                if (q + 1 < total_items && !convert_b(q + 1)) { ok = false; break; }     // one item ahead of the MMAs
                 // X_{i+1}: the one tile read from memory, staged by the TMA thread (zero outside the block)
                 {
                     const uint32_t xs = q & 1u;
