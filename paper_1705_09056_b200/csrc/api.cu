@@ -137,6 +137,7 @@ void release(dpsgd_ctx* c) {
     cudaFree(c->d_active);
     cudaFree(c->d_act);
     cudaFree(c->d_delta);
+    cudaFree(c->d_stream_parts);
     cudaFree(c->d_partials);
     cudaFree(c->d_conv_ws);
     cudaFree(c->d_result);
@@ -345,9 +346,9 @@ DPSGD_API dpsgd_status dpsgd_set_model(dpsgd_ctx* c, int32_t kind, const int32_t
     const dpsgd_status pending = c->bound ? collect_device_status(c) : DPSGD_OK;
     if (pending != DPSGD_OK) return pending;
     drop_graph(c);
-    cudaFree(c->d_idx); cudaFree(c->d_coef); cudaFree(c->d_act); cudaFree(c->d_delta);
+    cudaFree(c->d_idx); cudaFree(c->d_coef); cudaFree(c->d_act); cudaFree(c->d_delta); cudaFree(c->d_stream_parts);
     cudaFree(c->d_node_batch);
-    c->d_idx = nullptr; c->d_coef = nullptr; c->d_act = nullptr; c->d_delta = nullptr;
+    c->d_idx = nullptr; c->d_coef = nullptr; c->d_act = nullptr; c->d_delta = nullptr; c->d_stream_parts = nullptr;
     c->d_node_batch = nullptr;             // per-node sizes belong to the model they were set for
     c->model = kind; c->d = dims[0]; c->batch = batch; c->l2 = l2_lambda; c->mlp = shape;
     c->mlp_precision = mlp_precision;
@@ -358,6 +359,10 @@ DPSGD_API dpsgd_status dpsgd_set_model(dpsgd_ctx* c, int32_t kind, const int32_t
         c->delta_floats = mlp_delta_floats(c);
         e = cudaMalloc(&c->d_act, sizeof(float) * c->act_floats);
         if (e == cudaSuccess) e = cudaMalloc(&c->d_delta, sizeof(float) * c->delta_floats);
+        int sms = 0;
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
+        c->stream_parts_floats = mlp_stream_parts_floats(sms);
+        if (e == cudaSuccess) e = cudaMalloc(&c->d_stream_parts, sizeof(float) * c->stream_parts_floats);
     }
     if (e != cudaSuccess) { c->model = -1; return cuda_fail(c, e, "dpsgd_set_model allocation"); }
     return DPSGD_OK;

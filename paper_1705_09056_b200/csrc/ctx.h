@@ -93,6 +93,8 @@ struct dpsgd_ctx {
     float* d_act = nullptr;      // MLP activations h_0..h_L  (see grad_mlp.cu for the layout)
     float* d_delta = nullptr;    // MLP back-propagated errors
     size_t act_floats = 0, delta_floats = 0;
+    float* d_stream_parts = nullptr;   // MLP forward / input gradient: accumulators of tiles shared by two CTAs
+    size_t stream_parts_floats = 0;
     double* d_partials = nullptr;  // consensus partial sums, one per CTA
     int partials_cap = 0;
     dpsgd::ResultBlock* d_result = nullptr;  // final scalar + device status word
@@ -191,5 +193,6 @@ cudaError_t launch_tc_gemm_kmajor(dpsgd_ctx* c, const float* A, int64_t a_proble
                                   int M, int N, int K, int problems);
 size_t mlp_act_floats(const dpsgd_ctx* c);
 size_t mlp_delta_floats(const dpsgd_ctx* c);
+size_t mlp_stream_parts_floats(int sms);
 
 }  // namespace dpsgd

@@ -277,7 +277,7 @@ cudaError_t run_tc(dpsgd_ctx* c, tc::Args a, int max_tile, int problems = -1, bo
 // ---- weight-streaming kernel (tc_stream.cuh): forward and input-gradient products ----
 
 template <int NT, bool A_K, bool PRECISE>
-cudaError_t launch_tcs_inst(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap& mapB, const tcs::Args& a) {
+cudaError_t launch_tcs_inst(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtensorMap& mapB, tcs::Args a) {
     auto kernel = tcs::tc_stream_kernel<NT, A_K, PRECISE>;
     constexpr size_t smem = tcs::smem_bytes<NT, PRECISE>();
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -289,7 +289,15 @@ cudaError_t launch_tcs_inst(dpsgd_ctx* c, const CUtensorMap& mapA, const CUtenso
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     const int per_sm = NT <= 4 ? 2 : 1;                          // what the kernel's shared memory allows
     const int grid = std::min(a.total_tiles, sms * per_sm);      // persistent CTAs
+    // the tiles left over after the rounds that fill every CTA are cut by k-blocks and finished by stream_fixup_kernel
+    const int left_tiles = a.total_tiles % grid;
+    const bool cut = left_tiles != 0;
+    if (cut && (!c->d_stream_parts || (size_t)grid * 2 * 16 * NT * tcs::kTileM > c->stream_parts_floats)) return cudaErrorNotSupported;
+    a.partial = c->d_stream_parts;
     kernel<<<grid, tcs::kThreads, smem, c->stream>>>(mapA, mapB, a);
+    c->launches++;
+    if ((e = cudaGetLastError()) != cudaSuccess || !cut) return e;
+    tcs::stream_fixup_kernel<<<dim3(left_tiles, a.N), tcs::kTileM, 0, c->stream>>>(a, 16 * NT, grid);
     c->launches++;
     return cudaGetLastError();
 }
@@ -432,6 +440,9 @@ size_t mlp_act_floats(const dpsgd_ctx* c) {
     for (int l = 0; l <= c->mlp.nlayers; ++l) a += (size_t)c->n * c->batch * c->mlp.dims[l];
     return a;
 }
+
+// Scratch of the weight-streaming kernel: two 128 x 128 accumulator tiles per persistent CTA (two CTAs per SM).
+size_t mlp_stream_parts_floats(int sms) { return (size_t)sms * 2 * 2 * 128 * tcs::kTileM; }
 
 size_t mlp_delta_floats(const dpsgd_ctx* c) {
     size_t a = 0;

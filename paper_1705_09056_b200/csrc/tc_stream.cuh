@@ -27,9 +27,12 @@
 //   epilogue        the converter warps read the accumulator of a finished tile with tcgen05.ld and
 //                   store with m contiguous across lanes.
 //
-// CTAs are persistent (tile = blockIdx.x + i * gridDim.x over nodes x ceil(M/128)), so the loads of
-// the next tile are in flight while the current one is converted and drained; two CTAs share an SM
-// and cover each other's serial sections.  Out-of-range rows, columns and k are zero-filled by the
+// CTAs are persistent: tile = blockIdx.x + i * gridDim.x over nodes x ceil(M/128) for the rounds that fill
+// every CTA; the tiles left over after those rounds (1792 tiles on 296 CTAs: 16, which would cost a seventh
+// round for 0.05 rounds of work) are cut by k-blocks instead: their (tile, k-block) pairs form one sequence,
+// every CTA takes an equal part of it, writes the raw accumulator of each part to a scratch buffer, and
+// stream_fixup_kernel adds the parts of a tile in k order and applies the epilogue.  The loads of the next tile are in flight while
+// the current one is converted and drained; two CTAs share an SM and cover each other's serial sections.  Out-of-range rows, columns and k are zero-filled by the
 // TMA unit.  Every mbarrier wait is bounded; a wait that runs out raises the status word, the TMA
 // thread waits (bounded) for its loads in flight, and the CTA frees its TMEM columns before it
 // returns.
@@ -58,6 +61,38 @@ struct Args {
     int m_tiles, total_tiles;                                       // ceil(M/128), nodes * m_tiles
     int epi;
     int* status;
+    float* partial;          // [gridDim.x][2][16 NT][128]: accumulators of the tiles a CTA shares with a neighbour
+};
+
+// The work of a CTA, segment by segment: segment = (tile, k-blocks [kb0, kb1)).  First whole tiles, strided
+// (tile = cta + i * ctas for the rounds that fill every CTA: CTAs that run side by side then work on
+// neighbouring tiles of the same nodes and share their activations in L2); then the tiles left over
+// (fewer than ctas), whose k-blocks are dealt out evenly as one sequence, every CTA one contiguous range.
+struct Seg { int tile, kb0, kb1, slot; };     // slot: scratch slot of a left-over segment (0: first tile of the range, 1: a later one)
+struct SegWalk {
+    int i, rounds, KB, cta, ctas, first_left;
+    int u, u1, t_first;      // this CTA's range of the left-over k-blocks, the left-over tile it starts in
+    __device__ __forceinline__ SegWalk(int total_tiles, int KB_, unsigned cta_, unsigned ctas_)
+        : i(0), KB(KB_), cta((int)cta_), ctas((int)ctas_) {
+        rounds = total_tiles / ctas;
+        first_left = rounds * ctas;
+        const long long left = (long long)(total_tiles - first_left) * KB;
+        u = (int)(cta * left / ctas);
+        u1 = (int)((cta + 1) * left / ctas);
+        t_first = u / KB;
+    }
+    __device__ __forceinline__ bool next(Seg& s) {
+        if (i < rounds) {
+            s.tile = cta + i * ctas; s.kb0 = 0; s.kb1 = KB; s.slot = 0;
+            ++i;
+            return true;
+        }
+        if (u >= u1) return false;
+        const int t = u / KB, t0 = t * KB, end = min(t0 + KB, u1);
+        s.tile = first_left + t; s.kb0 = u - t0; s.kb1 = end - t0; s.slot = t == t_first ? 0 : 1;
+        u = end;
+        return true;
+    }
 };
 
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
@@ -188,10 +223,13 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
         bool ok = true;
         uint32_t q = 0, done_tiles = 0;
-        for (int tile = blockIdx.x; tile < g.total_tiles && ok; tile += gridDim.x, ++done_tiles) {
+        SegWalk walk(g.total_tiles, KB, blockIdx.x, gridDim.x);
+        Seg sg;
+        for (; ok && walk.next(sg); ++done_tiles) {
+            const int tile = sg.tile;
             const int node = tile / g.m_tiles;
             const int m0 = (tile - node * g.m_tiles) * kTileM;
-            for (int kb = 0; kb < KB; ++kb, ++q) {
+            for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++q) {
                 const uint32_t s = q % S, buf = q & 1u;
                 const bool landed = mbar_wait(raw_full + s, (q / S) & 1u) &&
                                     mbar_wait(conv_empty + buf, ((q >> 1) & 1u) ^ 1u);
@@ -241,6 +279,20 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             ok = __all_sync(0xffffffffu, ok);                   // tcgen05.ld below needs the whole warp
             if (!ok) break;
             tc::tc_fence_after();
+            if (sg.kb0 != 0 || sg.kb1 != KB) {
+                // part of a left-over tile: the raw accumulator goes to one of this CTA's two scratch slots
+                float* part = g.partial + ((int64_t)blockIdx.x * 2 + sg.slot) * (ROWS_B * kTileM) + tid;
+#pragma unroll 1
+                for (int c0 = 0; c0 < ROWS_B; c0 += 16) {
+                    if (c0 >= g.N) break;
+                    float v[16];
+                    tc::tmem_ld16(lane_base + (uint32_t)c0, v);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) part[(c0 + j) * kTileM] = v[j];
+                }
+                tc::tc_fence_before();
+                continue;
+            }
             const int m = m0 + warp * 32 + lane;
             float* C = g.C + (int64_t)node * g.c_node;
             const float* aux = g.aux ? g.aux + (int64_t)node * g.aux_node : nullptr;
@@ -278,9 +330,11 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                                    ((uint32_t)(kTileM >> 4) << 24);
             bool ok = true;
             uint32_t q = 0;
-            for (int tile = blockIdx.x; tile < g.total_tiles && ok; tile += gridDim.x) {
-                uint32_t acc = 0;                               // the first MMA of a tile overwrites the accumulator
-                for (int kb = 0; kb < KB; ++kb, ++q) {
+            SegWalk walk(g.total_tiles, KB, blockIdx.x, gridDim.x);
+            Seg sg;
+            while (ok && walk.next(sg)) {
+                uint32_t acc = 0;                               // the first MMA of a segment overwrites the accumulator
+                for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++q) {
                     const uint32_t buf = q & 1u;
                     if (!mbar_wait(conv_full + buf, (q >> 1) & 1u)) { ok = false; break; }
                     tc::tc_fence_after();
@@ -307,10 +361,12 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         // ------------------------------ TMA issuer ------------------------------
         bool ok = true;
         uint32_t q = 0;
-        for (int tile = blockIdx.x; tile < g.total_tiles && ok; tile += gridDim.x) {
-            const int node = tile / g.m_tiles;
-            const int m0 = (tile - node * g.m_tiles) * kTileM;
-            for (int kb = 0; kb < KB; ++kb, ++q) {
+        SegWalk walk(g.total_tiles, KB, blockIdx.x, gridDim.x);
+        Seg sg;
+        while (ok && walk.next(sg)) {
+            const int node = sg.tile / g.m_tiles;
+            const int m0 = (sg.tile - node * g.m_tiles) * kTileM;
+            for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++q) {
                 const uint32_t s = q % S;
                 if (!mbar_wait(raw_empty + s, ((q / S) & 1u) ^ 1u)) { ok = false; break; }
                 const uint32_t ra = base + s * RAW;
@@ -331,6 +387,59 @@ tc_stream_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     __syncthreads();
     if (warp == 4) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// Adds the parts of every left-over tile (in k order) and applies the epilogue.  One CTA per (left-over tile,
+// sample), thread = row of the tile.  rows = 16 NT of the stream kernel, ctas = its grid.
+static __global__ void __launch_bounds__(kTileM)
+stream_fixup_kernel(Args g, int rows, int ctas) {
+    const int KB = (g.K + kBK - 1) / kBK;
+    const int first_left = (g.total_tiles / ctas) * ctas;
+    const long long left = (long long)(g.total_tiles - first_left) * KB;
+    const int t = (int)blockIdx.x, tile = first_left + t;
+    const int t0 = t * KB, t1 = t0 + KB;
+    auto start = [&](int bb) { return (int)(bb * left / ctas); };     // first left-over k-block of stream CTA bb
+    int bb0 = (int)((long long)t0 * ctas / left);                     // the CTA whose range holds k-block t0
+    while (bb0 > 0 && start(bb0) > t0) --bb0;
+    while (bb0 + 1 < ctas && start(bb0 + 1) <= t0) ++bb0;
+    if (start(bb0) <= t0 && start(bb0 + 1) >= t1) return;             // one CTA ran the whole tile and finished it
+    const int node = tile / g.m_tiles;
+    const int m = (tile - node * g.m_tiles) * kTileM + (int)threadIdx.x;
+    if (m >= g.M) return;
+    float* C = g.C + (int64_t)node * g.c_node + m;
+    const float* aux = g.aux ? g.aux + (int64_t)node * g.aux_node : nullptr;
+    const int n = (int)blockIdx.y;                                    // one sample (column of the tile) per CTA
+    const float* part = g.partial + n * kTileM + threadIdx.x;
+    const int64_t pstride = (int64_t)2 * rows * kTileM;               // from one CTA's slot 0 to the next CTA's
+    float s;
+    if (left >= ctas) {
+        // no range is empty: the parts are those of CTAs bb0 .. bb1 - 1, all but possibly the first in slot 0,
+        // and their loads do not depend on one another
+        int bb1 = (int)(((long long)t1 * ctas + left - 1) / left);   // first CTA whose range starts at or after t1
+        while (bb1 > bb0 + 1 && start(bb1 - 1) >= t1) --bb1;
+        while (bb1 < ctas && start(bb1) < t1) ++bb1;
+        s = __ldcg(part + bb0 * pstride + (start(bb0) >= t0 ? 0 : rows * kTileM));
+#pragma unroll 8
+        for (int bb = bb0 + 1; bb < bb1; ++bb) s += __ldcg(part + bb * pstride);
+    } else {
+        // start(bb + 1) from start(bb) without a division: floor(bb * left / ctas) grows by 0 or 1
+        const int r = (int)left;
+        int u0 = start(bb0), err = (int)((long long)bb0 * left % ctas);
+        s = 0.f;
+        for (int bb = bb0; bb < ctas && u0 < t1; ++bb) {              // the CTAs whose ranges meet this tile, in k order
+            int u1 = u0;
+            err += r;
+            if (err >= ctas) { err -= ctas; ++u1; }
+            if (u1 > u0 && u1 > t0) s += __ldcg(part + bb * pstride + (u0 >= t0 ? 0 : rows * kTileM));
+            u0 = u1;
+        }
+    }
+    if (g.epi == tc::EPI_MASK) {
+        C[(int64_t)n * g.c_pitch] = __ldg(aux + (int64_t)n * g.aux_pitch + m) > 0.f ? s : 0.f;
+    } else {
+        const float x = s + (g.epi <= tc::EPI_BIAS ? __ldg(aux + m) : 0.f);
+        C[(int64_t)n * g.c_pitch] = (g.epi == tc::EPI_BIAS_RELU && x < 0.f) ? 0.f : x;
     }
 }
 

@@ -185,7 +185,7 @@ def test_config5_full_size_fused_step_on_column_slices():
     ctx.set_fused_step(1)
     before = ctx.launch_count()
     ctx.step(k)
-    assert ctx.launch_count() - before == 14
+    assert ctx.launch_count() - before == 17         # 14 kernels of the iteration + one fix-up per streamed product
     out = ctx.current()
     assert bool(torch.isfinite(out).all())
     for s in starts:

@@ -37,6 +37,9 @@ MLP_CASES = [
     (2, (1024, 2048, 2048, 10), 96, 64),     # the large network, two nodes
     (3, (130, 70, 3), 33, 1),                # minibatch of one
     (2, (128, 256, 128, 64, 10), 40, 24),    # four weight layers
+    # more row blocks than persistent CTAs: the blocks left over after the full rounds are cut by k-blocks
+    (80, (40, 512, 256, 10), 24, 8),         # fewer left-over k-blocks than CTAs (some CTAs get none)
+    (100, (96, 640, 10), 24, 8),             # ranges of two k-blocks that cross row blocks of three
 ]
 
 
