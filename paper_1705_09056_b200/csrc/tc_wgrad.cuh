@@ -482,8 +482,8 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         // Thread = (row m of the tile, 16 of its 64 columns): the accumulator's own layout, so a tile needs
         // no staging.  The CTA walks consecutive nodes i at one tile position; the tiles of X_{i-1} and X_i
         // are kept in two 64-column slots of tensor memory (each thread's own lane and columns: no
-        // synchronisation), so only X_{i+1} is read from memory - one read of X per element - after an L2
-        // prefetch two nodes ahead.
+        // synchronisation), so only X_{i+1} is read from memory - one read of X per element - from the
+        // shared-memory stage that the TMA thread filled one to two nodes ahead.
         // sixteen warps: lane quarter warp % 4 (the lanes a warp may address), column group by warp:
         // 0-3 -> 0, 12-15 -> 1, 16-19 -> 2, {20, 21, 10, 11} -> 3
         const int quarter = warp & 3, cg = warp < 4 ? 0 : (warp < 12 || warp >= 20 ? 3 : ((warp - 12) >> 2) + 1);
