@@ -60,21 +60,30 @@ conv_bias_grad_kernel(const float* __restrict__ dym, float* __restrict__ G, int6
 }
 
 // U[img][k = (c,kh,kw)][p = (i,j)] = x[img][c][s i + kh - 1][s j + kw - 1], zero outside the image.
+// Block (px, 256 / px): threadIdx.x walks the positions, VEC consecutive ones of an output row per thread (VEC = 4
+// when the output width is a multiple of 4: one 16-byte store), threadIdx.y the taps; grid (position chunks, tap
+// groups, images).
+template <int VEC>
 __global__ void __launch_bounds__(256)
-conv_unfold_kernel(const float* __restrict__ x, float* __restrict__ U, int64_t total, int c_in, int h, int w, int ho,
-                   int wo, int stride) {
-    const int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x;
-    if (t >= total) return;
-    const int pos = ho * wo, kc = 9 * c_in;
-    const int64_t img = t / ((int64_t)kc * pos);
-    const int r = (int)(t - img * (int64_t)kc * pos);
-    const int k = r / pos, q = r - k * pos;
+conv_unfold_kernel(const float* __restrict__ x, float* __restrict__ U, int c_in, int h, int w, int ho, int wo, int stride) {
+    const int pos = ho * wo;
+    const int q = (blockIdx.x * blockDim.x + threadIdx.x) * VEC;
+    const int k = blockIdx.y * blockDim.y + threadIdx.y;
+    if (q >= pos || k >= 9 * c_in) return;
     const int c = k / 9, tap = k - 9 * c, kh = tap / 3, kw = tap - 3 * kh;
+    const int64_t img = blockIdx.z;
     const int i = q / wo, j = q - i * wo;
-    const int hh = stride * i + kh - 1, ww = stride * j + kw - 1;
-    float v = 0.f;
-    if (hh >= 0 && hh < h && ww >= 0 && ww < w) v = __ldg(x + ((img * c_in + c) * (int64_t)h + hh) * w + ww);
-    U[t] = v;
+    const int hh = stride * i + kh - 1;
+    const float* row = x + ((img * c_in + c) * (int64_t)h + hh) * w;
+    float v[VEC];
+#pragma unroll
+    for (int u = 0; u < VEC; ++u) {
+        const int ww = stride * (j + u) + kw - 1;
+        v[u] = (hh >= 0 && hh < h && ww >= 0 && ww < w) ? __ldg(row + ww) : 0.f;
+    }
+    float* dst = U + (img * (9 * c_in) + k) * (int64_t)pos + q;
+    if (VEC == 4) *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1 % VEC], v[2 % VEC], v[3 % VEC]);
+    else dst[0] = v[0];
 }
 
 // G[node][w_off + e] = sum_b P[node][b][e], images added in order.
@@ -146,8 +155,16 @@ cudaError_t launch_conv3x3_backward(dpsgd_ctx* c, const float* x, const float* y
     const int64_t total = imgs * c_out * pos;
     conv_mask_kernel<<<blocks(total), 256, 0, c->stream>>>(dy, relu ? y : nullptr, dym, spread, total, pos, wo, h, w);
     conv_bias_grad_kernel<<<dim3(c_out, n), 256, 0, c->stream>>>(dym, c->G, c->ld, b_off, batch, c_out, pos);
-    const int64_t utotal = imgs * kc * pos;
-    conv_unfold_kernel<<<blocks(utotal), 256, 0, c->stream>>>(x, unf, utotal, c_in, h, w, ho, wo, stride);
+    {
+        const int vec = wo % 4 == 0 ? 4 : 1;                 // then pos % 4 == 0 too and every store is 16-byte aligned
+        const int chunks = (pos + vec - 1) / vec;
+        int px = 1;
+        while (px < chunks && px < 256) px *= 2;
+        const dim3 block((unsigned)px, (unsigned)(256 / px));
+        const dim3 grid((unsigned)((chunks + px - 1) / px), (unsigned)((kc + block.y - 1) / block.y), (unsigned)imgs);
+        if (vec == 4) conv_unfold_kernel<4><<<grid, block, 0, c->stream>>>(x, unf, c_in, h, w, ho, wo, stride);
+        else conv_unfold_kernel<1><<<grid, block, 0, c->stream>>>(x, unf, c_in, h, w, ho, wo, stride);
+    }
     c->launches += 3;
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     // per image: par[o][k] = sum_p unf[k][p] * dym[o][p]
