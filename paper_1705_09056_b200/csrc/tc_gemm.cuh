@@ -59,7 +59,7 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 }
 // One poll of a phase.  The suspend-time hint lets the hardware park the thread until the phase completes (it is
 // woken then) or the hint runs out, instead of returning after its short default slice.  Measured on the fused
-// weight-gradient kernel (22 warps, most of them waiting at any time): 4 % shorter per work item than tight polling,
+// weight-gradient kernel (two dozen warps, most of them waiting at any time): 4 % shorter per work item than tight polling,
 // which competes with the converting warps for their SM partition's issue slots and shared-memory queue.
 constexpr uint32_t kSuspendNs = 2000;
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {

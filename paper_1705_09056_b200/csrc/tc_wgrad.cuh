@@ -37,9 +37,10 @@
 //           X is read from memory once: the tile of X_{i+1}, which the TMA thread fetches one to two
 //           nodes ahead into two shared-memory stages (no mixer thread waits on HBM, no registers
 //           hold loads in flight).  One column tile per item (the window holds one position), hence
-//           one h tile AND one delta tile to convert per item: the four converter warps alone were the
-//           slowest stage (one warp per SM partition, ~500 dependent instructions per item), so here
-//           the mixer warps split the delta tile, one item ahead of the MMAs, two chunks per thread.
+//           one h tile AND one delta tile to convert per item: four converter warps alone were the
+//           slowest stage (one warp per SM partition, ~500 dependent instructions per item), and the
+//           mixers' chain of dependent steps per item is the next slowest, so the delta tiles are split
+//           by four warps of their own (26 warps, 72 registers).
 //
 // One persistent CTA per SM; a work item is (node, 128-row block of m, run of column tiles).  Every
 // mbarrier wait is bounded; a wait that runs out raises the status word, the TMA thread waits
@@ -62,7 +63,7 @@ using tcs::tma_load_3d;
 constexpr int kThreads = 320;        // 4 epilogue warps, 4 converter warps, MMA warp, TMA warp
 constexpr int kMixWarps = 16;        // kGather: warps 10..25 apply the gossip step to staged tiles
 constexpr int kThreadsFused = kThreads + 32 * kMixWarps;
-constexpr int kThreadsRing = 704;    // kRing: converters, MMA, TMA as above; warps 0-3 and 10-21 mix
+constexpr int kThreadsRing = 832;    // kRing: converters (h), MMA, TMA as above; warps 0-3 and 10-21 mix; warps 22-25 split delta
 enum { kStore = 0, kGather = 1, kRing = 2 };
 constexpr int kTileM = 128;
 constexpr int kMaxK = 64;            // minibatch rows a raw tile holds
@@ -257,7 +258,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     // threads that split the delta tiles: the converter warps, or in kRing the sixteen mixer warps (the converters
     // of a CTA with one h tile per column tile are the slowest stage otherwise)
-    constexpr uint32_t B_CONVERTERS = MODE == kRing ? 32u * kMixWarps : 128u;
+    constexpr uint32_t B_CONVERTERS = 128u;
     constexpr uint32_t A_BUFS = MODE == kRing ? 2u : 1u;     // raw h tiles in flight (a new one every column tile in kRing)
     const uint32_t a_raw = base;
     const uint32_t b_raw = a_raw + A_BUFS * A_RAW;
@@ -402,6 +403,35 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         }
         if (!ok && lane == 0) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
     }
+    else if (MODE == kRing && warp >= 22) {
+        // ------------------------------ kRing: delta converters ------------------------------
+        // With one h tile AND one delta tile per item the four converter warps are the slowest stage, and the
+        // mixers' chain per item is the next slowest, so the delta tiles get four warps of their own.
+        const uint32_t ct = (uint32_t)tid - 704u;
+        uint32_t q = 0;
+        for (Walk w(g); ok && w.next(g); ++q) {
+            const uint32_t s = q % SB, bb = q & 1u;
+            if (!mbar_wait(b_raw_full + s, (q / SB) & 1u) || !mbar_wait(b_conv_empty + bb, ((q >> 1) & 1u) ^ 1u)) {
+                ok = false;
+                break;
+            }
+            const uint32_t rb = b_raw + s * B_RAW;
+            const uint32_t b_hi = b_conv + bb * CONV_BUF, b_lo = b_hi + B_CONV;
+#pragma unroll
+            for (uint32_t j = 0; j < (uint32_t)(ROWS_B * (kMaxK / 4)) / 128u; ++j) {
+                const uint32_t idx = ct + j * 128u;
+                const uint32_t n = idx % ROWS_B, c = idx / ROWS_B;      // output unit, 16-byte chunk (four k)
+                const uint32_t src = rb + (4 * c) * (ROWS_B * 4) + n * 4;
+                const float4 v = make_float4(lds32(src), lds32(src + ROWS_B * 4), lds32(src + 2 * ROWS_B * 4),
+                                             lds32(src + 3 * ROWS_B * 4));
+                tcs::put<PRECISE>(b_hi, b_lo, c * B_LBO + (n >> 3) * SBO + (n & 7) * 16, v);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_arrive(b_conv_full + bb);
+            mbar_arrive(b_raw_empty + s);
+        }
+        if (!ok && lane == 0) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
+    }
     else if (warp == 8) {
         if (lane == 0) {
             // ------------------------------ MMA issuer ------------------------------
@@ -477,7 +507,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         }
         if (!ok) atomicExch(g.status, (int)DPSGD_ERR_TIMEOUT);
     }
-    if (MODE == kRing && (warp < 4 || warp >= 10)) {
+    if (MODE == kRing && (warp < 4 || (warp >= 10 && warp < 22))) {
         // ------------------------------ ring mixers: X window in tensor memory ------------------------------
         // Thread = (row m of the tile, 16 of its 64 columns): the accumulator's own layout, so a tile needs
         // no staging.  The CTA walks consecutive nodes i at one tile position; the tiles of X_{i-1} and X_i
@@ -504,35 +534,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         const int b = (int)blockIdx.x, grid = (int)gridDim.x;
         const int rounds = b < g.total_seqs ? (g.total_seqs - b + grid - 1) / grid : 0;
         const int per_split = g.m_tiles * g.chunks;
-        uint32_t total_items = 0;
-        for (int rd = 0; rd < rounds; ++rd) {
-            const int n0 = ((b + rd * grid) / per_split) * g.split_len;
-            total_items += (uint32_t)max(0, min(g.nodes, n0 + g.split_len) - n0);
-        }
-        // The delta tile of item qb: raw [k][n] -> TF32 heads and remainders in the MMA's K-major layout, two
-        // 16-byte chunks (four samples of one output unit) per mixer thread.
-        const uint32_t mi = (uint32_t)(warp < 4 ? warp : warp - 6) * 32u + (uint32_t)lane;
-        auto convert_b = [&](uint32_t qb) -> bool {
-            const uint32_t s = qb % SB, bb = qb & 1u;
-            if (!mbar_wait(b_raw_full + s, (qb / SB) & 1u) || !mbar_wait(b_conv_empty + bb, ((qb >> 1) & 1u) ^ 1u)) return false;
-            const uint32_t rb = b_raw + s * B_RAW;
-            const uint32_t b_hi = b_conv + bb * CONV_BUF, b_lo = b_hi + B_CONV;
-#pragma unroll
-            for (uint32_t j = 0; j < (uint32_t)(ROWS_B * (kMaxK / 4)) / B_CONVERTERS; ++j) {
-                const uint32_t idx = mi + j * B_CONVERTERS;
-                const uint32_t n = idx % ROWS_B, c = idx / ROWS_B;
-                const uint32_t src = rb + (4 * c) * (ROWS_B * 4) + n * 4;
-                const float4 v = make_float4(lds32(src), lds32(src + ROWS_B * 4), lds32(src + 2 * ROWS_B * 4),
-                                             lds32(src + 3 * ROWS_B * 4));
-                tcs::put<PRECISE>(b_hi, b_lo, c * B_LBO + (n >> 3) * SBO + (n & 7) * 16, v);
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            mbar_arrive(b_conv_full + bb);
-            mbar_arrive(b_raw_empty + s);
-            return true;
-        };
         uint32_t q = 0;
-        if (total_items > 0 && !convert_b(0)) ok = false;
         for (int rd = 0; rd < rounds && ok; ++rd) {
             // one node range at one tile position (decoded as in Walk; chunk == 1: one column tile)
             const int seq = b + rd * grid;
@@ -551,7 +553,6 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 float xr[16], tmp[16];
                 uint32_t bits[16];
                 const uint32_t jj = (uint32_t)(node - n0);
-                if (q + 1 < total_items && !convert_b(q + 1)) { ok = false; break; }     // one item ahead of the MMAs
                 // X_{i+1}: the one tile read from memory, staged by the TMA thread (zero outside the block)
                 {
                     const uint32_t xs = q & 1u;
